@@ -1,0 +1,194 @@
+/*
+ * knnssd - decode hot path of KNN-SSD self-speculative decoding on one NVIDIA B200.
+ *
+ * C ABI of libknnssd.so.  Plain pointers and sizes only; every pointer is marked
+ * HOST or DEVICE below.  All functions return a knnssd_status (0 = OK); on any
+ * non-OK status the session (context length, KV cache validity, active skip mask)
+ * is left as it was before the call, nothing aborts or throws across the boundary,
+ * and knnssd_last_error() gives a one-line reason.  A context is bound to the CUDA
+ * device that was current at knnssd_init and to the stream passed there; calls on
+ * one context must not overlap (not thread-safe per context).
+ *
+ * Notation follows the paper: L decoder layers = 2L sublayers; a skip mask
+ * z in {0,1}^{2L} with z[j] = 1 meaning "sublayer j is skipped while drafting"
+ * (Sec. 3.1; Sec. 4.1), index 2l = attention sublayer of layer l, 2l+1 = its MLP
+ * sublayer; A_i = {a_i1..a_ik} the anchors of domain i (Sec. 4.1, Eq. (2));
+ * k = draft length.
+ *
+ * Session protocol:  init -> prefill -> (select_skipset | set_skipmask)
+ *                    -> { draft -> verify }* ;  generate = all of it for one request.
+ */
+#ifndef KNNSSD_H
+#define KNNSSD_H
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct knnssd_ctx knnssd_ctx; /* opaque: model view + session state */
+
+typedef enum {
+    KNNSSD_OK = 0,
+    KNNSSD_ERR_INVALID_ARG = 1, /* NULL pointer, negative size, token id out of range, k > max_draft ... */
+    KNNSSD_ERR_SHAPE = 2,       /* configuration the kernels do not support (see knnssd_init) */
+    KNNSSD_ERR_CAPACITY = 3,    /* context would exceed max_seq */
+    KNNSSD_ERR_STATE = 4,       /* call out of protocol order (e.g. draft before prefill / before a mask is set) */
+    KNNSSD_ERR_DEGENERATE = 5,  /* zero or non-finite vector in the cosine search */
+    KNNSSD_ERR_CUDA = 6,        /* a CUDA runtime call failed; text in knnssd_last_error */
+    KNNSSD_ERR_TIMEOUT = 7      /* reserved: a bounded device-side wait gave up */
+} knnssd_status;
+
+typedef struct {
+    int n_layers, d_model, n_heads, n_kv_heads, head_dim, d_ff, vocab;
+    int max_seq;            /* KV-cache capacity in positions */
+    int max_draft;          /* largest k accepted by draft/verify/generate (1..15) */
+    float rms_eps, rope_theta;
+    int dtype;              /* 0: fp32 weights and KV cache; 1: bf16 weights and KV cache */
+    int n_domains;          /* number of domains (may be 0: no anchors, masks set explicitly) */
+    int anchors_per_domain; /* anchors per domain */
+    int pool_mode;          /* 0: mean of the prompt's last-layer hidden states; 1: last position only */
+} knnssd_config;
+
+/* All DEVICE pointers, row-major [out][in], borrowed for the lifetime of the context
+ * (the library makes no packed copy; the caller keeps them alive and unchanged).
+ * Big matrices are fp32 or bf16 per knnssd_config.dtype; norm gains are always fp32.
+ * The per-layer tables themselves are HOST arrays of n_layers DEVICE pointers. */
+typedef struct {
+    const void *tok_embed;         /* [vocab][d_model] */
+    const float *final_norm;       /* [d_model] */
+    const void *lm_head;           /* [vocab][d_model] */
+    const float *const *attn_norm; /* [d_model] */
+    const void *const *wq;         /* [n_heads*head_dim][d_model] */
+    const void *const *wk;         /* [n_kv_heads*head_dim][d_model] */
+    const void *const *wv;         /* [n_kv_heads*head_dim][d_model] */
+    const void *const *wo;         /* [d_model][n_heads*head_dim] */
+    const float *const *mlp_norm;  /* [d_model] */
+    const void *const *w_gate;     /* [d_ff][d_model] */
+    const void *const *w_up;       /* [d_ff][d_model] */
+    const void *const *w_down;     /* [d_model][d_ff] */
+} knnssd_weights;
+
+typedef struct {
+    int rounds;    /* draft+verify rounds run */
+    int drafted;   /* draft steps taken (sum of k_eff) */
+    int accepted;  /* draft tokens accepted */
+    int tokens;    /* tokens emitted */
+    float ms_prefill, ms_select, ms_draft, ms_verify; /* device time (CUDA events on the context's stream) */
+} knnssd_stats;
+
+/*
+ * Create a context for one model and one request at a time.
+ *   cfg, w            HOST structs (copied).  Supported: head_dim in {64, 128}, n_heads % n_kv_heads == 0,
+ *                     d_model, d_ff, n_heads*head_dim multiples of 8; else KNNSSD_ERR_SHAPE.
+ *   anchors_dev       DEVICE fp32 [n_domains*anchors_per_domain][d_model], borrowed; NULL iff n_domains == 0.
+ *                     Anchors need not be normalised; a zero or non-finite anchor -> KNNSSD_ERR_DEGENERATE.
+ *   skip_masks_host   HOST bytes [n_domains][2*n_layers], the stored per-domain masks z*_i (Sec. 4.1, Eq. (3)),
+ *                     copied; NULL iff n_domains == 0.
+ *   cuda_stream       a cudaStream_t (NULL = default stream); every kernel of this context runs on it.
+ * The context owns the KV cache ([n_layers][n_kv_heads][max_seq][head_dim], K and V) and its work buffers.
+ */
+knnssd_status knnssd_init(const knnssd_config *cfg, const knnssd_weights *w, const float *anchors_dev,
+                          const unsigned char *skip_masks_host, void *cuda_stream, knnssd_ctx **out);
+void knnssd_destroy(knnssd_ctx *ctx);
+
+/*
+ * Run the full model over the prompt (Sec. 4.2: the new sample's last hidden vector comes from a pass of the
+ * model over it): fills the KV cache for positions [0, n_tokens), keeps the pooled last-layer hidden state
+ * (after the final RMSNorm) for select_skipset, and makes the greedy token after the prompt the pending token.
+ *   tokens_host          HOST int32 [n_tokens], 1 <= n_tokens <= max_seq - 1
+ *   pooled_dev_or_null   DEVICE fp32 [d_model]: receives the pooled vector; may be NULL
+ *   first_token_or_null  HOST int: receives the pending token; may be NULL
+ * Resets the session (length, statistics) first; the active mask is kept.
+ */
+knnssd_status knnssd_prefill(knnssd_ctx *ctx, const int *tokens_host, int n_tokens, float *pooled_dev_or_null,
+                             int *first_token_or_null);
+
+/*
+ * Domain choice (Sec. 4.2, Eq. (4)): (i*, j*) = argmax_{i,j} cos(v, a_ij), lowest flat index on ties, then the
+ * stored mask of domain i* becomes the active one.
+ *   query_dev_or_null  DEVICE fp32 [d_model]; NULL = the pooled vector of the last prefill
+ *   domain, anchor, cosine   HOST outputs (each may be NULL)
+ * KNNSSD_ERR_DEGENERATE if the query has zero or non-finite norm; KNNSSD_ERR_STATE without anchors.
+ */
+knnssd_status knnssd_select_skipset(knnssd_ctx *ctx, const float *query_dev_or_null, int *domain, int *anchor,
+                                    float *cosine);
+
+/* Make an explicit mask active.  mask_host: HOST bytes [2*n_layers], 1 = skipped while drafting. */
+knnssd_status knnssd_set_skipmask(knnssd_ctx *ctx, const unsigned char *mask_host);
+
+/*
+ * Draft k tokens greedily with M(z), z the active mask (Sec. 4.2, drafting equation): step j feeds the pending
+ * token (j = 0) or draft j-1 at position len+j through the retained sublayers only - skipped sublayers read no
+ * weights and write no K/V - and takes the arg-max (lowest id on ties).
+ *   k                  1 <= k <= max_draft, len + k + 1 <= max_seq
+ *   draft_tokens_host  HOST int32 [k] output
+ *   logits_dev_or_null DEVICE fp32 [k][vocab]: the draft model's logits per step; may be NULL
+ * Does not change the committed length; K/V rows it writes are scratch until verify rewrites them.
+ */
+knnssd_status knnssd_draft(knnssd_ctx *ctx, int k, int *draft_tokens_host, float *logits_dev_or_null);
+
+/*
+ * Verify k drafted tokens with the full model in ONE pass over the k+1 rows [pending, d_0 .. d_{k-1}] at positions
+ * len .. len+k (Sec. 4.2, verification paragraph), accept the longest prefix on which the full model's greedy
+ * token equals the draft, emit the full model's own token after it, and commit len += n_accepted + 1 (rows beyond
+ * are rolled back: dead and overwritten later).  k = 0 is a plain one-token step of the full model.
+ *   draft_tokens_host   HOST int32 [k] (any tokens: need not come from knnssd_draft); may be NULL iff k == 0
+ *   n_accepted, next_token   HOST outputs; next_token becomes the pending token
+ *   logits_dev_or_null  DEVICE fp32 [k+1][vocab] full-model logits of the rows; may be NULL
+ *   hidden_dev_or_null  DEVICE fp32 [k+1][d_model] last-layer hidden states after the final RMSNorm; may be NULL
+ */
+knnssd_status knnssd_verify(knnssd_ctx *ctx, const int *draft_tokens_host, int k, int *n_accepted, int *next_token,
+                            float *logits_dev_or_null, float *hidden_dev_or_null);
+
+/*
+ * One request end to end: prefill, select_skipset (only if the context has anchors AND use_selection != 0;
+ * otherwise the active mask is used and must have been set), then rounds of draft + verify until exactly max_new
+ * tokens are out.  Each round drafts k_eff = min(k, remaining - 1) tokens, so the last round never overshoots.
+ *   prompt_host HOST int32 [n_prompt];  out_tokens_host HOST int32 [max_new] output;  n_out HOST output
+ *   accepts_host_or_null HOST int32 [max_new]: accepted count of each round (first stats.rounds entries)
+ *   domain_or_null HOST output (-1 when no selection ran);  stats_or_null HOST output
+ */
+knnssd_status knnssd_generate(knnssd_ctx *ctx, const int *prompt_host, int n_prompt, int max_new, int k,
+                              int use_selection, int *out_tokens_host, int *n_out, int *accepts_host_or_null,
+                              int *domain_or_null, knnssd_stats *stats_or_null);
+
+/* Committed context length (positions whose K/V are valid), and explicit rollback to a shorter length
+ * (new_len <= current length; the pending token is unchanged, so this is meant for tests and benchmarks). */
+int knnssd_get_length(const knnssd_ctx *ctx);
+knnssd_status knnssd_set_length(knnssd_ctx *ctx, int new_len);
+/* Replace the pending token (HOST value); lets a caller teacher-force a token stream. */
+knnssd_status knnssd_set_pending(knnssd_ctx *ctx, int token);
+
+knnssd_status knnssd_get_stats(const knnssd_ctx *ctx, knnssd_stats *out);
+const char *knnssd_last_error(const knnssd_ctx *ctx);
+
+/*
+ * Device-time measurement of the two passes at the current length, for benchmarks: runs `iters` draft passes of one
+ * step each (or verify passes over k+1 rows) without committing anything, bracketed by CUDA events on the context's
+ * stream, and returns the mean milliseconds per pass.  which: 0 = draft step, 1 = verify pass over k+1 rows.
+ * Also returns how many kernels one such pass launches and the mean device milliseconds spent per pass inside the
+ * weight-streaming linear kernels alone (events around each of them in a separate, untimed replay).
+ */
+knnssd_status knnssd_time_pass(knnssd_ctx *ctx, int which, int k, int iters, float *ms_per_pass,
+                               int *launches_per_pass, float *ms_linear_per_pass, int *linear_launches_per_pass);
+
+/* ---- stand-alone operators (same kernels the passes use; for per-kernel tests and measurements) ---- */
+
+/*
+ * y[m][o] = sum_i W[o][i] * x[m][i] for m < M <= 16: the weight-streaming linear kernel.
+ *   W DEVICE [n_out][n_in] (dtype as above), x DEVICE fp32 [M][n_in], y DEVICE fp32 [M][n_out]; n_in % 8 == 0.
+ */
+knnssd_status knnssd_linear(const void *W_dev, int dtype, int n_out, int n_in, const float *x_dev, int M,
+                            float *y_dev, void *cuda_stream);
+
+/*
+ * Cosine top-1 (Sec. 4.2, Eq. (4)) of one query against n anchors of dimension d, all DEVICE fp32; HOST outputs.
+ * KNNSSD_ERR_DEGENERATE for a zero / non-finite query or anchor.
+ */
+knnssd_status knnssd_cosine_top1(const float *query_dev, const float *anchors_dev, int n, int d, int *best,
+                                 float *cosine, void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KNNSSD_H */

@@ -57,6 +57,7 @@ def lib():
         _lib.orc_set_len.argtypes = [C.c_void_p, C.c_int]
         _lib.orc_forward.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p,
                                      C.c_void_p, C.c_void_p, C.c_void_p, C.c_int]
+        _lib.orc_linear.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_int, C.c_void_p]
         _lib.orc_pool_mean.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p]
         _lib.orc_knn_select.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
                                         C.POINTER(C.c_int), C.POINTER(C.c_int), C.POINTER(C.c_float)]
@@ -169,6 +170,17 @@ class OracleModel:
         if rc:
             raise ValueError(f"orc_greedy_full rc={rc}")
         return out, mm.value
+
+
+def linear(W: torch.Tensor, x: np.ndarray) -> np.ndarray:
+    """y = x . W^T with fp64 accumulation; W a CPU torch tensor (fp32 or bf16) [n_out][n_in], x fp32 [M][n_in]."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    M, n_in = x.shape
+    n_out = W.shape[0]
+    assert W.shape[1] == n_in and M <= 64
+    y = np.zeros((M, n_out), dtype=np.float32)
+    lib().orc_linear(_ptr(W), 0 if W.dtype == torch.float32 else 1, n_out, n_in, _ptr(x), M, _ptr(y))
+    return y
 
 
 def pool_mean(hidden: np.ndarray) -> np.ndarray:

@@ -103,6 +103,11 @@ static void linear(const void *W, int dtype, int n_out, int n_in, const float *x
     }
 }
 
+/* The linear map on its own, for per-kernel checks: y [M][n_out] = x [M][n_in] . W^T. */
+void orc_linear(const void *W, int dtype, int n_out, int n_in, const float *x, int M, float *y) {
+    linear(W, dtype, n_out, n_in, x, M, y);
+}
+
 /* RMSNorm: h = x * rsqrt(mean(x^2) + eps) * g */
 static void rmsnorm(const float *x, const float *g, int d, float eps, float *h) {
     double ss = 0.0;

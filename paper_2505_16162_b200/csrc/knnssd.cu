@@ -1,0 +1,700 @@
+// Host side of libknnssd.so: the C ABI declared in include/knnssd.h, the session state and the
+// sequencing of one decoder pass (which sublayers run, on how many rows, at which positions).
+// Every step of the path runs in the kernels of kernels.cuh; the host only enqueues them.
+#include "../../include/knnssd.h"
+#include "kernels.cuh"
+
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+using namespace knnssd;
+
+namespace {
+
+constexpr int kMaxRows = 16;       // most rows one pass carries (prefill chunk; verify uses k+1 <= 16)
+constexpr int kArgmaxBlocks = 64;  // slices per row in the arg-max
+
+struct Layer {
+    const float *attn_norm, *mlp_norm;
+    const void *wq, *wk, *wv, *wo, *w_gate, *w_up, *w_down;
+};
+
+}  // namespace
+
+struct knnssd_ctx {
+    knnssd_config cfg{};
+    std::vector<Layer> layers;
+    const void *tok_embed = nullptr, *lm_head = nullptr;
+    const float *final_norm = nullptr;
+    const float *anchors = nullptr;
+    std::vector<unsigned char> domain_masks;  // [n_domains][2L]
+    std::vector<unsigned char> active_mask;   // [2L]
+    bool has_mask = false, prefilled = false;
+    cudaStream_t stream = nullptr;
+    int device = 0, n_sms = 148;
+    size_t wbytes = 2;
+
+    // device buffers (owned)
+    void *kcache = nullptr, *vcache = nullptr;
+    float *x = nullptr, *qkv = nullptr, *attn = nullptr, *act = nullptr, *logits = nullptr, *hfinal = nullptr;
+    float *part_o = nullptr, *pooled = nullptr, *anchor_inv_norm = nullptr, *cosines = nullptr, *amax_v = nullptr;
+    float2 *part_ml = nullptr, *rope_cs = nullptr;
+    double *pool_sum = nullptr, *inv_freq = nullptr;
+    int *chain = nullptr, *target = nullptr, *prompt = nullptr, *out_tokens = nullptr, *accept_log = nullptr;
+    int *amax_i = nullptr, *flag = nullptr, *knn_out = nullptr;
+    DeviceState *state = nullptr;
+    int *pinned = nullptr;  // host, pinned: small read-backs
+    int n_splits = 1;
+
+    // host mirror of the session
+    int len = 0, pending = -1;
+    knnssd_stats stats{};
+    cudaEvent_t ev0 = nullptr, ev1 = nullptr, ev2 = nullptr;
+    std::string err;
+
+    // instrumentation
+    long long launches = 0;
+    bool time_linear = false;
+    std::vector<cudaEvent_t> lin_events;
+    size_t lin_used = 0;
+};
+
+namespace {
+
+knnssd_status fail(knnssd_ctx *c, knnssd_status s, const std::string &msg) {
+    if (c) c->err = msg;
+    return s;
+}
+
+#define CUDA_TRY(ctx, expr)                                                                          \
+    do {                                                                                             \
+        cudaError_t e_ = (expr);                                                                     \
+        if (e_ != cudaSuccess)                                                                       \
+            return fail(ctx, KNNSSD_ERR_CUDA, std::string(#expr) + ": " + cudaGetErrorString(e_));   \
+    } while (0)
+
+template <typename T> cudaError_t dev_alloc(T **p, size_t count) {
+    return cudaMalloc(reinterpret_cast<void **>(p), count * sizeof(T));
+}
+
+int pick_mt(int M) {
+    static const int opts[] = {1, 2, 3, 4, 5, 6, 7, 8, 9, 16};
+    for (int o : opts)
+        if (M <= o) return o;
+    return -1;
+}
+
+template <typename WT> void launch_linear_t(const LinearArgs &a, int grid, cudaStream_t s) {
+    switch (pick_mt(a.M)) {
+        case 1: linear_kernel<WT, 1><<<grid, 256, 0, s>>>(a); break;
+        case 2: linear_kernel<WT, 2><<<grid, 256, 0, s>>>(a); break;
+        case 3: linear_kernel<WT, 3><<<grid, 256, 0, s>>>(a); break;
+        case 4: linear_kernel<WT, 4><<<grid, 256, 0, s>>>(a); break;
+        case 5: linear_kernel<WT, 5><<<grid, 256, 0, s>>>(a); break;
+        case 6: linear_kernel<WT, 6><<<grid, 256, 0, s>>>(a); break;
+        case 7: linear_kernel<WT, 7><<<grid, 256, 0, s>>>(a); break;
+        case 8: linear_kernel<WT, 8><<<grid, 256, 0, s>>>(a); break;
+        case 9: linear_kernel<WT, 9><<<grid, 256, 0, s>>>(a); break;
+        default: linear_kernel<WT, 16><<<grid, 256, 0, s>>>(a); break;
+    }
+}
+
+void launch_linear(int dtype, const LinearArgs &a, int n_sms, cudaStream_t s) {
+    // enough warps that every SM holds 8 blocks of 8 warps, but never more warps than units
+    long long blocks = (long long)n_sms * 8;
+    const long long max_blocks = (a.units + 7) / 8;
+    if (blocks > max_blocks) blocks = max_blocks;
+    if (blocks < 1) blocks = 1;
+    if (dtype) launch_linear_t<bf16_t>(a, (int)blocks, s); else launch_linear_t<float>(a, (int)blocks, s);
+}
+
+void ctx_linear(knnssd_ctx *c, const LinearArgs &a) {
+    if (c->time_linear) {
+        if (c->lin_used + 2 > c->lin_events.size()) {
+            for (int i = 0; i < 2; ++i) {
+                cudaEvent_t e;
+                cudaEventCreate(&e);
+                c->lin_events.push_back(e);
+            }
+        }
+        cudaEventRecord(c->lin_events[c->lin_used], c->stream);
+    }
+    launch_linear(c->cfg.dtype, a, c->n_sms, c->stream);
+    if (c->time_linear) {
+        cudaEventRecord(c->lin_events[c->lin_used + 1], c->stream);
+        c->lin_used += 2;
+    }
+    c->launches++;
+}
+
+LinearArgs make_args(const void *W0, int rows0, int n_in, const float *x, const float *gain, float eps, float *y,
+                     int epi, int M) {
+    LinearArgs a{};
+    a.W[0] = W0; a.rows[0] = rows0; a.units = rows0; a.n_in = n_in; a.x = x; a.gain = gain; a.eps = eps; a.y = y;
+    a.epi = epi; a.M = M;
+    return a;
+}
+
+// One decoder pass over M rows whose token ids are tok_dev[0..M) at positions state.len + pos_off + m.
+//   mask       nullptr = full model, else [2L] with 1 = skipped
+//   head_row0  first row that gets logits and an arg-max (M = no head at all)
+//   argmax_out device ints, entry (m - head_row0) receives row m's greedy token
+//   want_hidden  also write RMSNorm_final(x) of all rows to c->hfinal
+template <typename WT>
+void run_pass_t(knnssd_ctx *c, int M, const int *tok_dev, int pos_off, const unsigned char *mask, int head_row0,
+                int *argmax_out, bool want_hidden) {
+    const knnssd_config &g = c->cfg;
+    const int d = g.d_model, H = g.n_heads, Hkv = g.n_kv_heads, hd = g.head_dim, F = g.d_ff, V = g.vocab;
+    const int nq = H * hd, nkv = Hkv * hd;
+    cudaStream_t s = c->stream;
+    embed_rope_kernel<WT><<<M, 256, 0, s>>>(reinterpret_cast<const WT *>(c->tok_embed), tok_dev, d, c->x, c->state, pos_off,
+                                            c->inv_freq, hd / 2, c->rope_cs);
+    c->launches++;
+    const size_t layer_stride = (size_t)Hkv * g.max_seq * hd;
+    for (int l = 0; l < g.n_layers; ++l) {
+        const Layer &ly = c->layers[l];
+        if (!mask || !mask[2 * l]) {
+            LinearArgs a = make_args(ly.wq, nq, d, c->x, ly.attn_norm, g.rms_eps, c->qkv, EPI_STORE, M);
+            a.W[1] = ly.wk; a.rows[1] = nkv; a.W[2] = ly.wv; a.rows[2] = nkv; a.units = nq + 2 * nkv;
+            ctx_linear(c, a);
+            WT *kc = reinterpret_cast<WT *>(c->kcache) + (size_t)l * layer_stride;
+            WT *vc = reinterpret_cast<WT *>(c->vcache) + (size_t)l * layer_stride;
+            rope_kv_kernel<WT><<<dim3(H + 2 * Hkv, M), hd / 2, 0, s>>>(c->qkv, H, Hkv, hd, c->rope_cs, kc, vc, g.max_seq,
+                                                                      c->state, pos_off);
+            const dim3 ag(H, M, c->n_splits);
+            if (hd == 128) {
+                attn_partial_kernel<WT, 128><<<ag, 128, 0, s>>>(c->qkv, H, Hkv, kc, vc, g.max_seq, c->state, pos_off,
+                                                                 c->part_o, c->part_ml, c->n_splits);
+                attn_merge_kernel<128><<<dim3(H, M), 128, 0, s>>>(c->part_o, c->part_ml, H, c->state, pos_off, c->n_splits,
+                                                                   c->attn);
+            } else {
+                attn_partial_kernel<WT, 64><<<ag, 128, 0, s>>>(c->qkv, H, Hkv, kc, vc, g.max_seq, c->state, pos_off,
+                                                                c->part_o, c->part_ml, c->n_splits);
+                attn_merge_kernel<64><<<dim3(H, M), 64, 0, s>>>(c->part_o, c->part_ml, H, c->state, pos_off, c->n_splits,
+                                                                 c->attn);
+            }
+            c->launches += 3;
+            ctx_linear(c, make_args(ly.wo, d, nq, c->attn, nullptr, 0.f, c->x, EPI_ADD, M));
+        }
+        if (!mask || !mask[2 * l + 1]) {
+            LinearArgs a = make_args(ly.w_gate, F, d, c->x, ly.mlp_norm, g.rms_eps, c->act, EPI_SWIGLU, M);
+            a.W[1] = ly.w_up; a.rows[1] = F; a.units = F;
+            ctx_linear(c, a);
+            ctx_linear(c, make_args(ly.w_down, d, F, c->act, nullptr, 0.f, c->x, EPI_ADD, M));
+        }
+    }
+    if (want_hidden) {
+        rmsnorm_rows_kernel<<<M, 256, 0, s>>>(c->x, c->final_norm, d, g.rms_eps, c->hfinal);
+        c->launches++;
+    }
+    if (head_row0 < M) {
+        const int hm = M - head_row0;
+        ctx_linear(c, make_args(c->lm_head, V, d, c->x + (size_t)head_row0 * d, c->final_norm, g.rms_eps,
+                                c->logits + (size_t)head_row0 * V, EPI_STORE, hm));
+        argmax_partial_kernel<<<dim3(kArgmaxBlocks, hm), 256, 0, s>>>(c->logits + (size_t)head_row0 * V, V, kArgmaxBlocks,
+                                                                      c->amax_v, c->amax_i);
+        argmax_final_kernel<<<hm, 32, 0, s>>>(c->amax_v, c->amax_i, kArgmaxBlocks, argmax_out);
+        c->launches += 2;
+    }
+}
+
+void run_pass(knnssd_ctx *c, int M, const int *tok_dev, int pos_off, const unsigned char *mask, int head_row0,
+              int *argmax_out, bool want_hidden) {
+    if (c->cfg.dtype) run_pass_t<bf16_t>(c, M, tok_dev, pos_off, mask, head_row0, argmax_out, want_hidden);
+    else run_pass_t<float>(c, M, tok_dev, pos_off, mask, head_row0, argmax_out, want_hidden);
+}
+
+knnssd_status sync_check(knnssd_ctx *c, const char *what) {
+    cudaError_t e = cudaStreamSynchronize(c->stream);
+    if (e == cudaSuccess) e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(c, KNNSSD_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
+    return KNNSSD_OK;
+}
+
+void free_all(knnssd_ctx *c) {
+    void *ptrs[] = {c->kcache, c->vcache, c->x, c->qkv, c->attn, c->act, c->logits, c->hfinal, c->part_o, c->pooled,
+                    c->anchor_inv_norm, c->cosines, c->amax_v, c->part_ml, c->rope_cs, c->pool_sum, c->inv_freq, c->chain,
+                    c->target, c->prompt, c->out_tokens, c->accept_log, c->amax_i, c->flag, c->knn_out, c->state};
+    for (void *p : ptrs)
+        if (p) cudaFree(p);
+    if (c->pinned) cudaFreeHost(c->pinned);
+    if (c->ev0) cudaEventDestroy(c->ev0);
+    if (c->ev1) cudaEventDestroy(c->ev1);
+    if (c->ev2) cudaEventDestroy(c->ev2);
+    for (cudaEvent_t e : c->lin_events) cudaEventDestroy(e);
+}
+
+struct DeviceGuard {
+    int prev = 0;
+    explicit DeviceGuard(int dev) { cudaGetDevice(&prev); if (prev != dev) cudaSetDevice(dev); else prev = -1; }
+    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+float elapsed_ms(knnssd_ctx *c) {
+    float ms = 0.f;
+    cudaEventElapsedTime(&ms, c->ev0, c->ev1);
+    return ms;
+}
+
+knnssd_status do_prefill(knnssd_ctx *c, const int *tokens_host, int n, float *pooled_dev, int *first_token) {
+    const knnssd_config &g = c->cfg;
+    if (!tokens_host || n < 1) return fail(c, KNNSSD_ERR_INVALID_ARG, "prefill: need at least one prompt token");
+    if (n > g.max_seq - 1) return fail(c, KNNSSD_ERR_CAPACITY, "prefill: prompt does not fit in max_seq - 1");
+    for (int i = 0; i < n; ++i)
+        if (tokens_host[i] < 0 || tokens_host[i] >= g.vocab)
+            return fail(c, KNNSSD_ERR_INVALID_ARG, "prefill: token id out of range");
+    cudaStream_t s = c->stream;
+    c->prefilled = false;
+    CUDA_TRY(c, cudaMemcpyAsync(c->prompt, tokens_host, sizeof(int) * n, cudaMemcpyHostToDevice, s));
+    set_state_kernel<<<1, 1, 0, s>>>(c->state, 0, 0);
+    cudaEventRecord(c->ev0, s);
+    const int d = g.d_model;
+    for (int t0 = 0; t0 < n; t0 += kMaxRows) {
+        const int M = (n - t0 < kMaxRows) ? n - t0 : kMaxRows;
+        const bool last = t0 + M == n;
+        // mean pooling needs every row's final hidden state; last-token pooling only the last row's
+        const bool hidden = g.pool_mode == 0 || last;
+        run_pass(c, M, c->prompt + t0, t0, nullptr, last ? M - 1 : M, c->chain, hidden);
+        if (g.pool_mode == 0) {
+            pool_accumulate_kernel<<<(d + 255) / 256, 256, 0, s>>>(c->hfinal, M, d, c->pool_sum, t0 == 0);
+        } else if (last) {
+            pool_accumulate_kernel<<<(d + 255) / 256, 256, 0, s>>>(c->hfinal + (size_t)(M - 1) * d, 1, d, c->pool_sum, 1);
+        }
+    }
+    pool_finish_kernel<<<(d + 255) / 256, 256, 0, s>>>(c->pool_sum, d, g.pool_mode == 0 ? 1.0 / (double)n : 1.0, c->pooled);
+    emit_first_token_kernel<<<1, 1, 0, s>>>(c->chain, c->state, c->out_tokens, n);
+    cudaEventRecord(c->ev1, s);
+    if (pooled_dev) CUDA_TRY(c, cudaMemcpyAsync(pooled_dev, c->pooled, sizeof(float) * d, cudaMemcpyDeviceToDevice, s));
+    CUDA_TRY(c, cudaMemcpyAsync(c->pinned, c->chain, sizeof(int), cudaMemcpyDeviceToHost, s));
+    knnssd_status st = sync_check(c, "prefill");
+    if (st != KNNSSD_OK) return st;
+    c->len = n;
+    c->pending = c->pinned[0];
+    c->prefilled = true;
+    c->stats = knnssd_stats{};
+    c->stats.tokens = 1;
+    c->stats.ms_prefill = elapsed_ms(c);
+    if (first_token) *first_token = c->pending;
+    return KNNSSD_OK;
+}
+
+knnssd_status do_select(knnssd_ctx *c, const float *query_dev, int *domain, int *anchor, float *cosine) {
+    const knnssd_config &g = c->cfg;
+    if (g.n_domains <= 0) return fail(c, KNNSSD_ERR_STATE, "select_skipset: the context has no anchors");
+    if (!query_dev && !c->prefilled) return fail(c, KNNSSD_ERR_STATE, "select_skipset: no pooled vector (prefill first)");
+    const int n = g.n_domains * g.anchors_per_domain;
+    cudaStream_t s = c->stream;
+    CUDA_TRY(c, cudaMemsetAsync(c->flag, 0, sizeof(int), s));
+    cudaEventRecord(c->ev0, s);
+    cosine_scores_kernel<<<(n + 7) / 8, 256, 0, s>>>(query_dev ? query_dev : c->pooled, c->anchors, c->anchor_inv_norm, n,
+                                                     g.d_model, c->cosines, c->flag);
+    cosine_argmax_kernel<<<1, 256, 0, s>>>(c->cosines, n, c->knn_out);
+    cudaEventRecord(c->ev1, s);
+    CUDA_TRY(c, cudaMemcpyAsync(c->pinned, c->knn_out, 2 * sizeof(int), cudaMemcpyDeviceToHost, s));
+    CUDA_TRY(c, cudaMemcpyAsync(c->pinned + 2, c->flag, sizeof(int), cudaMemcpyDeviceToHost, s));
+    knnssd_status st = sync_check(c, "select_skipset");
+    if (st != KNNSSD_OK) return st;
+    if (c->pinned[2]) return fail(c, KNNSSD_ERR_DEGENERATE, "select_skipset: query has zero or non-finite norm");
+    const int best = c->pinned[0];
+    float cs;
+    std::memcpy(&cs, &c->pinned[1], sizeof(float));
+    const int dom = best / g.anchors_per_domain;
+    c->active_mask.assign(c->domain_masks.begin() + (size_t)dom * 2 * g.n_layers,
+                          c->domain_masks.begin() + (size_t)(dom + 1) * 2 * g.n_layers);
+    c->has_mask = true;
+    c->stats.ms_select = elapsed_ms(c);
+    if (domain) *domain = dom;
+    if (anchor) *anchor = best % g.anchors_per_domain;
+    if (cosine) *cosine = cs;
+    return KNNSSD_OK;
+}
+
+// Enqueue k draft steps: step j reads chain[j] at position len + j and writes chain[j + 1].
+void enqueue_draft(knnssd_ctx *c, int k) {
+    for (int j = 0; j < k; ++j) run_pass(c, 1, c->chain + j, j, c->active_mask.data(), 0, c->chain + j + 1, false);
+}
+
+// Enqueue the verification pass over chain[0..k] and the accept/rollback step.
+void enqueue_verify(knnssd_ctx *c, int k, bool want_hidden, int round_idx) {
+    run_pass(c, k + 1, c->chain, 0, nullptr, 0, c->target, want_hidden);
+    accept_kernel<<<1, 32, 0, c->stream>>>(c->chain, c->target, k, c->state, c->out_tokens, c->cfg.max_seq, c->accept_log,
+                                           round_idx);
+    c->launches++;
+}
+
+}  // namespace
+
+extern "C" {
+
+knnssd_status knnssd_init(const knnssd_config *cfg, const knnssd_weights *w, const float *anchors_dev,
+                          const unsigned char *skip_masks_host, void *cuda_stream, knnssd_ctx **out) {
+    if (!cfg || !w || !out) return KNNSSD_ERR_INVALID_ARG;
+    *out = nullptr;
+    const knnssd_config &g = *cfg;
+    if (g.n_layers < 1 || g.d_model < 8 || g.n_heads < 1 || g.n_kv_heads < 1 || g.d_ff < 8 || g.vocab < 2 ||
+        g.max_seq < 2 || g.max_draft < 1 || g.n_domains < 0 || (g.n_domains > 0 && g.anchors_per_domain < 1) ||
+        (g.dtype != 0 && g.dtype != 1) || (g.pool_mode != 0 && g.pool_mode != 1) || !(g.rms_eps > 0.f) ||
+        !(g.rope_theta > 0.f))
+        return KNNSSD_ERR_INVALID_ARG;
+    if ((g.head_dim != 64 && g.head_dim != 128) || g.n_heads % g.n_kv_heads != 0 || g.d_model % 8 != 0 ||
+        g.d_ff % 8 != 0 || g.max_draft > kMaxRows - 1)
+        return KNNSSD_ERR_SHAPE;
+    if ((g.n_domains > 0) != (anchors_dev != nullptr) || (g.n_domains > 0) != (skip_masks_host != nullptr))
+        return KNNSSD_ERR_INVALID_ARG;
+    if (!w->tok_embed || !w->final_norm || !w->lm_head || !w->attn_norm || !w->wq || !w->wk || !w->wv || !w->wo ||
+        !w->mlp_norm || !w->w_gate || !w->w_up || !w->w_down)
+        return KNNSSD_ERR_INVALID_ARG;
+    knnssd_ctx *c = new (std::nothrow) knnssd_ctx();
+    if (!c) return KNNSSD_ERR_CUDA;
+    c->cfg = g;
+    c->stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+    c->wbytes = g.dtype ? 2 : 4;
+    c->tok_embed = w->tok_embed; c->final_norm = w->final_norm; c->lm_head = w->lm_head;
+    for (int l = 0; l < g.n_layers; ++l) {
+        Layer ly{w->attn_norm[l], w->mlp_norm[l], w->wq[l], w->wk[l], w->wv[l], w->wo[l], w->w_gate[l], w->w_up[l],
+                 w->w_down[l]};
+        const void *all[] = {ly.attn_norm, ly.mlp_norm, ly.wq, ly.wk, ly.wv, ly.wo, ly.w_gate, ly.w_up, ly.w_down};
+        for (const void *p : all)
+            if (!p || (reinterpret_cast<uintptr_t>(p) & 15u)) { delete c; return KNNSSD_ERR_INVALID_ARG; }
+        c->layers.push_back(ly);
+    }
+    if ((reinterpret_cast<uintptr_t>(w->tok_embed) & 15u) || (reinterpret_cast<uintptr_t>(w->lm_head) & 15u) ||
+        (reinterpret_cast<uintptr_t>(w->final_norm) & 15u)) { delete c; return KNNSSD_ERR_INVALID_ARG; }
+    c->anchors = anchors_dev;
+    const int L2 = 2 * g.n_layers;
+    if (g.n_domains > 0) {
+        c->domain_masks.assign(skip_masks_host, skip_masks_host + (size_t)g.n_domains * L2);
+        for (unsigned char b : c->domain_masks)
+            if (b > 1) { delete c; return KNNSSD_ERR_INVALID_ARG; }
+    }
+    auto bail = [&](knnssd_status s) { free_all(c); delete c; return s; };
+    if (cudaGetDevice(&c->device) != cudaSuccess) return bail(KNNSSD_ERR_CUDA);
+    cudaDeviceGetAttribute(&c->n_sms, cudaDevAttrMultiProcessorCount, c->device);
+    const int d = g.d_model, hd = g.head_dim, nq = g.n_heads * hd, nkv = g.n_kv_heads * hd;
+    const size_t cache_elems = (size_t)g.n_layers * g.n_kv_heads * g.max_seq * hd;
+    c->n_splits = (g.max_seq + ATT_CHUNK - 1) / ATT_CHUNK;
+    const int na = g.n_domains * g.anchors_per_domain;
+    bool ok = true;
+    ok &= cudaMalloc(&c->kcache, cache_elems * c->wbytes) == cudaSuccess;
+    ok &= cudaMalloc(&c->vcache, cache_elems * c->wbytes) == cudaSuccess;
+    ok &= dev_alloc(&c->x, (size_t)kMaxRows * d) == cudaSuccess;
+    ok &= dev_alloc(&c->qkv, (size_t)kMaxRows * (nq + 2 * nkv)) == cudaSuccess;
+    ok &= dev_alloc(&c->attn, (size_t)kMaxRows * nq) == cudaSuccess;
+    ok &= dev_alloc(&c->act, (size_t)kMaxRows * g.d_ff) == cudaSuccess;
+    ok &= dev_alloc(&c->logits, (size_t)kMaxRows * g.vocab) == cudaSuccess;
+    ok &= dev_alloc(&c->hfinal, (size_t)kMaxRows * d) == cudaSuccess;
+    ok &= dev_alloc(&c->part_o, (size_t)kMaxRows * g.n_heads * c->n_splits * hd) == cudaSuccess;
+    ok &= dev_alloc(&c->part_ml, (size_t)kMaxRows * g.n_heads * c->n_splits) == cudaSuccess;
+    ok &= dev_alloc(&c->rope_cs, (size_t)kMaxRows * (hd / 2)) == cudaSuccess;
+    ok &= dev_alloc(&c->pooled, (size_t)d) == cudaSuccess;
+    ok &= dev_alloc(&c->pool_sum, (size_t)d) == cudaSuccess;
+    ok &= dev_alloc(&c->inv_freq, (size_t)hd / 2) == cudaSuccess;
+    ok &= dev_alloc(&c->amax_v, (size_t)kMaxRows * kArgmaxBlocks) == cudaSuccess;
+    ok &= dev_alloc(&c->amax_i, (size_t)kMaxRows * kArgmaxBlocks) == cudaSuccess;
+    ok &= dev_alloc(&c->chain, (size_t)kMaxRows + 1) == cudaSuccess;
+    ok &= dev_alloc(&c->target, (size_t)kMaxRows) == cudaSuccess;
+    ok &= dev_alloc(&c->prompt, (size_t)g.max_seq) == cudaSuccess;
+    ok &= dev_alloc(&c->out_tokens, (size_t)g.max_seq) == cudaSuccess;
+    ok &= dev_alloc(&c->accept_log, (size_t)g.max_seq) == cudaSuccess;
+    ok &= dev_alloc(&c->flag, 1) == cudaSuccess;
+    ok &= dev_alloc(&c->knn_out, 2) == cudaSuccess;
+    ok &= dev_alloc(&c->state, 1) == cudaSuccess;
+    ok &= dev_alloc(&c->cosines, (size_t)(na > 0 ? na : 1)) == cudaSuccess;
+    ok &= dev_alloc(&c->anchor_inv_norm, (size_t)(na > 0 ? na : 1)) == cudaSuccess;
+    ok &= cudaMallocHost(reinterpret_cast<void **>(&c->pinned), 64 * sizeof(int)) == cudaSuccess;
+    ok &= cudaEventCreate(&c->ev0) == cudaSuccess && cudaEventCreate(&c->ev1) == cudaSuccess &&
+          cudaEventCreate(&c->ev2) == cudaSuccess;
+    if (!ok) { cudaGetLastError(); return bail(KNNSSD_ERR_CUDA); }
+    // K/V start at zero so that no kernel ever reads uninitialised memory
+    cudaMemsetAsync(c->kcache, 0, cache_elems * c->wbytes, c->stream);
+    cudaMemsetAsync(c->vcache, 0, cache_elems * c->wbytes, c->stream);
+    std::vector<double> inv_freq(hd / 2);
+    for (int i = 0; i < hd / 2; ++i) inv_freq[i] = std::pow((double)g.rope_theta, -2.0 * (double)i / (double)hd);
+    cudaMemcpyAsync(c->inv_freq, inv_freq.data(), sizeof(double) * inv_freq.size(), cudaMemcpyHostToDevice, c->stream);
+    set_state_kernel<<<1, 1, 0, c->stream>>>(c->state, 0, 0);
+    cudaMemsetAsync(c->flag, 0, sizeof(int), c->stream);
+    if (na > 0) anchor_inv_norm_kernel<<<(na + 7) / 8, 256, 0, c->stream>>>(c->anchors, na, d, c->anchor_inv_norm, c->flag);
+    cudaMemcpyAsync(c->pinned, c->flag, sizeof(int), cudaMemcpyDeviceToHost, c->stream);
+    if (sync_check(c, "init") != KNNSSD_OK) return bail(KNNSSD_ERR_CUDA);
+    if (c->pinned[0]) return bail(KNNSSD_ERR_DEGENERATE);
+    *out = c;
+    return KNNSSD_OK;
+}
+
+void knnssd_destroy(knnssd_ctx *c) {
+    if (!c) return;
+    DeviceGuard dg(c->device);
+    cudaStreamSynchronize(c->stream);
+    free_all(c);
+    delete c;
+}
+
+knnssd_status knnssd_prefill(knnssd_ctx *c, const int *tokens_host, int n_tokens, float *pooled_dev_or_null,
+                             int *first_token_or_null) {
+    if (!c) return KNNSSD_ERR_INVALID_ARG;
+    DeviceGuard dg(c->device);
+    return do_prefill(c, tokens_host, n_tokens, pooled_dev_or_null, first_token_or_null);
+}
+
+knnssd_status knnssd_select_skipset(knnssd_ctx *c, const float *query_dev_or_null, int *domain, int *anchor,
+                                    float *cosine) {
+    if (!c) return KNNSSD_ERR_INVALID_ARG;
+    DeviceGuard dg(c->device);
+    return do_select(c, query_dev_or_null, domain, anchor, cosine);
+}
+
+knnssd_status knnssd_set_skipmask(knnssd_ctx *c, const unsigned char *mask_host) {
+    if (!c) return KNNSSD_ERR_INVALID_ARG;
+    if (!mask_host) return fail(c, KNNSSD_ERR_INVALID_ARG, "set_skipmask: NULL mask");
+    const int n = 2 * c->cfg.n_layers;
+    for (int j = 0; j < n; ++j)
+        if (mask_host[j] > 1) return fail(c, KNNSSD_ERR_INVALID_ARG, "set_skipmask: entries must be 0 or 1");
+    c->active_mask.assign(mask_host, mask_host + n);
+    c->has_mask = true;
+    return KNNSSD_OK;
+}
+
+knnssd_status knnssd_draft(knnssd_ctx *c, int k, int *draft_tokens_host, float *logits_dev_or_null) {
+    if (!c) return KNNSSD_ERR_INVALID_ARG;
+    DeviceGuard dg(c->device);
+    if (!draft_tokens_host || k < 1 || k > c->cfg.max_draft) return fail(c, KNNSSD_ERR_INVALID_ARG, "draft: bad k or NULL output");
+    if (!c->prefilled) return fail(c, KNNSSD_ERR_STATE, "draft: prefill first");
+    if (!c->has_mask) return fail(c, KNNSSD_ERR_STATE, "draft: no active skip mask (select_skipset or set_skipmask first)");
+    if (c->len + k + 1 > c->cfg.max_seq) return fail(c, KNNSSD_ERR_CAPACITY, "draft: len + k + 1 exceeds max_seq");
+    cudaStream_t s = c->stream;
+    cudaEventRecord(c->ev0, s);
+    for (int j = 0; j < k; ++j) {
+        run_pass(c, 1, c->chain + j, j, c->active_mask.data(), 0, c->chain + j + 1, false);
+        if (logits_dev_or_null)
+            CUDA_TRY(c, cudaMemcpyAsync(logits_dev_or_null + (size_t)j * c->cfg.vocab, c->logits, sizeof(float) * c->cfg.vocab,
+                                        cudaMemcpyDeviceToDevice, s));
+    }
+    cudaEventRecord(c->ev1, s);
+    CUDA_TRY(c, cudaMemcpyAsync(c->pinned, c->chain + 1, sizeof(int) * k, cudaMemcpyDeviceToHost, s));
+    knnssd_status st = sync_check(c, "draft");
+    if (st != KNNSSD_OK) return st;
+    for (int j = 0; j < k; ++j) draft_tokens_host[j] = c->pinned[j];
+    c->stats.ms_draft += elapsed_ms(c);
+    return KNNSSD_OK;
+}
+
+knnssd_status knnssd_verify(knnssd_ctx *c, const int *draft_tokens_host, int k, int *n_accepted, int *next_token,
+                            float *logits_dev_or_null, float *hidden_dev_or_null) {
+    if (!c) return KNNSSD_ERR_INVALID_ARG;
+    DeviceGuard dg(c->device);
+    const knnssd_config &g = c->cfg;
+    if (k < 0 || k > g.max_draft || (k > 0 && !draft_tokens_host)) return fail(c, KNNSSD_ERR_INVALID_ARG, "verify: bad k or NULL drafts");
+    if (!c->prefilled) return fail(c, KNNSSD_ERR_STATE, "verify: prefill first");
+    if (c->len + k + 1 > g.max_seq) return fail(c, KNNSSD_ERR_CAPACITY, "verify: len + k + 1 exceeds max_seq");
+    for (int j = 0; j < k; ++j)
+        if (draft_tokens_host[j] < 0 || draft_tokens_host[j] >= g.vocab)
+            return fail(c, KNNSSD_ERR_INVALID_ARG, "verify: draft token id out of range");
+    cudaStream_t s = c->stream;
+    if (k > 0) CUDA_TRY(c, cudaMemcpyAsync(c->chain + 1, draft_tokens_host, sizeof(int) * k, cudaMemcpyHostToDevice, s));
+    cudaEventRecord(c->ev0, s);
+    enqueue_verify(c, k, hidden_dev_or_null != nullptr, c->stats.rounds % g.max_seq);
+    cudaEventRecord(c->ev1, s);
+    if (logits_dev_or_null)
+        CUDA_TRY(c, cudaMemcpyAsync(logits_dev_or_null, c->logits, sizeof(float) * (size_t)(k + 1) * g.vocab,
+                                    cudaMemcpyDeviceToDevice, s));
+    if (hidden_dev_or_null)
+        CUDA_TRY(c, cudaMemcpyAsync(hidden_dev_or_null, c->hfinal, sizeof(float) * (size_t)(k + 1) * g.d_model,
+                                    cudaMemcpyDeviceToDevice, s));
+    CUDA_TRY(c, cudaMemcpyAsync(c->pinned, c->state, sizeof(DeviceState), cudaMemcpyDeviceToHost, s));
+    knnssd_status st = sync_check(c, "verify");
+    if (st != KNNSSD_OK) return st;
+    const DeviceState *hs = reinterpret_cast<const DeviceState *>(c->pinned);
+    c->len = hs->len;
+    c->pending = hs->last_next;
+    c->stats.rounds += 1;
+    c->stats.drafted += k;
+    c->stats.accepted += hs->last_accept;
+    c->stats.tokens += hs->last_accept + 1;
+    c->stats.ms_verify += elapsed_ms(c);
+    if (n_accepted) *n_accepted = hs->last_accept;
+    if (next_token) *next_token = hs->last_next;
+    return KNNSSD_OK;
+}
+
+knnssd_status knnssd_generate(knnssd_ctx *c, const int *prompt_host, int n_prompt, int max_new, int k, int use_selection,
+                              int *out_tokens_host, int *n_out, int *accepts_host_or_null, int *domain_or_null,
+                              knnssd_stats *stats_or_null) {
+    if (!c) return KNNSSD_ERR_INVALID_ARG;
+    DeviceGuard dg(c->device);
+    const knnssd_config &g = c->cfg;
+    if (!out_tokens_host || !n_out || max_new < 1 || k < 0 || k > g.max_draft)
+        return fail(c, KNNSSD_ERR_INVALID_ARG, "generate: bad arguments");
+    if (n_prompt + max_new + 1 > g.max_seq) return fail(c, KNNSSD_ERR_CAPACITY, "generate: prompt + max_new + 1 exceeds max_seq");
+    const bool select = use_selection && g.n_domains > 0;
+    if (!select && !c->has_mask) return fail(c, KNNSSD_ERR_STATE, "generate: no active skip mask and no selection");
+    knnssd_status st = do_prefill(c, prompt_host, n_prompt, nullptr, nullptr);
+    if (st != KNNSSD_OK) return st;
+    int domain = -1;
+    if (select) {
+        st = do_select(c, nullptr, &domain, nullptr, nullptr);
+        if (st != KNNSSD_OK) return st;
+    }
+    cudaStream_t s = c->stream;
+    int produced = 1, round = 0;
+    while (produced < max_new) {
+        const int remaining = max_new - produced;
+        const int keff = k < remaining - 1 ? k : remaining - 1;
+        cudaEventRecord(c->ev0, s);
+        enqueue_draft(c, keff);
+        cudaEventRecord(c->ev1, s);
+        enqueue_verify(c, keff, false, round);
+        cudaEventRecord(c->ev2, s);
+        CUDA_TRY(c, cudaMemcpyAsync(c->pinned, c->state, sizeof(DeviceState), cudaMemcpyDeviceToHost, s));
+        st = sync_check(c, "generate");
+        if (st != KNNSSD_OK) return st;
+        const DeviceState *hs = reinterpret_cast<const DeviceState *>(c->pinned);
+        float ms = 0.f;
+        cudaEventElapsedTime(&ms, c->ev0, c->ev1);
+        c->stats.ms_draft += ms;
+        cudaEventElapsedTime(&ms, c->ev1, c->ev2);
+        c->stats.ms_verify += ms;
+        produced = hs->produced;
+        c->len = hs->len;
+        c->pending = hs->last_next;
+        c->stats.rounds += 1;
+        c->stats.drafted += keff;
+        c->stats.accepted += hs->last_accept;
+        ++round;
+    }
+    c->stats.tokens = produced;
+    CUDA_TRY(c, cudaMemcpyAsync(out_tokens_host, c->out_tokens, sizeof(int) * max_new, cudaMemcpyDeviceToHost, s));
+    if (accepts_host_or_null && round > 0)
+        CUDA_TRY(c, cudaMemcpyAsync(accepts_host_or_null, c->accept_log, sizeof(int) * round, cudaMemcpyDeviceToHost, s));
+    st = sync_check(c, "generate");
+    if (st != KNNSSD_OK) return st;
+    *n_out = max_new;
+    if (domain_or_null) *domain_or_null = domain;
+    if (stats_or_null) *stats_or_null = c->stats;
+    return KNNSSD_OK;
+}
+
+int knnssd_get_length(const knnssd_ctx *c) { return c ? c->len : -1; }
+
+knnssd_status knnssd_set_length(knnssd_ctx *c, int new_len) {
+    if (!c) return KNNSSD_ERR_INVALID_ARG;
+    DeviceGuard dg(c->device);
+    if (!c->prefilled) return fail(c, KNNSSD_ERR_STATE, "set_length: prefill first");
+    if (new_len < 1 || new_len > c->len) return fail(c, KNNSSD_ERR_INVALID_ARG, "set_length: can only roll back (1 <= new_len <= length)");
+    CUDA_TRY(c, cudaMemcpyAsync(&c->state->len, &new_len, sizeof(int), cudaMemcpyHostToDevice, c->stream));
+    knnssd_status st = sync_check(c, "set_length");
+    if (st != KNNSSD_OK) return st;
+    c->len = new_len;
+    return KNNSSD_OK;
+}
+
+knnssd_status knnssd_set_pending(knnssd_ctx *c, int token) {
+    if (!c) return KNNSSD_ERR_INVALID_ARG;
+    DeviceGuard dg(c->device);
+    if (!c->prefilled) return fail(c, KNNSSD_ERR_STATE, "set_pending: prefill first");
+    if (token < 0 || token >= c->cfg.vocab) return fail(c, KNNSSD_ERR_INVALID_ARG, "set_pending: token id out of range");
+    CUDA_TRY(c, cudaMemcpyAsync(c->chain, &token, sizeof(int), cudaMemcpyHostToDevice, c->stream));
+    knnssd_status st = sync_check(c, "set_pending");
+    if (st != KNNSSD_OK) return st;
+    c->pending = token;
+    return KNNSSD_OK;
+}
+
+knnssd_status knnssd_get_stats(const knnssd_ctx *c, knnssd_stats *out) {
+    if (!c || !out) return KNNSSD_ERR_INVALID_ARG;
+    *out = c->stats;
+    return KNNSSD_OK;
+}
+
+const char *knnssd_last_error(const knnssd_ctx *c) { return c ? c->err.c_str() : "NULL context"; }
+
+knnssd_status knnssd_time_pass(knnssd_ctx *c, int which, int k, int iters, float *ms_per_pass, int *launches_per_pass,
+                               float *ms_linear_per_pass, int *linear_launches_per_pass) {
+    if (!c) return KNNSSD_ERR_INVALID_ARG;
+    DeviceGuard dg(c->device);
+    const knnssd_config &g = c->cfg;
+    if ((which != 0 && which != 1) || iters < 1 || k < 0 || k > g.max_draft) return fail(c, KNNSSD_ERR_INVALID_ARG, "time_pass: bad arguments");
+    if (!c->prefilled) return fail(c, KNNSSD_ERR_STATE, "time_pass: prefill first");
+    if (which == 0 && !c->has_mask) return fail(c, KNNSSD_ERR_STATE, "time_pass: no active skip mask");
+    if (c->len + k + 1 > g.max_seq) return fail(c, KNNSSD_ERR_CAPACITY, "time_pass: len + k + 1 exceeds max_seq");
+    cudaStream_t s = c->stream;
+    // the chain must hold valid token ids for the rows a verify pass reads
+    std::vector<int> fill(k + 1, c->pending);
+    CUDA_TRY(c, cudaMemcpyAsync(c->chain, fill.data(), sizeof(int) * (k + 1), cudaMemcpyHostToDevice, s));
+    auto one = [&]() {
+        if (which == 0) run_pass(c, 1, c->chain, 0, c->active_mask.data(), 0, c->target, false);
+        else run_pass(c, k + 1, c->chain, 0, nullptr, 0, c->target, false);
+    };
+    const long long l0 = c->launches;
+    one();
+    const int launches = (int)(c->launches - l0);
+    knnssd_status st = sync_check(c, "time_pass warm-up");
+    if (st != KNNSSD_OK) return st;
+    cudaEventRecord(c->ev0, s);
+    for (int i = 0; i < iters; ++i) one();
+    cudaEventRecord(c->ev1, s);
+    st = sync_check(c, "time_pass");
+    if (st != KNNSSD_OK) return st;
+    if (ms_per_pass) *ms_per_pass = elapsed_ms(c) / (float)iters;
+    if (launches_per_pass) *launches_per_pass = launches;
+    // separate replay with events around every linear kernel
+    c->time_linear = true;
+    c->lin_used = 0;
+    one();
+    c->time_linear = false;
+    st = sync_check(c, "time_pass linear replay");
+    if (st != KNNSSD_OK) return st;
+    float tot = 0.f;
+    for (size_t i = 0; i + 1 < c->lin_used; i += 2) {
+        float ms = 0.f;
+        cudaEventElapsedTime(&ms, c->lin_events[i], c->lin_events[i + 1]);
+        tot += ms;
+    }
+    if (ms_linear_per_pass) *ms_linear_per_pass = tot;
+    if (linear_launches_per_pass) *linear_launches_per_pass = (int)(c->lin_used / 2);
+    // restore the pending token the chain held
+    CUDA_TRY(c, cudaMemcpyAsync(c->chain, &c->pending, sizeof(int), cudaMemcpyHostToDevice, s));
+    return sync_check(c, "time_pass restore");
+}
+
+knnssd_status knnssd_linear(const void *W_dev, int dtype, int n_out, int n_in, const float *x_dev, int M, float *y_dev,
+                            void *cuda_stream) {
+    if (!W_dev || !x_dev || !y_dev || n_out < 1 || n_in < 8 || M < 1 || M > kMaxRows || (dtype != 0 && dtype != 1))
+        return KNNSSD_ERR_INVALID_ARG;
+    if (n_in % 8 != 0 || (reinterpret_cast<uintptr_t>(W_dev) & 15u) || (reinterpret_cast<uintptr_t>(x_dev) & 15u))
+        return KNNSSD_ERR_SHAPE;
+    int dev = 0, n_sms = 148;
+    if (cudaGetDevice(&dev) != cudaSuccess) return KNNSSD_ERR_CUDA;
+    cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev);
+    LinearArgs a = make_args(W_dev, n_out, n_in, x_dev, nullptr, 0.f, y_dev, EPI_STORE, M);
+    launch_linear(dtype, a, n_sms, reinterpret_cast<cudaStream_t>(cuda_stream));
+    return cudaGetLastError() == cudaSuccess ? KNNSSD_OK : KNNSSD_ERR_CUDA;
+}
+
+knnssd_status knnssd_cosine_top1(const float *query_dev, const float *anchors_dev, int n, int d, int *best, float *cosine,
+                                 void *cuda_stream) {
+    if (!query_dev || !anchors_dev || n < 1 || d < 1) return KNNSSD_ERR_INVALID_ARG;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+    float *cos_dev = nullptr;
+    int *small = nullptr;  // [0..1] result, [2] flag
+    if (cudaMalloc(reinterpret_cast<void **>(&cos_dev), sizeof(float) * n) != cudaSuccess) return KNNSSD_ERR_CUDA;
+    if (cudaMalloc(reinterpret_cast<void **>(&small), sizeof(int) * 4) != cudaSuccess) { cudaFree(cos_dev); return KNNSSD_ERR_CUDA; }
+    cudaMemsetAsync(small, 0, sizeof(int) * 4, s);
+    cosine_scores_kernel<<<(n + 7) / 8, 256, 0, s>>>(query_dev, anchors_dev, nullptr, n, d, cos_dev, small + 2);
+    cosine_argmax_kernel<<<1, 256, 0, s>>>(cos_dev, n, small);
+    int host[4] = {0, 0, 0, 0};
+    cudaError_t e = cudaMemcpyAsync(host, small, sizeof(int) * 4, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    cudaFree(cos_dev);
+    cudaFree(small);
+    if (e != cudaSuccess) return KNNSSD_ERR_CUDA;
+    if (host[2]) return KNNSSD_ERR_DEGENERATE;
+    if (best) *best = host[0];
+    if (cosine) std::memcpy(cosine, &host[1], sizeof(float));
+    return KNNSSD_OK;
+}
+
+}  // extern "C"
