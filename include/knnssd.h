@@ -152,6 +152,17 @@ knnssd_status knnssd_generate(knnssd_ctx *ctx, const int *prompt_host, int n_pro
                               int use_selection, int *out_tokens_host, int *n_out, int *accepts_host_or_null,
                               int *domain_or_null, knnssd_stats *stats_or_null);
 
+/*
+ * The decode part of knnssd_generate on an already prefilled session: optional select_skipset on the pooled vector
+ * of the last prefill, then rounds of draft + verify until max_new tokens are out, the first of them being the
+ * pending token.  Arguments as in knnssd_generate.  Statistics of rounds are restarted by this call.
+ */
+knnssd_status knnssd_decode(knnssd_ctx *ctx, int max_new, int k, int use_selection, int *out_tokens_host, int *n_out,
+                            int *accepts_host_or_null, int *domain_or_null, knnssd_stats *stats_or_null);
+
+/* Number of kernels this context has launched since it was created (-1 for a NULL context). */
+long long knnssd_get_launch_count(const knnssd_ctx *ctx);
+
 /* Committed context length (positions whose K/V are valid), and explicit rollback to a shorter length
  * (new_len <= current length; the pending token is unchanged, so this is meant for tests and benchmarks). */
 int knnssd_get_length(const knnssd_ctx *ctx);

@@ -21,7 +21,7 @@ STATUS = {0: "OK", 1: "ERR_INVALID_ARG", 2: "ERR_SHAPE", 3: "ERR_CAPACITY", 4: "
           5: "ERR_DEGENERATE", 6: "ERR_CUDA", 7: "ERR_TIMEOUT"}
 
 EXPORTS = ["knnssd_init", "knnssd_destroy", "knnssd_prefill", "knnssd_select_skipset", "knnssd_set_skipmask",
-           "knnssd_draft", "knnssd_verify", "knnssd_generate", "knnssd_get_length", "knnssd_set_length",
+           "knnssd_draft", "knnssd_verify", "knnssd_generate", "knnssd_decode", "knnssd_get_launch_count", "knnssd_get_length", "knnssd_set_length",
            "knnssd_set_pending", "knnssd_get_stats", "knnssd_last_error", "knnssd_time_pass", "knnssd_linear",
            "knnssd_cosine_top1"]
 
@@ -66,6 +66,8 @@ def _load():
         "knnssd_draft": (I, [P, I, P, P]),
         "knnssd_verify": (I, [P, P, I, PI, PI, P, P]),
         "knnssd_generate": (I, [P, P, I, I, I, I, P, PI, P, PI, C.POINTER(Stats)]),
+        "knnssd_decode": (I, [P, I, I, I, P, PI, P, PI, C.POINTER(Stats)]),
+        "knnssd_get_launch_count": (C.c_longlong, [P]),
         "knnssd_get_length": (I, [P]),
         "knnssd_set_length": (I, [P, I]),
         "knnssd_set_pending": (I, [P, I]),
@@ -232,6 +234,19 @@ class Session:
                                          out.ctypes.data, C.byref(n_out), acc.ctypes.data, C.byref(dom), C.byref(st)))
         return {"tokens": out[:n_out.value], "accepts": acc[:st.rounds].copy(), "domain": dom.value,
                 "stats": {f: getattr(st, f) for f, _ in Stats._fields_}}
+
+    def decode(self, max_new: int, k: int, use_selection: bool = False):
+        out = np.zeros(max_new, dtype=np.int32)
+        acc = np.full(max_new, -1, dtype=np.int32)
+        n_out, dom, st = C.c_int(), C.c_int(), Stats()
+        self._check(_lib.knnssd_decode(self.h, max_new, k, int(use_selection), out.ctypes.data, C.byref(n_out),
+                                       acc.ctypes.data, C.byref(dom), C.byref(st)))
+        return {"tokens": out[:n_out.value], "accepts": acc[:st.rounds].copy(), "domain": dom.value,
+                "stats": {f: getattr(st, f) for f, _ in Stats._fields_}}
+
+    @property
+    def launch_count(self) -> int:
+        return _lib.knnssd_get_launch_count(self.h)
 
     @property
     def length(self) -> int:

@@ -3,6 +3,7 @@
 // Every step of the path runs in the kernels of kernels.cuh; the host only enqueues them.
 #include "../../include/knnssd.h"
 #include "kernels.cuh"
+#include "linear_stream.cuh"
 
 #include <cmath>
 #include <cstdio>
@@ -103,8 +104,49 @@ template <typename WT> void launch_linear_t(const LinearArgs &a, int grid, cudaS
     }
 }
 
+// Set by the streaming kernel if one of its bounded waits ever gives up (never in normal operation).
+__device__ int g_stream_err;
+
+int *stream_err_ptr() {
+    static int *p = nullptr;
+    if (!p) cudaGetSymbolAddress(reinterpret_cast<void **>(&p), g_stream_err);
+    return p;
+}
+
+template <int MT> void launch_stream_t(const stream::Args &sa, int n_sms, cudaStream_t s) {
+    static bool configured = false;
+    if (!configured) {
+        cudaFuncSetAttribute(stream::linear_stream_kernel<MT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             stream::smem_bytes(MT));
+        configured = true;
+    }
+    stream::linear_stream_kernel<MT><<<n_sms, stream::NTHREADS, stream::smem_bytes(MT), s>>>(sa);
+}
+
+bool stream_eligible(int dtype, const LinearArgs &a) {
+    return dtype == 1 && a.M <= 8 && a.n_in % 128 == 0 && a.n_in >= 256;
+}
+
+void launch_stream(const LinearArgs &a, int n_sms, cudaStream_t s) {
+    stream::Args sa{};
+    for (int i = 0; i < 3; ++i) { sa.W[i] = reinterpret_cast<const bf16_t *>(a.W[i]); sa.rows[i] = a.rows[i]; }
+    sa.units = a.units; sa.K = a.n_in; sa.x = a.x; sa.gain = a.gain; sa.eps = a.eps; sa.y = a.y; sa.epi = a.epi; sa.M = a.M;
+    sa.err = stream_err_ptr();
+    switch (a.M) {
+        case 1: launch_stream_t<1>(sa, n_sms, s); break;
+        case 2: launch_stream_t<2>(sa, n_sms, s); break;
+        case 3: launch_stream_t<3>(sa, n_sms, s); break;
+        case 4: launch_stream_t<4>(sa, n_sms, s); break;
+        case 5: launch_stream_t<5>(sa, n_sms, s); break;
+        case 6: launch_stream_t<6>(sa, n_sms, s); break;
+        case 7: launch_stream_t<7>(sa, n_sms, s); break;
+        default: launch_stream_t<8>(sa, n_sms, s); break;
+    }
+}
+
 void launch_linear(int dtype, const LinearArgs &a, int n_sms, cudaStream_t s) {
-    // enough warps that every SM holds 8 blocks of 8 warps, but never more warps than units
+    if (stream_eligible(dtype, a)) { launch_stream(a, n_sms, s); return; }
+    // generic kernel: enough warps that every SM holds 8 blocks of 8 warps, but never more warps than units
     long long blocks = (long long)n_sms * 8;
     const long long max_blocks = (a.units + 7) / 8;
     if (blocks > max_blocks) blocks = max_blocks;
@@ -215,6 +257,18 @@ knnssd_status sync_check(knnssd_ctx *c, const char *what) {
     return KNNSSD_OK;
 }
 
+// A bounded wait inside the streaming kernel gave up: report it once and clear the word.
+knnssd_status check_stream_err(knnssd_ctx *c, const char *what) {
+    int code = 0;
+    if (cudaMemcpy(&code, stream_err_ptr(), sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess)
+        return fail(c, KNNSSD_ERR_CUDA, std::string(what) + ": cannot read the device error word");
+    if (code) {
+        cudaMemset(stream_err_ptr(), 0, sizeof(int));
+        return fail(c, KNNSSD_ERR_TIMEOUT, std::string(what) + ": a device-side wait gave up (code " + std::to_string(code) + ")");
+    }
+    return KNNSSD_OK;
+}
+
 void free_all(knnssd_ctx *c) {
     void *ptrs[] = {c->kcache, c->vcache, c->x, c->qkv, c->attn, c->act, c->logits, c->hfinal, c->part_o, c->pooled,
                     c->anchor_inv_norm, c->cosines, c->amax_v, c->part_ml, c->rope_cs, c->pool_sum, c->inv_freq, c->chain,
@@ -271,6 +325,7 @@ knnssd_status do_prefill(knnssd_ctx *c, const int *tokens_host, int n, float *po
     if (pooled_dev) CUDA_TRY(c, cudaMemcpyAsync(pooled_dev, c->pooled, sizeof(float) * d, cudaMemcpyDeviceToDevice, s));
     CUDA_TRY(c, cudaMemcpyAsync(c->pinned, c->chain, sizeof(int), cudaMemcpyDeviceToHost, s));
     knnssd_status st = sync_check(c, "prefill");
+    if (st == KNNSSD_OK) st = check_stream_err(c, "prefill");
     if (st != KNNSSD_OK) return st;
     c->len = n;
     c->pending = c->pinned[0];
@@ -476,6 +531,7 @@ knnssd_status knnssd_draft(knnssd_ctx *c, int k, int *draft_tokens_host, float *
     cudaEventRecord(c->ev1, s);
     CUDA_TRY(c, cudaMemcpyAsync(c->pinned, c->chain + 1, sizeof(int) * k, cudaMemcpyDeviceToHost, s));
     knnssd_status st = sync_check(c, "draft");
+    if (st == KNNSSD_OK) st = check_stream_err(c, "draft");
     if (st != KNNSSD_OK) return st;
     for (int j = 0; j < k; ++j) draft_tokens_host[j] = c->pinned[j];
     c->stats.ms_draft += elapsed_ms(c);
@@ -506,6 +562,7 @@ knnssd_status knnssd_verify(knnssd_ctx *c, const int *draft_tokens_host, int k, 
                                     cudaMemcpyDeviceToDevice, s));
     CUDA_TRY(c, cudaMemcpyAsync(c->pinned, c->state, sizeof(DeviceState), cudaMemcpyDeviceToHost, s));
     knnssd_status st = sync_check(c, "verify");
+    if (st == KNNSSD_OK) st = check_stream_err(c, "verify");
     if (st != KNNSSD_OK) return st;
     const DeviceState *hs = reinterpret_cast<const DeviceState *>(c->pinned);
     c->len = hs->len;
@@ -520,26 +577,28 @@ knnssd_status knnssd_verify(knnssd_ctx *c, const int *draft_tokens_host, int k, 
     return KNNSSD_OK;
 }
 
-knnssd_status knnssd_generate(knnssd_ctx *c, const int *prompt_host, int n_prompt, int max_new, int k, int use_selection,
-                              int *out_tokens_host, int *n_out, int *accepts_host_or_null, int *domain_or_null,
-                              knnssd_stats *stats_or_null) {
-    if (!c) return KNNSSD_ERR_INVALID_ARG;
-    DeviceGuard dg(c->device);
+static knnssd_status do_decode(knnssd_ctx *c, int max_new, int k, int use_selection, int *out_tokens_host, int *n_out,
+                               int *accepts_host_or_null, int *domain_or_null, knnssd_stats *stats_or_null) {
     const knnssd_config &g = c->cfg;
     if (!out_tokens_host || !n_out || max_new < 1 || k < 0 || k > g.max_draft)
-        return fail(c, KNNSSD_ERR_INVALID_ARG, "generate: bad arguments");
-    if (n_prompt + max_new + 1 > g.max_seq) return fail(c, KNNSSD_ERR_CAPACITY, "generate: prompt + max_new + 1 exceeds max_seq");
+        return fail(c, KNNSSD_ERR_INVALID_ARG, "decode: bad arguments");
+    if (!c->prefilled) return fail(c, KNNSSD_ERR_STATE, "decode: prefill first");
+    if (c->len + max_new + 1 > g.max_seq) return fail(c, KNNSSD_ERR_CAPACITY, "decode: length + max_new + 1 exceeds max_seq");
     const bool select = use_selection && g.n_domains > 0;
-    if (!select && !c->has_mask) return fail(c, KNNSSD_ERR_STATE, "generate: no active skip mask and no selection");
-    knnssd_status st = do_prefill(c, prompt_host, n_prompt, nullptr, nullptr);
-    if (st != KNNSSD_OK) return st;
+    if (!select && !c->has_mask) return fail(c, KNNSSD_ERR_STATE, "decode: no active skip mask and no selection");
+    knnssd_status st;
     int domain = -1;
     if (select) {
         st = do_select(c, nullptr, &domain, nullptr, nullptr);
         if (st != KNNSSD_OK) return st;
     }
     cudaStream_t s = c->stream;
+    // the pending token is the first token of this call's output
+    emit_first_token_kernel<<<1, 1, 0, s>>>(c->chain, c->state, c->out_tokens, c->len);
+    c->launches++;
     int produced = 1, round = 0;
+    c->stats.rounds = c->stats.drafted = c->stats.accepted = 0;
+    c->stats.ms_draft = c->stats.ms_verify = 0.f;
     while (produced < max_new) {
         const int remaining = max_new - produced;
         const int keff = k < remaining - 1 ? k : remaining - 1;
@@ -549,7 +608,7 @@ knnssd_status knnssd_generate(knnssd_ctx *c, const int *prompt_host, int n_promp
         enqueue_verify(c, keff, false, round);
         cudaEventRecord(c->ev2, s);
         CUDA_TRY(c, cudaMemcpyAsync(c->pinned, c->state, sizeof(DeviceState), cudaMemcpyDeviceToHost, s));
-        st = sync_check(c, "generate");
+        st = sync_check(c, "decode");
         if (st != KNNSSD_OK) return st;
         const DeviceState *hs = reinterpret_cast<const DeviceState *>(c->pinned);
         float ms = 0.f;
@@ -569,13 +628,41 @@ knnssd_status knnssd_generate(knnssd_ctx *c, const int *prompt_host, int n_promp
     CUDA_TRY(c, cudaMemcpyAsync(out_tokens_host, c->out_tokens, sizeof(int) * max_new, cudaMemcpyDeviceToHost, s));
     if (accepts_host_or_null && round > 0)
         CUDA_TRY(c, cudaMemcpyAsync(accepts_host_or_null, c->accept_log, sizeof(int) * round, cudaMemcpyDeviceToHost, s));
-    st = sync_check(c, "generate");
+    st = sync_check(c, "decode");
+    if (st == KNNSSD_OK) st = check_stream_err(c, "decode");
     if (st != KNNSSD_OK) return st;
     *n_out = max_new;
     if (domain_or_null) *domain_or_null = domain;
     if (stats_or_null) *stats_or_null = c->stats;
     return KNNSSD_OK;
 }
+
+knnssd_status knnssd_decode(knnssd_ctx *c, int max_new, int k, int use_selection, int *out_tokens_host, int *n_out,
+                            int *accepts_host_or_null, int *domain_or_null, knnssd_stats *stats_or_null) {
+    if (!c) return KNNSSD_ERR_INVALID_ARG;
+    DeviceGuard dg(c->device);
+    return do_decode(c, max_new, k, use_selection, out_tokens_host, n_out, accepts_host_or_null, domain_or_null,
+                     stats_or_null);
+}
+
+knnssd_status knnssd_generate(knnssd_ctx *c, const int *prompt_host, int n_prompt, int max_new, int k, int use_selection,
+                              int *out_tokens_host, int *n_out, int *accepts_host_or_null, int *domain_or_null,
+                              knnssd_stats *stats_or_null) {
+    if (!c) return KNNSSD_ERR_INVALID_ARG;
+    DeviceGuard dg(c->device);
+    const knnssd_config &g = c->cfg;
+    if (!out_tokens_host || !n_out || max_new < 1 || k < 0 || k > g.max_draft)
+        return fail(c, KNNSSD_ERR_INVALID_ARG, "generate: bad arguments");
+    if (n_prompt + max_new + 1 > g.max_seq) return fail(c, KNNSSD_ERR_CAPACITY, "generate: prompt + max_new + 1 exceeds max_seq");
+    if (!(use_selection && g.n_domains > 0) && !c->has_mask)
+        return fail(c, KNNSSD_ERR_STATE, "generate: no active skip mask and no selection");
+    knnssd_status st = do_prefill(c, prompt_host, n_prompt, nullptr, nullptr);
+    if (st != KNNSSD_OK) return st;
+    return do_decode(c, max_new, k, use_selection, out_tokens_host, n_out, accepts_host_or_null, domain_or_null,
+                     stats_or_null);
+}
+
+long long knnssd_get_launch_count(const knnssd_ctx *c) { return c ? c->launches : -1; }
 
 int knnssd_get_length(const knnssd_ctx *c) { return c ? c->len : -1; }
 
@@ -657,7 +744,9 @@ knnssd_status knnssd_time_pass(knnssd_ctx *c, int which, int k, int iters, float
     if (linear_launches_per_pass) *linear_launches_per_pass = (int)(c->lin_used / 2);
     // restore the pending token the chain held
     CUDA_TRY(c, cudaMemcpyAsync(c->chain, &c->pending, sizeof(int), cudaMemcpyHostToDevice, s));
-    return sync_check(c, "time_pass restore");
+    st = sync_check(c, "time_pass restore");
+    if (st == KNNSSD_OK) st = check_stream_err(c, "time_pass");
+    return st;
 }
 
 knnssd_status knnssd_linear(const void *W_dev, int dtype, int n_out, int n_in, const float *x_dev, int M, float *y_dev,

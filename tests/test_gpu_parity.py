@@ -47,7 +47,11 @@ def _pair(kb, shape_name, seed=0, max_seq=160, gain_spread=0.1, damp=None, ancho
 
 @pytest.mark.parametrize("dtype", ["bf16", "fp32"])
 @pytest.mark.parametrize("n_out,n_in,M", [(1, 8, 1), (37, 72, 3), (1003, 328, 1), (1003, 328, 5), (2051, 1384, 9),
-                                          (515, 2056, 16), (4099, 512, 2), (300, 5120, 7)])
+                                          (515, 2056, 16), (4099, 512, 2), (300, 5120, 7),
+                                          # streaming-kernel shapes (bf16, n_in % 128 == 0, M <= 8): one and several
+                                          # batches per CTA, partial last column tile, fewer rows than CTAs
+                                          (20011, 256, 3), (5120, 5120, 5), (333, 13824, 8), (4099, 1152, 1),
+                                          (160, 1024, 8), (7, 2048, 2), (40000, 384, 1)])
 def test_linear_matches_oracle(kb, dtype, n_out, n_in, M):
     W = si.normal_weight(1, 77, n_out, n_in, 0.02, dtype)
     x = si.normal_f32(2, 78, torch.arange(M * n_in), 1.0).view(M, n_in).contiguous()
@@ -58,12 +62,13 @@ def test_linear_matches_oracle(kb, dtype, n_out, n_in, M):
 
 def test_linear_rows_do_not_depend_on_batch(kb):
     """A row of an M-row launch is bit-identical to the same row launched alone."""
-    W = si.normal_weight(1, 77, 1003, 1384, 0.02, "bf16").cuda()
-    x = si.normal_f32(2, 78, torch.arange(9 * 1384), 1.0).view(9, 1384).contiguous().cuda()
-    full = kb.knnssd_linear(W, x)
-    for M in (1, 2, 5):
-        assert torch.equal(kb.knnssd_linear(W, x[:M].contiguous()), full[:M])
-    assert torch.equal(kb.knnssd_linear(W, x[4:5].contiguous())[0], full[4])
+    for n_in, top in ((1384, 9), (1152, 8)):          # generic kernel; streaming kernel
+        W = si.normal_weight(1, 77, 1003, n_in, 0.02, "bf16").cuda()
+        x = si.normal_f32(2, 78, torch.arange(top * n_in), 1.0).view(top, n_in).contiguous().cuda()
+        full = kb.knnssd_linear(W, x)
+        for M in (1, 2, 5):
+            assert torch.equal(kb.knnssd_linear(W, x[:M].contiguous()), full[:M])
+        assert torch.equal(kb.knnssd_linear(W, x[4:5].contiguous())[0], full[4])
 
 
 def test_linear_rejects_bad_arguments(kb):
@@ -99,7 +104,8 @@ def test_cosine_top1_matches_oracle(kb):
 
 # ---- whole path on small shapes -------------------------------------------------------------------
 
-CASES = [("tiny", 32, 32), ("gqa-fp32", 21, 19), ("ragged-bf16", 33, 24), ("gqa-bf16", 40, 24)]
+CASES = [("tiny", 32, 32), ("gqa-fp32", 21, 19), ("ragged-bf16", 33, 24), ("gqa-bf16", 40, 24),
+         ("stream-bf16", 37, 24)]
 
 
 @pytest.mark.parametrize("shape_name,prompt_len,max_new", CASES)
