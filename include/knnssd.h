@@ -199,6 +199,29 @@ knnssd_status knnssd_linear(const void *W_dev, int dtype, int n_out, int n_in, c
 knnssd_status knnssd_cosine_top1(const float *query_dev, const float *anchors_dev, int n, int d, int *best,
                                  float *cosine, void *cuda_stream);
 
+/*
+ * knnssd_cosine_top1 for callers that must not allocate device memory.  (No counterpart in the paper: this is a
+ * deployment variant of the call above, same arithmetic, same results.)
+ *
+ * Who needs it: code that runs where cudaMalloc / cudaFree are off limits - inside a serving loop whose memory pool
+ * was sized and handed out at start-up, in a process that shares the GPU under a fixed memory reservation, or in a
+ * latency path where the implicit device synchronisation of cudaFree is not acceptable.  knnssd_cosine_top1 makes two
+ * small cudaMalloc / cudaFree pairs per call for its per-anchor cosines and its result words; this variant keeps that
+ * scratch in a fixed array inside the library's device image instead, and calls no allocating routine at all.
+ *
+ *   arguments   as knnssd_cosine_top1 (query_dev, anchors_dev DEVICE fp32; best, cosine HOST outputs)
+ *   limit       n <= KNNSSD_STATIC_MAX_ANCHORS; a larger n returns KNNSSD_ERR_CAPACITY and touches nothing
+ *   cost        every GPU that loads the library holds the array (about 16 KB) until the process exits
+ *   first call  the first call on each device looks up the array's device address (once per device, with that device
+ *               current); make that first call before starting any stream capture
+ *   sharing     all calls on a device use the same array, and it keeps what the previous call left there; the call
+ *               clears the words that must start at zero itself.  Two calls that overlap on one GPU (different
+ *               streams or host threads) race on it: serialise them
+ */
+#define KNNSSD_STATIC_MAX_ANCHORS 4096
+knnssd_status knnssd_cosine_top1_static(const float *query_dev, const float *anchors_dev, int n, int d, int *best,
+                                        float *cosine, void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

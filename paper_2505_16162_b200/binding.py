@@ -23,7 +23,7 @@ STATUS = {0: "OK", 1: "ERR_INVALID_ARG", 2: "ERR_SHAPE", 3: "ERR_CAPACITY", 4: "
 EXPORTS = ["knnssd_init", "knnssd_destroy", "knnssd_prefill", "knnssd_select_skipset", "knnssd_set_skipmask",
            "knnssd_draft", "knnssd_verify", "knnssd_generate", "knnssd_decode", "knnssd_get_launch_count", "knnssd_get_length", "knnssd_set_length",
            "knnssd_set_pending", "knnssd_get_stats", "knnssd_last_error", "knnssd_time_pass", "knnssd_linear",
-           "knnssd_cosine_top1"]
+           "knnssd_cosine_top1", "knnssd_cosine_top1_static"]
 
 
 class KnnssdError(RuntimeError):
@@ -76,6 +76,7 @@ def _load():
         "knnssd_time_pass": (I, [P, I, I, I, PF, PI, PF, PI]),
         "knnssd_linear": (I, [P, I, I, I, P, I, P, P]),
         "knnssd_cosine_top1": (I, [P, P, I, I, PI, PF, P]),
+        "knnssd_cosine_top1_static": (I, [P, P, I, I, PI, PF, P]),
     }
     for name, (res, args) in sigs.items():
         fn = getattr(lib, name)
@@ -128,6 +129,25 @@ def knnssd_cosine_top1(query: torch.Tensor, anchors: torch.Tensor):
                                      C.byref(best), C.byref(cs), torch.cuda.current_stream().cuda_stream)
     if rc:
         raise KnnssdError(rc, "knnssd_cosine_top1")
+    return best.value, cs.value
+
+
+STATIC_MAX_ANCHORS = 4096
+
+
+def knnssd_cosine_top1_static(query: torch.Tensor, anchors: torch.Tensor):
+    """Same search and same result as ``knnssd_cosine_top1``, for callers that may not allocate device memory
+    (a serving loop living inside a pre-sized pool, a process under a fixed memory reservation): the library keeps
+    the per-anchor cosines in a fixed array of its own, so nothing is allocated or freed here either - the inputs
+    are used in place and the two results come back as Python numbers.  At most ``STATIC_MAX_ANCHORS`` anchors
+    (ERR_CAPACITY beyond that).  All calls on a GPU share that array: do not overlap them."""
+    n, d = anchors.shape
+    best, cs = C.c_int(), C.c_float()
+    with torch.cuda.device(query.device):
+        rc = _lib.knnssd_cosine_top1_static(_dev_ptr(query, torch.float32), _dev_ptr(anchors, torch.float32), n, d,
+                                            C.byref(best), C.byref(cs), torch.cuda.current_stream().cuda_stream)
+    if rc:
+        raise KnnssdError(rc, "knnssd_cosine_top1_static")
     return best.value, cs.value
 
 

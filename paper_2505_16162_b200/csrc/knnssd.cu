@@ -8,6 +8,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <string>
 #include <vector>
@@ -787,3 +788,55 @@ knnssd_status knnssd_cosine_top1(const float *query_dev, const float *anchors_de
 }
 
 }  // extern "C"
+
+// ---- cosine top-1 without any allocation ------------------------------------------------------------------------
+// Scratch of knnssd_cosine_top1_static: the per-anchor cosines, then four result words (best index, cosine bits,
+// degenerate-input flag, spare).  It lives in the library's device image, one copy per GPU that loads the library.
+// In host code the name below is only a handle for cudaGetSymbolAddress; kernels get the address that call returns.
+namespace {
+constexpr int kStaticWords = KNNSSD_STATIC_MAX_ANCHORS + 4;
+constexpr int kMaxDevices = 64;
+}  // namespace
+static __device__ __align__(256) float g_top1_static_scratch[kStaticWords];
+
+namespace {
+// Device address of the array on the current device, looked up once per device.
+cudaError_t static_scratch_address(int dev, float **out) {
+    static float *addr[kMaxDevices] = {};
+    static std::mutex mu;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!addr[dev]) {
+        float *p = nullptr;
+        const cudaError_t e = cudaGetSymbolAddress(reinterpret_cast<void **>(&p), g_top1_static_scratch);
+        if (e != cudaSuccess) return e;
+        addr[dev] = p;
+    }
+    *out = addr[dev];
+    return cudaSuccess;
+}
+}  // namespace
+
+extern "C" knnssd_status knnssd_cosine_top1_static(const float *query_dev, const float *anchors_dev, int n, int d,
+                                                   int *best, float *cosine, void *cuda_stream) {
+    if (!query_dev || !anchors_dev || n < 1 || d < 1) return KNNSSD_ERR_INVALID_ARG;
+    if (n > KNNSSD_STATIC_MAX_ANCHORS) return KNNSSD_ERR_CAPACITY;   // beyond the fixed scratch: refuse, touch nothing
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return KNNSSD_ERR_CUDA;
+    float *scratch = nullptr;
+    if (static_scratch_address(dev, &scratch) != cudaSuccess) { cudaGetLastError(); return KNNSSD_ERR_CUDA; }
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+    float *cos_dev = scratch;
+    int *small = reinterpret_cast<int *>(scratch + KNNSSD_STATIC_MAX_ANCHORS);   // [0..1] result, [2] flag
+    // the array still holds the previous call's result and flag: the words that must start at zero are cleared here
+    if (cudaMemsetAsync(small, 0, sizeof(int) * 4, s) != cudaSuccess) return KNNSSD_ERR_CUDA;
+    cosine_scores_kernel<<<(n + 7) / 8, 256, 0, s>>>(query_dev, anchors_dev, nullptr, n, d, cos_dev, small + 2);
+    cosine_argmax_kernel<<<1, 256, 0, s>>>(cos_dev, n, small);
+    int host[4] = {0, 0, 0, 0};
+    cudaError_t e = cudaMemcpyAsync(host, small, sizeof(int) * 4, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return KNNSSD_ERR_CUDA;
+    if (host[2]) return KNNSSD_ERR_DEGENERATE;
+    if (best) *best = host[0];
+    if (cosine) std::memcpy(cosine, &host[1], sizeof(float));
+    return KNNSSD_OK;
+}
