@@ -114,35 +114,24 @@ int *stream_err_ptr() {
     return p;
 }
 
-template <int MT> void launch_stream_t(const stream::Args &sa, int n_sms, cudaStream_t s) {
-    static bool configured = false;
-    if (!configured) {
-        cudaFuncSetAttribute(stream::linear_stream_kernel<MT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             stream::smem_bytes(MT));
-        configured = true;
-    }
-    stream::linear_stream_kernel<MT><<<n_sms, stream::NTHREADS, stream::smem_bytes(MT), s>>>(sa);
-}
-
 bool stream_eligible(int dtype, const LinearArgs &a) {
     return dtype == 1 && a.M <= 8 && a.n_in % 128 == 0 && a.n_in >= 256;
 }
 
+stream::LinPhase to_phase(const LinearArgs &a) {
+    stream::LinPhase p{};
+    for (int i = 0; i < 3; ++i) { p.W[i] = reinterpret_cast<const bf16_t *>(a.W[i]); p.rows[i] = a.rows[i]; }
+    p.units = a.units; p.K = a.n_in; p.x = a.x; p.gain = a.gain; p.eps = a.eps; p.y = a.y; p.epi = a.epi; p.M = a.M;
+    return p;
+}
+
 void launch_stream(const LinearArgs &a, int n_sms, cudaStream_t s) {
-    stream::Args sa{};
-    for (int i = 0; i < 3; ++i) { sa.W[i] = reinterpret_cast<const bf16_t *>(a.W[i]); sa.rows[i] = a.rows[i]; }
-    sa.units = a.units; sa.K = a.n_in; sa.x = a.x; sa.gain = a.gain; sa.eps = a.eps; sa.y = a.y; sa.epi = a.epi; sa.M = a.M;
-    sa.err = stream_err_ptr();
-    switch (a.M) {
-        case 1: launch_stream_t<1>(sa, n_sms, s); break;
-        case 2: launch_stream_t<2>(sa, n_sms, s); break;
-        case 3: launch_stream_t<3>(sa, n_sms, s); break;
-        case 4: launch_stream_t<4>(sa, n_sms, s); break;
-        case 5: launch_stream_t<5>(sa, n_sms, s); break;
-        case 6: launch_stream_t<6>(sa, n_sms, s); break;
-        case 7: launch_stream_t<7>(sa, n_sms, s); break;
-        default: launch_stream_t<8>(sa, n_sms, s); break;
+    static bool configured = false;
+    if (!configured) {
+        cudaFuncSetAttribute(stream::linear_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, stream::SMEM_BYTES);
+        configured = true;
     }
+    stream::linear_stream_kernel<<<n_sms, stream::NTHREADS, stream::SMEM_BYTES, s>>>(to_phase(a), stream_err_ptr());
 }
 
 void launch_linear(int dtype, const LinearArgs &a, int n_sms, cudaStream_t s) {
