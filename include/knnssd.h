@@ -183,6 +183,21 @@ const char *knnssd_last_error(const knnssd_ctx *ctx);
 knnssd_status knnssd_time_pass(knnssd_ctx *ctx, int which, int k, int iters, float *ms_per_pass,
                                int *launches_per_pass, float *ms_linear_per_pass, int *linear_launches_per_pass);
 
+/*
+ * Per-operation timing inside the persistent pass kernel (bf16 models it serves; KNNSSD_ERR_SHAPE otherwise): runs
+ * one pass as knnssd_time_pass does (which: 0 = draft step, 1 = verify pass over k+1 rows) with CTA 0 stamping the
+ * device's nanosecond timer after each operation's work and after the grid barrier that follows it.
+ *   cap          capacity of the four HOST output arrays
+ *   op_types     0 embedding, 2 attention, 3 hidden-state output, 4 arg-max, 10 linear (store: QKV), 11 linear with
+ *                residual add (O / down projection), 12 gate/up linear with SwiGLU, 14 LM head
+ *   op_layers    decoder layer of the operation (0 for embedding / head / arg-max)
+ *   us_work      microseconds from the previous operation's barrier to the end of this operation's work on CTA 0
+ *   us_barrier   microseconds CTA 0 then waited at the barrier
+ *   n_ops        operations reported
+ */
+knnssd_status knnssd_trace_pass(knnssd_ctx *ctx, int which, int k, int cap, int *op_types, int *op_layers, float *us_work,
+                                float *us_barrier, int *n_ops);
+
 /* ---- stand-alone operators (same kernels the passes use; for per-kernel tests and measurements) ---- */
 
 /*

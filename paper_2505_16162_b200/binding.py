@@ -22,7 +22,7 @@ STATUS = {0: "OK", 1: "ERR_INVALID_ARG", 2: "ERR_SHAPE", 3: "ERR_CAPACITY", 4: "
 
 EXPORTS = ["knnssd_init", "knnssd_destroy", "knnssd_prefill", "knnssd_select_skipset", "knnssd_set_skipmask",
            "knnssd_draft", "knnssd_verify", "knnssd_generate", "knnssd_decode", "knnssd_get_launch_count", "knnssd_get_length", "knnssd_set_length",
-           "knnssd_set_pending", "knnssd_get_stats", "knnssd_last_error", "knnssd_time_pass", "knnssd_linear",
+           "knnssd_set_pending", "knnssd_get_stats", "knnssd_last_error", "knnssd_time_pass", "knnssd_trace_pass", "knnssd_linear",
            "knnssd_cosine_top1", "knnssd_cosine_top1_static"]
 
 
@@ -74,6 +74,7 @@ def _load():
         "knnssd_get_stats": (I, [P, C.POINTER(Stats)]),
         "knnssd_last_error": (C.c_char_p, [P]),
         "knnssd_time_pass": (I, [P, I, I, I, PF, PI, PF, PI]),
+        "knnssd_trace_pass": (I, [P, I, I, I, PI, PI, PF, PF, PI]),
         "knnssd_linear": (I, [P, I, I, I, P, I, P, P]),
         "knnssd_cosine_top1": (I, [P, P, I, I, PI, PF, P]),
         "knnssd_cosine_top1_static": (I, [P, P, I, I, PI, PF, P]),
@@ -282,6 +283,14 @@ class Session:
         st = Stats()
         self._check(_lib.knnssd_get_stats(self.h, C.byref(st)))
         return {f: getattr(st, f) for f, _ in Stats._fields_}
+
+    def trace_pass(self, which: int, k: int, cap: int = 512):
+        """Per-operation (type, layer, us of work, us at the barrier) of one pass, as stamped by CTA 0."""
+        ty, ly = (C.c_int * cap)(), (C.c_int * cap)()
+        uw, ub = (C.c_float * cap)(), (C.c_float * cap)()
+        n = C.c_int()
+        self._check(_lib.knnssd_trace_pass(self.h, which, k, cap, ty, ly, uw, ub, C.byref(n)))
+        return [(ty[i], ly[i], uw[i], ub[i]) for i in range(n.value)]
 
     def time_pass(self, which: int, k: int, iters: int):
         ms, n, msl, nl = C.c_float(), C.c_int(), C.c_float(), C.c_int()

@@ -4,6 +4,7 @@
 #include "../../include/knnssd.h"
 #include "kernels.cuh"
 #include "linear_stream.cuh"
+#include "pass_kernel.cuh"
 
 #include <cmath>
 #include <cstdio>
@@ -57,6 +58,19 @@ struct knnssd_ctx {
     knnssd_stats stats{};
     cudaEvent_t ev0 = nullptr, ev1 = nullptr, ev2 = nullptr;
     std::string err;
+
+    // persistent pass kernel (bf16 models whose widths are multiples of 128)
+    bool mega_ok = false;
+    pass::Model model{};
+    pass::Op *ops_full = nullptr, *ops_draft = nullptr;     // device op lists
+    int n_ops_full = 0, n_ops_draft = 0, bar_full = 0, bar_draft = 0;   // ops and barriers (without head / hidden parts)
+    std::vector<unsigned char> ops_draft_mask;              // the mask ops_draft was built for
+    unsigned long long *bar = nullptr, bar_total = 0;
+    int *gabort = nullptr, *attn_cnt = nullptr, *amax_cnt = nullptr;
+    float *mpart_o = nullptr, *mamax_v = nullptr;
+    float2 *mpart_ml = nullptr;
+    int *mamax_i = nullptr;
+    unsigned long long *trace = nullptr;
 
     // instrumentation
     long long launches = 0;
@@ -171,6 +185,120 @@ LinearArgs make_args(const void *W0, int rows0, int n_in, const float *x, const 
     return a;
 }
 
+// ---- persistent pass kernel: op lists and launch ----------------------------------------------------------------
+// The list of one pass under a skip mask (nullptr = full model).  n_bar receives the number of grid barriers of the
+// body; the head part (when rows get logits) adds one more.
+std::vector<pass::Op> build_ops(const knnssd_ctx *c, const unsigned char *mask, int *n_bar) {
+    const knnssd_config &g = c->cfg;
+    const int d = g.d_model, hd = g.head_dim, nq = g.n_heads * hd, nkv = g.n_kv_heads * hd, F = g.d_ff, V = g.vocab;
+    std::vector<pass::Op> ops;
+    int bars = 0;
+    auto lin = [&](const void *W0, int rows0, int K, const float *x, const float *gain, float *y, int epi) {
+        pass::Op o{};
+        o.type = pass::OP_LINEAR; o.barrier_after = 1;
+        o.lin.W[0] = reinterpret_cast<const bf16_t *>(W0); o.lin.rows[0] = rows0; o.lin.units = rows0; o.lin.K = K;
+        o.lin.x = x; o.lin.gain = gain; o.lin.eps = g.rms_eps; o.lin.y = y; o.lin.epi = epi; o.lin.M = 1;
+        return o;
+    };
+    pass::Op e{};
+    e.type = pass::OP_EMBED; e.barrier_after = 1;
+    ops.push_back(e); ++bars;
+    const size_t layer_stride = (size_t)g.n_kv_heads * g.max_seq * hd;
+    for (int l = 0; l < g.n_layers; ++l) {
+        const Layer &ly = c->layers[l];
+        if (!mask || !mask[2 * l]) {
+            pass::Op q = lin(ly.wq, nq, d, c->x, ly.attn_norm, c->qkv, EPI_STORE);
+            q.lin.W[1] = reinterpret_cast<const bf16_t *>(ly.wk); q.lin.rows[1] = nkv;
+            q.lin.W[2] = reinterpret_cast<const bf16_t *>(ly.wv); q.lin.rows[2] = nkv;
+            q.lin.units = nq + 2 * nkv; q.layer = l;
+            ops.push_back(q);
+            pass::Op a{};
+            a.type = pass::OP_ATTN; a.barrier_after = 1; a.layer = l;
+            a.kc = reinterpret_cast<bf16_t *>(c->kcache) + (size_t)l * layer_stride;
+            a.vc = reinterpret_cast<bf16_t *>(c->vcache) + (size_t)l * layer_stride;
+            ops.push_back(a);
+            pass::Op o = lin(ly.wo, d, nq, c->attn, nullptr, c->x, EPI_ADD);
+            o.layer = l;
+            ops.push_back(o);
+            bars += 3;
+        }
+        if (!mask || !mask[2 * l + 1]) {
+            pass::Op gu = lin(ly.w_gate, F, d, c->x, ly.mlp_norm, c->act, EPI_SWIGLU);
+            gu.lin.W[1] = reinterpret_cast<const bf16_t *>(ly.w_up); gu.lin.rows[1] = F; gu.layer = l;
+            ops.push_back(gu);
+            pass::Op dn = lin(ly.w_down, d, F, c->act, nullptr, c->x, EPI_ADD);
+            dn.layer = l;
+            ops.push_back(dn);
+            bars += 2;
+        }
+    }
+    pass::Op hdn{};
+    hdn.type = pass::OP_HIDDEN;                      // runs only when the pass wants hidden states; no barrier: reads x only
+    ops.push_back(hdn);
+    pass::Op head = lin(c->lm_head, V, d, c->x, c->final_norm, c->logits, EPI_STORE);
+    head.is_head = 1;                                // runs only when rows get logits; its barrier counts only then
+    ops.push_back(head);
+    pass::Op am{};
+    am.type = pass::OP_ARGMAX;
+    ops.push_back(am);
+    *n_bar = bars;
+    return ops;
+}
+
+knnssd_status upload_ops(knnssd_ctx *c, const std::vector<pass::Op> &ops, pass::Op *dst) {
+    CUDA_TRY(c, cudaMemcpyAsync(dst, ops.data(), ops.size() * sizeof(pass::Op), cudaMemcpyHostToDevice, c->stream));
+    // the host vector goes away after this call: wait for the copy (mask changes are rare)
+    CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+    return KNNSSD_OK;
+}
+
+template <int HD> cudaError_t launch_pass_t(knnssd_ctx *c, const pass::Params &pr) {
+    static bool configured = false;
+    if (!configured) {
+        cudaFuncSetAttribute(pass::pass_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, stream::SMEM_BYTES);
+        configured = true;
+    }
+    void *args[] = {const_cast<pass::Model *>(&c->model), const_cast<pass::Params *>(&pr)};
+    return cudaLaunchCooperativeKernel(reinterpret_cast<void *>(pass::pass_kernel<HD>), dim3(c->n_sms), dim3(stream::NTHREADS),
+                                       args, stream::SMEM_BYTES, c->stream);
+}
+
+// One pass through the persistent kernel.  Errors surface at the caller's next synchronisation.
+void run_pass_mega(knnssd_ctx *c, int M, const int *tok_dev, int pos_off, const unsigned char *mask, int head_row0,
+                   int *argmax_out, bool want_hidden) {
+    pass::Params pr{};
+    int bars;
+    if (!mask) {
+        pr.ops = c->ops_full; pr.n_ops = c->n_ops_full; bars = c->bar_full;
+    } else {
+        const size_t n = 2 * (size_t)c->cfg.n_layers;
+        if (c->ops_draft_mask.size() != n || std::memcmp(c->ops_draft_mask.data(), mask, n) != 0) {
+            const std::vector<pass::Op> ops = build_ops(c, mask, &c->bar_draft);
+            c->n_ops_draft = (int)ops.size();
+            if (upload_ops(c, ops, c->ops_draft) != KNNSSD_OK) return;
+            c->ops_draft_mask.assign(mask, mask + n);
+        }
+        pr.ops = c->ops_draft; pr.n_ops = c->n_ops_draft; bars = c->bar_draft;
+    }
+    pr.M = M; pr.tok = tok_dev; pr.pos_off = pos_off; pr.head_row0 = head_row0; pr.argmax_out = argmax_out;
+    pr.want_hidden = want_hidden ? 1 : 0;
+    pr.bar_base = c->bar_total;
+    if (head_row0 < M) bars += 1;
+    const cudaError_t e = c->cfg.head_dim == 128 ? launch_pass_t<128>(c, pr) : launch_pass_t<64>(c, pr);
+    if (e == cudaSuccess) c->bar_total += (unsigned long long)bars * (unsigned long long)c->n_sms;
+    c->launches++;
+}
+
+// After a pass kernel gave up: bring the barrier counter and the work counters back to their idle state.
+void reset_mega_state(knnssd_ctx *c) {
+    if (!c->mega_ok) return;
+    cudaMemset(c->bar, 0, sizeof(unsigned long long));
+    cudaMemset(c->gabort, 0, sizeof(int));
+    cudaMemset(c->attn_cnt, 0, sizeof(int) * pass::MAXM * c->cfg.n_heads);
+    cudaMemset(c->amax_cnt, 0, sizeof(int));
+    c->bar_total = 0;
+}
+
 // One decoder pass over M rows whose token ids are tok_dev[0..M) at positions state.len + pos_off + m.
 //   mask       nullptr = full model, else [2L] with 1 = skipped
 //   head_row0  first row that gets logits and an arg-max (M = no head at all)
@@ -236,6 +364,7 @@ void run_pass_t(knnssd_ctx *c, int M, const int *tok_dev, int pos_off, const uns
 
 void run_pass(knnssd_ctx *c, int M, const int *tok_dev, int pos_off, const unsigned char *mask, int head_row0,
               int *argmax_out, bool want_hidden) {
+    if (c->mega_ok && M <= pass::MAXM) { run_pass_mega(c, M, tok_dev, pos_off, mask, head_row0, argmax_out, want_hidden); return; }
     if (c->cfg.dtype) run_pass_t<bf16_t>(c, M, tok_dev, pos_off, mask, head_row0, argmax_out, want_hidden);
     else run_pass_t<float>(c, M, tok_dev, pos_off, mask, head_row0, argmax_out, want_hidden);
 }
@@ -254,6 +383,7 @@ knnssd_status check_stream_err(knnssd_ctx *c, const char *what) {
         return fail(c, KNNSSD_ERR_CUDA, std::string(what) + ": cannot read the device error word");
     if (code) {
         cudaMemset(stream_err_ptr(), 0, sizeof(int));
+        reset_mega_state(c);
         return fail(c, KNNSSD_ERR_TIMEOUT, std::string(what) + ": a device-side wait gave up (code " + std::to_string(code) + ")");
     }
     return KNNSSD_OK;
@@ -262,7 +392,9 @@ knnssd_status check_stream_err(knnssd_ctx *c, const char *what) {
 void free_all(knnssd_ctx *c) {
     void *ptrs[] = {c->kcache, c->vcache, c->x, c->qkv, c->attn, c->act, c->logits, c->hfinal, c->part_o, c->pooled,
                     c->anchor_inv_norm, c->cosines, c->amax_v, c->part_ml, c->rope_cs, c->pool_sum, c->inv_freq, c->chain,
-                    c->target, c->prompt, c->out_tokens, c->accept_log, c->amax_i, c->flag, c->knn_out, c->state};
+                    c->target, c->prompt, c->out_tokens, c->accept_log, c->amax_i, c->flag, c->knn_out, c->state,
+                    c->ops_full, c->ops_draft, c->bar, c->gabort, c->attn_cnt, c->amax_cnt, c->mpart_o, c->mamax_v, c->mpart_ml,
+                    c->mamax_i, c->trace};
     for (void *p : ptrs)
         if (p) cudaFree(p);
     if (c->pinned) cudaFreeHost(c->pinned);
@@ -297,8 +429,9 @@ knnssd_status do_prefill(knnssd_ctx *c, const int *tokens_host, int n, float *po
     set_state_kernel<<<1, 1, 0, s>>>(c->state, 0, 0);
     cudaEventRecord(c->ev0, s);
     const int d = g.d_model;
-    for (int t0 = 0; t0 < n; t0 += kMaxRows) {
-        const int M = (n - t0 < kMaxRows) ? n - t0 : kMaxRows;
+    const int chunk = c->mega_ok ? pass::MAXM : kMaxRows;   // rows per pass: what the faster path takes
+    for (int t0 = 0; t0 < n; t0 += chunk) {
+        const int M = (n - t0 < chunk) ? n - t0 : chunk;
         const bool last = t0 + M == n;
         // mean pooling needs every row's final hidden state; last-token pooling only the last row's
         const bool hidden = g.pool_mode == 0 || last;
@@ -466,6 +599,38 @@ knnssd_status knnssd_init(const knnssd_config *cfg, const knnssd_weights *w, con
     cudaMemcpyAsync(c->pinned, c->flag, sizeof(int), cudaMemcpyDeviceToHost, c->stream);
     if (sync_check(c, "init") != KNNSSD_OK) return bail(KNNSSD_ERR_CUDA);
     if (c->pinned[0]) return bail(KNNSSD_ERR_DEGENERATE);
+    // the persistent pass kernel serves bf16 models whose linear maps all have inputs that are multiples of 128
+    int coop = 0;
+    cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, c->device);
+    if (g.dtype == 1 && coop && d % 128 == 0 && nq % 128 == 0 && g.d_ff % 128 == 0 && d >= 256 && nq >= 256 && g.d_ff >= 256) {
+        const int n_seg_max = (g.max_seq + pass::SEGP - 1) / pass::SEGP;
+        const int n_ops_cap = 5 * g.n_layers + 8;
+        bool ok2 = true;
+        ok2 &= dev_alloc(&c->ops_full, (size_t)n_ops_cap) == cudaSuccess;
+        ok2 &= dev_alloc(&c->ops_draft, (size_t)n_ops_cap) == cudaSuccess;
+        ok2 &= dev_alloc(&c->bar, 1) == cudaSuccess;
+        ok2 &= dev_alloc(&c->gabort, 1) == cudaSuccess;
+        ok2 &= dev_alloc(&c->attn_cnt, (size_t)pass::MAXM * g.n_heads) == cudaSuccess;
+        ok2 &= dev_alloc(&c->amax_cnt, 1) == cudaSuccess;
+        ok2 &= dev_alloc(&c->mpart_o, (size_t)pass::MAXM * g.n_heads * n_seg_max * hd) == cudaSuccess;
+        ok2 &= dev_alloc(&c->mpart_ml, (size_t)pass::MAXM * g.n_heads * n_seg_max) == cudaSuccess;
+        ok2 &= dev_alloc(&c->mamax_v, (size_t)pass::MAXM * c->n_sms) == cudaSuccess;
+        ok2 &= dev_alloc(&c->mamax_i, (size_t)pass::MAXM * c->n_sms) == cudaSuccess;
+        ok2 &= dev_alloc(&c->trace, (size_t)2 * n_ops_cap) == cudaSuccess;
+        if (!ok2) { cudaGetLastError(); return bail(KNNSSD_ERR_CUDA); }
+        pass::Model &md = c->model;
+        md.tok_embed = reinterpret_cast<const bf16_t *>(c->tok_embed); md.final_norm = c->final_norm; md.rms_eps = g.rms_eps;
+        md.d_model = d; md.H = g.n_heads; md.Hkv = g.n_kv_heads; md.hd = hd; md.vocab = g.vocab; md.max_seq = g.max_seq;
+        md.n_seg_max = n_seg_max; md.inv_freq = c->inv_freq;
+        md.x = c->x; md.qkv = c->qkv; md.attn = c->attn; md.logits = c->logits; md.hfinal = c->hfinal; md.rope_cs = c->rope_cs;
+        md.part_o = c->mpart_o; md.part_ml = c->mpart_ml; md.attn_cnt = c->attn_cnt; md.amax_v = c->mamax_v; md.amax_i = c->mamax_i;
+        md.amax_cnt = c->amax_cnt; md.state = c->state; md.bar = c->bar; md.gabort = c->gabort; md.err = stream_err_ptr();
+        c->mega_ok = true;
+        reset_mega_state(c);
+        const std::vector<pass::Op> ops = build_ops(c, nullptr, &c->bar_full);
+        c->n_ops_full = (int)ops.size();
+        if (upload_ops(c, ops, c->ops_full) != KNNSSD_OK) return bail(KNNSSD_ERR_CUDA);
+    }
     *out = c;
     return KNNSSD_OK;
 }
@@ -736,6 +901,57 @@ knnssd_status knnssd_time_pass(knnssd_ctx *c, int which, int k, int iters, float
     CUDA_TRY(c, cudaMemcpyAsync(c->chain, &c->pending, sizeof(int), cudaMemcpyHostToDevice, s));
     st = sync_check(c, "time_pass restore");
     if (st == KNNSSD_OK) st = check_stream_err(c, "time_pass");
+    return st;
+}
+
+knnssd_status knnssd_trace_pass(knnssd_ctx *c, int which, int k, int cap, int *op_types, int *op_layers, float *us_work,
+                                float *us_barrier, int *n_ops) {
+    if (!c || !op_types || !op_layers || !us_work || !us_barrier || !n_ops) return KNNSSD_ERR_INVALID_ARG;
+    DeviceGuard dg(c->device);
+    const knnssd_config &g = c->cfg;
+    if ((which != 0 && which != 1) || k < 0 || k > g.max_draft || cap < 1) return fail(c, KNNSSD_ERR_INVALID_ARG, "trace_pass: bad arguments");
+    if (!c->mega_ok || (which == 1 && k + 1 > pass::MAXM)) return fail(c, KNNSSD_ERR_SHAPE, "trace_pass: this pass does not run in the persistent kernel");
+    if (!c->prefilled) return fail(c, KNNSSD_ERR_STATE, "trace_pass: prefill first");
+    if (which == 0 && !c->has_mask) return fail(c, KNNSSD_ERR_STATE, "trace_pass: no active skip mask");
+    if (c->len + k + 1 > g.max_seq) return fail(c, KNNSSD_ERR_CAPACITY, "trace_pass: len + k + 1 exceeds max_seq");
+    cudaStream_t s = c->stream;
+    std::vector<int> fill(k + 1, c->pending);
+    CUDA_TRY(c, cudaMemcpyAsync(c->chain, fill.data(), sizeof(int) * (k + 1), cudaMemcpyHostToDevice, s));
+    auto one = [&]() {
+        if (which == 0) run_pass(c, 1, c->chain, 0, c->active_mask.data(), 0, c->target, false);
+        else run_pass(c, k + 1, c->chain, 0, nullptr, 0, c->target, false);
+    };
+    one();                                       // warm-up (also builds the draft list for the active mask)
+    knnssd_status st = sync_check(c, "trace_pass warm-up");
+    if (st != KNNSSD_OK) return st;
+    std::vector<pass::Op> ops;
+    int bars = 0;
+    ops = build_ops(c, which == 0 ? c->active_mask.data() : nullptr, &bars);
+    const int n = (int)ops.size();
+    CUDA_TRY(c, cudaMemsetAsync(c->trace, 0, sizeof(unsigned long long) * 2 * n, s));
+    c->model.trace = c->trace;
+    one();
+    c->model.trace = nullptr;
+    std::vector<unsigned long long> t(2 * (size_t)n);
+    CUDA_TRY(c, cudaMemcpyAsync(t.data(), c->trace, sizeof(unsigned long long) * 2 * n, cudaMemcpyDeviceToHost, s));
+    st = sync_check(c, "trace_pass");
+    if (st != KNNSSD_OK) return st;
+    unsigned long long prev = 0;
+    int out = 0;
+    for (int i = 0; i < n && out < cap; ++i) {
+        if (t[2 * i] == 0) continue;
+        if (prev == 0) prev = t[2 * i];          // the first operation's start is not stamped: its work reads as 0
+        op_types[out] = ops[i].type == pass::OP_LINEAR ? (ops[i].is_head ? 14 : 10 + ops[i].lin.epi) : ops[i].type;
+        op_layers[out] = ops[i].layer;
+        us_work[out] = (float)((double)(t[2 * i] - prev) * 1e-3);
+        us_barrier[out] = (float)((double)(t[2 * i + 1] - t[2 * i]) * 1e-3);
+        prev = t[2 * i + 1];
+        ++out;
+    }
+    *n_ops = out;
+    CUDA_TRY(c, cudaMemcpyAsync(c->chain, &c->pending, sizeof(int), cudaMemcpyHostToDevice, s));
+    st = sync_check(c, "trace_pass restore");
+    if (st == KNNSSD_OK) st = check_stream_err(c, "trace_pass");
     return st;
 }
 
