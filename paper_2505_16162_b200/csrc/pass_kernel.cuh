@@ -199,12 +199,13 @@ __device__ __forceinline__ void argmax_phase(const Model &md, const Params &pr, 
 // ---- attention over the KV cache ------------------------------------------------------------------------------
 // Rows m = 0..M-1 sit at positions P0 + m; row m attends to positions [0, P0 + m].  The context is cut at fixed
 // absolute boundaries into segments of SEGP positions; one warp handles one (query head, segment) for all rows:
-// it reads each K and V row of the segment once (8 bytes per lane, a whole 256-byte row per warp access), takes
-// the dot products of a 32-position chunk with a transposed butterfly (lane i ends up with position i's score),
-// keeps an online softmax per row and writes an un-normalised partial (max, sum, o).  The warp that completes the
-// last segment of a (row, head) merges the partials in segment order.  K/V of the M new positions come from the
-// projection buffer (rotated, rounded to bf16 exactly as they are stored); the warp of the first query head of
-// each KV group also writes them to the cache.
+// it reads each K and V row of the segment once (8 bytes per lane, a whole 256-byte row per warp access), in
+// register batches of 16 positions with the next batch always in flight, takes the 16 dot products of a batch with
+// a transposed butterfly, keeps an online softmax per row over 32-position chunks and writes an un-normalised
+// partial (max, sum, o).  The warp that completes the last segment of a (row, head) merges the partials in segment
+// order.  K/V of the M new positions come from the projection buffer (rotated, rounded to bf16 exactly as they are
+// stored); the warp of the first query head of each KV group also writes them to the cache.  Loops over batches stay
+// rolled on purpose: the unrolled form of this code does not fit the instruction cache.
 template <int HD> struct KVVec;
 template <> struct KVVec<128> { typedef uint2 T; };
 template <> struct KVVec<64> { typedef uint32_t T; };
@@ -229,10 +230,10 @@ template <int HD> __device__ __forceinline__ typename KVVec<HD>::T kv_zero();
 template <> __device__ __forceinline__ uint2 kv_zero<128>() { return make_uint2(0u, 0u); }
 template <> __device__ __forceinline__ uint32_t kv_zero<64>() { return 0u; }
 
-// Sum over lanes of v[i], delivered to lane i (i = 0..31): 31 shuffles instead of 32 x 5.
-__device__ __forceinline__ float transposed_sum32(float (&v)[32], int lane) {
+// Sum over lanes of v[i], delivered to every lane whose (lane & 15) == i (i = 0..15): 16 shuffles for 16 sums.
+__device__ __forceinline__ float transposed_sum16(float (&v)[16], int lane) {
 #pragma unroll
-    for (int step = 16; step >= 1; step >>= 1) {
+    for (int step = 8; step >= 1; step >>= 1) {
         const bool up = (lane & step) != 0;
 #pragma unroll
         for (int i = 0; i < step; ++i) {
@@ -241,10 +242,13 @@ __device__ __forceinline__ float transposed_sum32(float (&v)[32], int lane) {
             v[i] = keep + __shfl_xor_sync(0xffffffffu, send, step);
         }
     }
-    return v[0];
+    return v[0] + __shfl_xor_sync(0xffffffffu, v[0], 16);
 }
 
-template <int HD>
+constexpr int ATT_B = 16;          // positions per register batch (one batch is always in flight ahead of the math)
+
+// MR = rows the code is unrolled for (1: draft steps, 8: verification); rows >= M are skipped at run time.
+template <int HD, int MR>
 __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const Params &pr, const Ring &r, int cta, int n_cta,
                                            int warp, int lane) {
     constexpr int DPL = HD / 32, HALF = HD / 2;
@@ -269,7 +273,7 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
 
         // new K/V rows that fall into this segment: rotate, round, stash (and store if this warp is the writer)
         __syncwarp();
-        for (int mp = max(0, p_begin - P0); mp < M && P0 + mp < p_end; ++mp) {
+        for (int mp = m_first; mp < M && P0 + mp < p_end; ++mp) {
             const float *kraw = md.qkv + (size_t)mp * qstride + (size_t)(H + kvh) * HD + d0;
             const float *vraw = md.qkv + (size_t)mp * qstride + (size_t)(H + Hkv + kvh) * HD + d0;
             float kf[DPL], vf[DPL];
@@ -292,10 +296,10 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
         __syncwarp();
 
         // rotated queries of the rows that see this segment
-        float q[MAXM][DPL], o[MAXM][DPL], mx[MAXM], l[MAXM];
+        float q[MR][DPL], o[MR][DPL], mx[MR], l[MR], sreg[MR];
 #pragma unroll
-        for (int m = 0; m < MAXM; ++m) {
-            mx[m] = -INFINITY; l[m] = 0.f;
+        for (int m = 0; m < MR; ++m) {
+            mx[m] = -INFINITY; l[m] = 0.f; sreg[m] = 0.f;
 #pragma unroll
             for (int e = 0; e < DPL; ++e) { q[m][e] = 0.f; o[m][e] = 0.f; }
             if (m >= m_first && m < M) {
@@ -311,66 +315,82 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
             }
         }
 
-        for (int p0 = p_begin; p0 < p_end; p0 += 32) {
-            VT kv[32];
-            float prob[MAXM];
-            // ---- K rows of the chunk, scores, online softmax ----
+        // The segment as a flat list of register batches: per 32-position chunk, K rows 0-15, K rows 16-31, V rows
+        // 0-15, V rows 16-31.  Batch it + 1 is loading while batch it is being used.
+        auto load_batch = [&](int it, VT (&dst)[ATT_B]) {
+            const int sub = it & 3, pb = p_begin + (it >> 2) * 32 + (sub & 1) * ATT_B;
+            const bf16_t *cache = (sub >> 1) ? vbase : kbase;
+            const bf16_t *stash = (sub >> 1) ? stash_v : stash_k;
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                const int p = p0 + j;
-                const bf16_t *src = p < P0 ? kbase + (size_t)p * HD + d0 : stash_k + (p - P0) * HD + d0;
-                kv[j] = p < p_end ? *reinterpret_cast<const VT *>(src) : kv_zero<HD>();
+            for (int j = 0; j < ATT_B; ++j) {
+                const int p = pb + j;
+                const bf16_t *src = p < P0 ? cache + (size_t)p * HD + d0 : stash + (p - P0) * HD + d0;
+                dst[j] = p < p_end ? *reinterpret_cast<const VT *>(src) : kv_zero<HD>();
             }
+        };
+        const int n_it = 4 * ((p_end - p_begin + 31) >> 5);
+        VT cur[ATT_B], nxt[ATT_B];
+        load_batch(0, cur);
+        for (int it = 0; it < n_it; ++it) {
+            if (it + 1 < n_it) load_batch(it + 1, nxt);
+            const int sub = it & 3, half = sub & 1, p0 = p_begin + (it >> 2) * 32;
+            if (sub < 2) {
+                // ---- scores of 16 positions: lane (half * 16 + i) keeps position i's score ----
 #pragma unroll
-            for (int m = 0; m < MAXM; ++m) {
-                prob[m] = 0.f;
-                if (m < m_first || m >= M || p0 > P0 + m) continue;      // row does not see this chunk
-                float part[32];
+                for (int m = 0; m < MR; ++m) {
+                    if (m < m_first || m >= M || p0 > P0 + m) continue;      // row does not see this chunk
+                    float part[ATT_B];
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    float kf[DPL];
-                    kv_unpack<HD>(kv[j], kf);
-                    float s = 0.f;
+                    for (int j = 0; j < ATT_B; ++j) {
+                        float kf[DPL];
+                        kv_unpack<HD>(cur[j], kf);
+                        float s = 0.f;
 #pragma unroll
-                    for (int e = 0; e < DPL; ++e) s = fmaf(q[m][e], kf[e], s);
-                    part[j] = s;
+                        for (int e = 0; e < DPL; ++e) s = fmaf(q[m][e], kf[e], s);
+                        part[j] = s;
+                    }
+                    const float tot = transposed_sum16(part, lane);
+                    if ((lane >> 4) == half) sreg[m] = tot;
                 }
-                float s = transposed_sum32(part, lane) * scale;
-                const bool valid = p0 + lane <= P0 + m;
-                s = valid ? s : -INFINITY;
-                const float mnew = fmaxf(mx[m], warp_max(s));
-                const float corr = expf(mx[m] - mnew);
-                const float pj = valid ? expf(s - mnew) : 0.f;
-                l[m] = fmaf(l[m], corr, warp_sum(pj));
+                if (sub == 1) {
+                    // ---- online softmax over the chunk's 32 positions (lane = position) ----
 #pragma unroll
-                for (int e = 0; e < DPL; ++e) o[m][e] *= corr;
-                mx[m] = mnew;
-                prob[m] = pj;
-            }
-            // ---- V rows of the chunk, o += p V ----
+                    for (int m = 0; m < MR; ++m) {
+                        if (m < m_first || m >= M || p0 > P0 + m) continue;
+                        const bool valid = p0 + lane <= P0 + m;
+                        const float s = valid ? sreg[m] * scale : -INFINITY;
+                        const float mnew = fmaxf(mx[m], warp_max(s));
+                        const float corr = expf(mx[m] - mnew);
+                        const float pj = valid ? expf(s - mnew) : 0.f;
+                        l[m] = fmaf(l[m], corr, warp_sum(pj));
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                const int p = p0 + j;
-                const bf16_t *src = p < P0 ? vbase + (size_t)p * HD + d0 : stash_v + (p - P0) * HD + d0;
-                kv[j] = p < p_end ? *reinterpret_cast<const VT *>(src) : kv_zero<HD>();
-            }
+                        for (int e = 0; e < DPL; ++e) o[m][e] *= corr;
+                        mx[m] = mnew;
+                        sreg[m] = pj;
+                    }
+                }
+            } else {
+                // ---- o += p V over 16 positions ----
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                float vf[DPL];
-                kv_unpack<HD>(kv[j], vf);
+                for (int j = 0; j < ATT_B; ++j) {
+                    float vf[DPL];
+                    kv_unpack<HD>(cur[j], vf);
 #pragma unroll
-                for (int m = 0; m < MAXM; ++m) {
-                    if (m < m_first || m >= M || p0 > P0 + m) continue;
-                    const float pj = __shfl_sync(0xffffffffu, prob[m], j);
+                    for (int m = 0; m < MR; ++m) {
+                        if (m < m_first || m >= M || p0 > P0 + m) continue;
+                        const float pj = __shfl_sync(0xffffffffu, sreg[m], half * ATT_B + j);
 #pragma unroll
-                    for (int e = 0; e < DPL; ++e) o[m][e] = fmaf(pj, vf[e], o[m][e]);
+                        for (int e = 0; e < DPL; ++e) o[m][e] = fmaf(pj, vf[e], o[m][e]);
+                    }
                 }
             }
+#pragma unroll
+            for (int j = 0; j < ATT_B; ++j) cur[j] = nxt[j];
         }
 
         // ---- partials out; the last warp of a (row, head) merges ----
 #pragma unroll
-        for (int m = 0; m < MAXM; ++m) {
+        for (int m = 0; m < MR; ++m) {
             if (m < m_first || m >= M) continue;
             const size_t pidx = ((size_t)m * H + h) * md.n_seg_max + seg;
             if (lane == 0) __stcg(md.part_ml + pidx, make_float2(mx[m], l[m]));
@@ -457,7 +477,10 @@ __global__ void __launch_bounds__(stream::NTHREADS, 1) pass_kernel(const Model m
             if (ran) stream::consume_linear(lp, r, cta, n_cta, warp, lane, w_use, alive);
         } else if (alive) {
             if (op.type == OP_EMBED) embed_phase(md, pr, cta, tid);
-            else if (op.type == OP_ATTN) attn_phase<HD>(md, op, pr, r, cta, n_cta, warp, lane);
+            else if (op.type == OP_ATTN) {
+                if (pr.M == 1) attn_phase<HD, 1>(md, op, pr, r, cta, n_cta, warp, lane);
+                else attn_phase<HD, MAXM>(md, op, pr, r, cta, n_cta, warp, lane);
+            }
             else if (op.type == OP_HIDDEN) { if (pr.want_hidden) hidden_phase(md, pr, r, cta, tid); else ran = false; }
             else if (op.type == OP_ARGMAX) { if (pr.head_row0 < pr.M) argmax_phase(md, pr, r, cta, n_cta, tid); else ran = false; }
         }
