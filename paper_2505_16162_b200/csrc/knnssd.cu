@@ -71,6 +71,8 @@ struct knnssd_ctx {
     float2 *mpart_ml = nullptr;
     int *mamax_i = nullptr;
     unsigned long long *trace = nullptr;
+    uint32_t *xs_x = nullptr, *xs_attn = nullptr, *xs_act = nullptr;   // pre-split activations (see LinPhase::xs)
+    float *ssp = nullptr;                                              // [MAXM][n_sms] partial sums of squares of x rows
 
     // instrumentation
     long long launches = 0;
@@ -202,6 +204,7 @@ std::vector<pass::Op> build_ops(const knnssd_ctx *c, const unsigned char *mask, 
     };
     pass::Op e{};
     e.type = pass::OP_EMBED; e.barrier_after = 1;
+    e.lin.K = d; e.lin.ys = c->xs_x; e.lin.ss_out = c->ssp;
     ops.push_back(e); ++bars;
     const size_t layer_stride = (size_t)g.n_kv_heads * g.max_seq * hd;
     for (int l = 0; l < g.n_layers; ++l) {
@@ -211,23 +214,28 @@ std::vector<pass::Op> build_ops(const knnssd_ctx *c, const unsigned char *mask, 
             q.lin.W[1] = reinterpret_cast<const bf16_t *>(ly.wk); q.lin.rows[1] = nkv;
             q.lin.W[2] = reinterpret_cast<const bf16_t *>(ly.wv); q.lin.rows[2] = nkv;
             q.lin.units = nq + 2 * nkv; q.layer = l;
+            q.lin.xs = c->xs_x; q.lin.ss_in = c->ssp;
             ops.push_back(q);
             pass::Op a{};
             a.type = pass::OP_ATTN; a.barrier_after = 1; a.layer = l;
             a.kc = reinterpret_cast<bf16_t *>(c->kcache) + (size_t)l * layer_stride;
             a.vc = reinterpret_cast<bf16_t *>(c->vcache) + (size_t)l * layer_stride;
+            a.lin.ys = c->xs_attn;
             ops.push_back(a);
             pass::Op o = lin(ly.wo, d, nq, c->attn, nullptr, c->x, EPI_ADD);
             o.layer = l;
+            o.lin.xs = c->xs_attn; o.lin.ys = c->xs_x; o.lin.ss_out = c->ssp;
             ops.push_back(o);
             bars += 3;
         }
         if (!mask || !mask[2 * l + 1]) {
             pass::Op gu = lin(ly.w_gate, F, d, c->x, ly.mlp_norm, c->act, EPI_SWIGLU);
             gu.lin.W[1] = reinterpret_cast<const bf16_t *>(ly.w_up); gu.lin.rows[1] = F; gu.layer = l;
+            gu.lin.xs = c->xs_x; gu.lin.ss_in = c->ssp; gu.lin.ys = c->xs_act;
             ops.push_back(gu);
             pass::Op dn = lin(ly.w_down, d, F, c->act, nullptr, c->x, EPI_ADD);
             dn.layer = l;
+            dn.lin.xs = c->xs_act; dn.lin.ys = c->xs_x; dn.lin.ss_out = c->ssp;
             ops.push_back(dn);
             bars += 2;
         }
@@ -237,10 +245,18 @@ std::vector<pass::Op> build_ops(const knnssd_ctx *c, const unsigned char *mask, 
     ops.push_back(hdn);
     pass::Op head = lin(c->lm_head, V, d, c->x, c->final_norm, c->logits, EPI_STORE);
     head.is_head = 1;                                // runs only when rows get logits; its barrier counts only then
+    head.lin.xs = c->xs_x; head.lin.ss_in = c->ssp;
     ops.push_back(head);
     pass::Op am{};
     am.type = pass::OP_ARGMAX;
     ops.push_back(am);
+    // whoever writes the residual stream also writes it pre-split, times the gain of the RMSNorm that reads it next
+    const float *next_gain = nullptr;
+    for (int i = (int)ops.size() - 1; i >= 0; --i) {
+        pass::Op &o = ops[i];
+        if (o.type == pass::OP_EMBED || (o.type == pass::OP_LINEAR && o.lin.epi == EPI_ADD)) o.lin.next_gain = next_gain;
+        if (o.type == pass::OP_LINEAR && o.lin.gain) next_gain = o.lin.gain;
+    }
     *n_bar = bars;
     return ops;
 }
@@ -394,7 +410,7 @@ void free_all(knnssd_ctx *c) {
                     c->anchor_inv_norm, c->cosines, c->amax_v, c->part_ml, c->rope_cs, c->pool_sum, c->inv_freq, c->chain,
                     c->target, c->prompt, c->out_tokens, c->accept_log, c->amax_i, c->flag, c->knn_out, c->state,
                     c->ops_full, c->ops_draft, c->bar, c->gabort, c->attn_cnt, c->amax_cnt, c->mpart_o, c->mamax_v, c->mpart_ml,
-                    c->mamax_i, c->trace};
+                    c->mamax_i, c->trace, c->xs_x, c->xs_attn, c->xs_act, c->ssp};
     for (void *p : ptrs)
         if (p) cudaFree(p);
     if (c->pinned) cudaFreeHost(c->pinned);
@@ -567,7 +583,7 @@ knnssd_status knnssd_init(const knnssd_config *cfg, const knnssd_weights *w, con
     ok &= dev_alloc(&c->hfinal, (size_t)kMaxRows * d) == cudaSuccess;
     ok &= dev_alloc(&c->part_o, (size_t)kMaxRows * g.n_heads * c->n_splits * hd) == cudaSuccess;
     ok &= dev_alloc(&c->part_ml, (size_t)kMaxRows * g.n_heads * c->n_splits) == cudaSuccess;
-    ok &= dev_alloc(&c->rope_cs, (size_t)kMaxRows * (hd / 2)) == cudaSuccess;
+    ok &= dev_alloc(&c->rope_cs, (size_t)(c->n_sms > 1 ? c->n_sms : 1) * kMaxRows * (hd / 2)) == cudaSuccess;   // one copy per CTA of the pass kernel
     ok &= dev_alloc(&c->pooled, (size_t)d) == cudaSuccess;
     ok &= dev_alloc(&c->pool_sum, (size_t)d) == cudaSuccess;
     ok &= dev_alloc(&c->inv_freq, (size_t)hd / 2) == cudaSuccess;
@@ -602,7 +618,8 @@ knnssd_status knnssd_init(const knnssd_config *cfg, const knnssd_weights *w, con
     // the persistent pass kernel serves bf16 models whose linear maps all have inputs that are multiples of 128
     int coop = 0;
     cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, c->device);
-    if (g.dtype == 1 && coop && d % 128 == 0 && nq % 128 == 0 && g.d_ff % 128 == 0 && d >= 256 && nq >= 256 && g.d_ff >= 256) {
+    if (g.dtype == 1 && coop && d % 128 == 0 && nq % 128 == 0 && g.d_ff % 128 == 0 && d >= 256 && nq >= 256 && g.d_ff >= 256 &&
+        g.max_seq <= 64 * pass::SEGP) {            // the attention merge keeps at most 64 segment statistics per warp
         const int n_seg_max = (g.max_seq + pass::SEGP - 1) / pass::SEGP;
         const int n_ops_cap = 5 * g.n_layers + 8;
         bool ok2 = true;
@@ -617,6 +634,10 @@ knnssd_status knnssd_init(const knnssd_config *cfg, const knnssd_weights *w, con
         ok2 &= dev_alloc(&c->mamax_v, (size_t)pass::MAXM * c->n_sms) == cudaSuccess;
         ok2 &= dev_alloc(&c->mamax_i, (size_t)pass::MAXM * c->n_sms) == cudaSuccess;
         ok2 &= dev_alloc(&c->trace, (size_t)2 * n_ops_cap) == cudaSuccess;
+        ok2 &= dev_alloc(&c->xs_x, (size_t)pass::MAXM * (d / 128) * 192) == cudaSuccess;
+        ok2 &= dev_alloc(&c->xs_attn, (size_t)pass::MAXM * (nq / 128) * 192) == cudaSuccess;
+        ok2 &= dev_alloc(&c->xs_act, (size_t)pass::MAXM * (g.d_ff / 128) * 192) == cudaSuccess;
+        ok2 &= dev_alloc(&c->ssp, (size_t)pass::MAXM * c->n_sms) == cudaSuccess;
         if (!ok2) { cudaGetLastError(); return bail(KNNSSD_ERR_CUDA); }
         pass::Model &md = c->model;
         md.tok_embed = reinterpret_cast<const bf16_t *>(c->tok_embed); md.final_norm = c->final_norm; md.rms_eps = g.rms_eps;

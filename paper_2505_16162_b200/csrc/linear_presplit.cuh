@@ -1,0 +1,152 @@
+// Consumer half of the weight-streaming linear engine for PRE-SPLIT activations (persistent pass kernel).
+//
+// Same ring, same tiles, same sum order per output as consume_linear, but the activation operand arrives already
+// split into its three bf16 terms and laid out fragment by fragment (LinPhase::xs), written once by whoever produced
+// the activation.  The consumer therefore spends no arithmetic on the split that every CTA would otherwise repeat:
+// per column tile a lane loads twelve 16-byte pieces, one tile ahead of the tensor-core work.  RMSNorm's scalar comes
+// from per-CTA partial sums of squares that the producer of the row left in LinPhase::ss_in.
+//
+// The epilogue writes what the NEXT map needs: the fp32 result where something reads it as fp32 (projection buffer,
+// residual stream, logits) and, for the residual update and the SwiGLU product, the pre-split form (times the next
+// RMSNorm's gain) plus this CTA's partial sums of squares.
+#pragma once
+#include "linear_stream.cuh"
+
+namespace knnssd {
+namespace stream {
+
+__device__ __forceinline__ uint4 ld_frag4(const uint32_t *p) { return __ldcg(reinterpret_cast<const uint4 *>(p)); }
+
+__device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring &r, int cta, int n_cta, int warp, int lane,
+                                                   int &w_use, bool &alive) {
+    const Share s = make_share(p, cta, n_cta);
+    const int tid = warp * 32 + lane;
+    const int g8 = lane >> 2, t4 = lane & 3;
+    const int lm_row = (lane & 7) + ((lane >> 3) & 1) * 8, lm_col = (lane >> 4) * 8;   // ldmatrix source of this lane
+    const bool normed = p.ss_in != nullptr;
+    const bool row_live = g8 < p.M;
+    const int nslots = p.K >> 7;
+    // this lane's 16-word runs: row g8, lane group t4; + slot * 192 + term * 64
+    const uint32_t *xsrow = p.xs + (((size_t)min(g8, p.M - 1) * nslots * 3) * 4 + t4) * 16;
+    int ws = w_use % WS, it = w_use / WS;
+    float *red = r.red, *red_ss = r.red_ss;
+
+    // RMSNorm scalar of every row from the producers' partial sums: warp w takes row w, lanes take CTAs lane, lane + 32, ...
+    if (normed && warp < p.M) {
+        float tot = 0.f;
+        for (int c = lane; c < n_cta; c += 32) tot += __ldcg(p.ss_in + (size_t)warp * n_cta + c);
+        tot = warp_sum(tot);
+        if (lane == 0) red_ss[warp] = 1.0f / sqrtf(tot / (float)p.K + p.eps);
+    }
+    float ss_acc = 0.f;                                     // token thread (tid < M): this CTA's sum of squares of y
+
+    for (int b = 0; b < s.n_batches; ++b) {
+        const int g0 = b * GB, ng = min(s.n_groups - g0, GB);
+        float acc[GB][4];
+#pragma unroll
+        for (int i = 0; i < GB; ++i) { acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f; }
+        uint4 nx[3][4];                                      // fragments of the next column tile (hi, mid, lo)
+        auto fetch = [&](int kt) {
+            const int slot = kt * NCW + warp;
+            const bool ld = alive && row_live && slot < nslots;
+#pragma unroll
+            for (int t = 0; t < 3; ++t)
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                    nx[t][q] = ld ? ld_frag4(xsrow + (size_t)slot * 192 + t * 64 + q * 4) : make_uint4(0u, 0u, 0u, 0u);
+        };
+        fetch(0);
+        for (int kt = 0; kt < s.n_kt; ++kt) {
+            const bool slot_valid = kt * NCW + warp < nslots;
+            uint32_t bh[KSTEPS][2], bm[KSTEPS][2], bl[KSTEPS][2];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                bh[2 * q][0] = nx[0][q].x; bh[2 * q][1] = nx[0][q].y; bh[2 * q + 1][0] = nx[0][q].z; bh[2 * q + 1][1] = nx[0][q].w;
+                bm[2 * q][0] = nx[1][q].x; bm[2 * q][1] = nx[1][q].y; bm[2 * q + 1][0] = nx[1][q].z; bm[2 * q + 1][1] = nx[1][q].w;
+                bl[2 * q][0] = nx[2][q].x; bl[2 * q][1] = nx[2][q].y; bl[2 * q + 1][0] = nx[2][q].z; bl[2 * q + 1][1] = nx[2][q].w;
+            }
+            if (kt + 1 < s.n_kt) fetch(kt + 1);
+#pragma unroll
+            for (int gi = 0; gi < GB; ++gi) {
+                if (gi >= ng) break;
+                if (alive) alive = mbar_wait(&r.full_w[ws], it & 1, r.abort_flag, r.err, 5);
+                if (alive && slot_valid) {
+                    const uint32_t base = smem_u32(r.wring + ws * WSTAGE) + lm_row * WPITCH + (warp * SLOT + lm_col) * 2;
+                    // six independent accumulator chains: term x parity of the k-step
+                    float tl[2][4] = {}, tm[2][4] = {}, th[2][4] = {};
+#pragma unroll
+                    for (int j = 0; j < KSTEPS; ++j) {
+                        uint32_t a0, a1, a2, a3;
+                        ldmatrix_x4(base + j * 32, a0, a1, a2, a3);
+                        mma_bf16(tl[j & 1], a0, a1, a2, a3, bl[j][0], bl[j][1]);
+                        mma_bf16(tm[j & 1], a0, a1, a2, a3, bm[j][0], bm[j][1]);
+                        mma_bf16(th[j & 1], a0, a1, a2, a3, bh[j][0], bh[j][1]);
+                    }
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        acc[gi][e] += ((tl[0][e] + tl[1][e]) + (tm[0][e] + tm[1][e])) + (th[0][e] + th[1][e]);
+                }
+                __syncwarp();
+                if (alive && lane == 0) mbar_arrive(&r.empty_w[ws]);
+                ++w_use;
+                if (++ws == WS) { ws = 0; ++it; }
+            }
+        }
+        // ---- batch end: partial sums of the 8 column slots meet in shared memory, in warp order ----
+#pragma unroll
+        for (int gi = 0; gi < GB; ++gi)
+            *reinterpret_cast<float4 *>(red + ((warp * GB + gi) * 32 + lane) * 4) =
+                make_float4(acc[gi][0], acc[gi][1], acc[gi][2], acc[gi][3]);
+        asm volatile("bar.sync 1, %0;" ::"n"(NCW * 32) : "memory");
+        const int per_group = s.gsz * 8;                            // (unit, token) pairs per group
+        if (alive) {
+            for (int idx = tid; idx < ng * per_group; idx += NCW * 32) {
+                const int gi = idx / per_group, rem = idx % per_group;
+                const int rr = rem >> 3, n = rem & 7;                 // unit within group, token
+                if (rr >= s.group_size(g0 + gi) || n >= p.M) continue;
+                // rows 0..7 of the tile: regs 0,1; rows 8..15: regs 2,3
+                const int src_lane = (rr & 7) * 4 + (n >> 1), reg = n & 1;
+                const int e0 = s.swiglu ? reg : (rr >> 3) * 2 + reg;
+                float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+                for (int w = 0; w < NCW; ++w) {
+                    const float *q = red + ((w * GB + gi) * 32 + src_lane) * 4;
+                    s0 += q[e0];
+                    if (s.swiglu) s1 += q[2 + reg];
+                }
+                const float ri = normed ? red_ss[n] : 1.0f;
+                const int u = s.u_lo + s.group_lo(g0 + gi) + rr;
+                float *yp = p.y + (size_t)n * p.units + u;
+                if (s.swiglu) {
+                    const float gt = s0 * ri, up = s1 * ri;
+                    const float a = gt / (1.0f + expf(-gt)) * up;
+                    if (p.ys) store_split(p.ys, p.units >> 7, n, u, a); else __stcg(yp, a);
+                } else if (p.epi == EPI_ADD) {
+                    const float v = __ldcg(yp) + s0 * ri;
+                    __stcg(yp, v);
+                    if (p.ys) store_split(p.ys, p.units >> 7, n, u, p.next_gain ? v * __ldg(p.next_gain + u) : v);
+                    // leave v^2 where this thread alone read its first partial: the token thread adds them up below
+                    red[((0 * GB + gi) * 32 + src_lane) * 4 + e0] = v * v;
+                } else {
+                    __stcg(yp, s0 * ri);
+                }
+            }
+        }
+        if (p.ss_out) {
+            asm volatile("bar.sync 1, %0;" ::"n"(NCW * 32) : "memory");
+            if (alive && tid < p.M) {
+                const int n = tid;
+                for (int gi = 0; gi < ng; ++gi) {
+                    const int gs = s.group_size(g0 + gi);
+                    for (int rr = 0; rr < gs; ++rr)
+                        ss_acc += red[((0 * GB + gi) * 32 + (rr & 7) * 4 + (n >> 1)) * 4 + (rr >> 3) * 2 + (n & 1)];
+                }
+            }
+        }
+        asm volatile("bar.sync 1, %0;" ::"n"(NCW * 32) : "memory");
+    }
+    if (p.ss_out && alive && tid < p.M) __stcg(p.ss_out + (size_t)tid * n_cta + cta, ss_acc);
+}
+
+}  // namespace stream
+}  // namespace knnssd

@@ -61,7 +61,23 @@ struct LinPhase {
     float *y;           // [M][units]
     int epi;
     int M;              // 1..8
+    // Pre-split form (persistent pass kernel): the producer of an activation writes it already split into the three
+    // bf16 terms, in the order the tensor-core operand wants, so the consuming map only loads fragments.
+    const uint32_t *xs;      // input  [M][K/128][3 terms][4][16] words (see split_index); nullptr = read x / gain
+    const float *ss_in;      // [M][n_cta] partial sums of squares of the input rows (maps behind an RMSNorm); or nullptr
+    uint32_t *ys;            // output in the same form for the next map (EPI_ADD: y * next_gain, SWIGLU: y); or nullptr
+    const float *next_gain;  // [units] RMSNorm gain of the next map that reads y (EPI_ADD); nullptr = none
+    float *ss_out;           // [M][n_cta] this CTA's partial sum of squares of each y row (EPI_ADD); or nullptr
 };
+
+// Word index of term 0 of column `col` of row m in a pre-split buffer with nslots = K / 128 column slots; the terms
+// of one value sit 64 words apart.  Inside a slot the words are ordered (lane group t4, k-step j, half h) so that the
+// 16 words a lane needs for one term of one slot are contiguous: word 2j + h of group t4 packs columns
+// (16j + 8h + 2t4, 16j + 8h + 2t4 + 1) of the slot - the pair an m16n8k16 "col" operand register holds.
+__host__ __device__ __forceinline__ size_t split_index(int nslots, int m, int col) {
+    const int s = col >> 7, within = col & 127, j = within >> 4, r = within & 15, h = r >> 3, t4 = (r & 7) >> 1;
+    return ((((size_t)m * nslots + s) * 3) * 4 + t4) * 16 + 2 * j + h;
+}
 
 // Shared-memory ring and its barriers, carved out of the CTA's dynamic shared memory.
 struct Ring {
@@ -129,6 +145,16 @@ __device__ __forceinline__ void split3(float v, uint32_t &hi, uint32_t &mid, uin
     mid = float_to_bf16_rne(r1);
     const float r2 = r1 - __uint_as_float(mid << 16);
     lo = float_to_bf16_rne(r2);
+}
+
+// Write one activation value in pre-split form.
+__device__ __forceinline__ void store_split(uint32_t *buf, int nslots, int m, int col, float v) {
+    uint32_t hi, mid, lo;
+    split3(v, hi, mid, lo);
+    bf16_t *b = reinterpret_cast<bf16_t *>(buf) + 2 * split_index(nslots, m, col) + (col & 1);
+    __stcg(b, (bf16_t)hi);
+    __stcg(b + 128, (bf16_t)mid);
+    __stcg(b + 256, (bf16_t)lo);
 }
 
 // The CTA's share of a linear map: units [u_lo, u_lo + n_units) in n_groups groups whose sizes differ by at

@@ -14,7 +14,7 @@
 // Every wait is bounded.  A barrier or ring wait that gives up raises a device-wide abort word; every CTA then
 // falls through the rest of the list without waiting or touching memory, and the host reports a timeout.
 #pragma once
-#include "linear_stream.cuh"
+#include "linear_presplit.cuh"
 
 namespace knnssd {
 namespace pass {
@@ -34,7 +34,7 @@ struct Op {
     int barrier_after;   // 1: all CTAs meet before the next operation starts
     int is_head;         // OP_LINEAR: the LM head (runs on rows head_row0.. only)
     int layer;
-    LinPhase lin;        // OP_LINEAR
+    LinPhase lin;        // OP_LINEAR; OP_EMBED and OP_ATTN use its ys / next_gain / ss_out fields for their output
     bf16_t *kc, *vc;     // OP_ATTN: this layer's cache [n_kv_heads][max_seq][head_dim]
 };
 
@@ -45,7 +45,7 @@ struct Model {           // what does not change from pass to pass
     int d_model, H, Hkv, hd, vocab, max_seq, n_seg_max;
     const double *inv_freq;    // [hd/2]
     float *x, *qkv, *attn, *logits, *hfinal;
-    float2 *rope_cs;           // [MAXM][hd/2]
+    float2 *rope_cs;           // [grid][MAXM][hd/2]: one copy per CTA, written and read by that CTA only
     float *part_o;             // [MAXM][H][n_seg_max][hd]
     float2 *part_ml;           // [MAXM][H][n_seg_max]
     int *attn_cnt;             // [MAXM][H], zero between passes
@@ -86,9 +86,9 @@ __device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long
 
 // Called by all 256 consumer threads.  Returns false once the pass has been aborted.
 __device__ __forceinline__ bool grid_barrier(const Model &md, const Ring &r, unsigned long long target, int tid, bool alive) {
-    __threadfence();
     asm volatile("bar.sync 1, %0;" ::"n"(NCW * 32) : "memory");
     if (tid == 0 && alive) {
+        __threadfence();                       // cumulative: covers the writes of the CTA's other threads ordered by the bar.sync
         atomicAdd(md.bar, 1ULL);
         unsigned spins = 0;
         while (ld_acquire_u64(md.bar) < target) {
@@ -108,22 +108,40 @@ __device__ __forceinline__ bool grid_barrier(const Model &md, const Ring &r, uns
 }
 
 // ---- embedding gather + rotary table ----------------------------------------------------------------------
-__device__ __forceinline__ void embed_phase(const Model &md, const Params &pr, int cta, int tid) {
+__device__ __forceinline__ void embed_phase(const Model &md, const Op &op, const Params &pr, const Ring &r, int cta, int n_cta,
+                                            int tid) {
     const int d = md.d_model, half = md.hd >> 1;
-    if (cta < pr.M) {
-        const int m = cta;
-        const bf16_t *row = md.tok_embed + (size_t)pr.tok[m] * d;
-        for (int i = tid; i < d; i += NCW * 32) __stcg(md.x + (size_t)m * d + i, bf16_bits_to_float(row[i]));
-    }
-    if (cta == (pr.M < (int)gridDim.x ? pr.M : 0)) {       // one more CTA fills the (cos, sin) table of all rows
+    {   // every CTA fills its own copy of the (cos, sin) table of all rows: 148 readers of one copy would queue up at L2
         const int p0 = md.state->len + pr.pos_off;
+        float2 *mine = md.rope_cs + (size_t)cta * MAXM * half;
         for (int idx = tid; idx < pr.M * half; idx += NCW * 32) {
             const int m = idx / half, i = idx % half;
             double s, c;
             sincos((double)(p0 + m) * md.inv_freq[i], &s, &c);
-            __stcg(md.rope_cs + idx, make_float2((float)c, (float)s));
+            mine[idx] = make_float2((float)c, (float)s);
         }
     }
+    if (cta >= pr.M) return;                               // whole CTAs only: the named barrier below is CTA-local
+    // row m = cta: residual stream in fp32, its pre-split form times the first RMSNorm's gain, its sum of squares
+    const int m = cta, lane = tid & 31, warp = tid >> 5;
+    const bf16_t *row = md.tok_embed + (size_t)pr.tok[m] * d;
+    float ss = 0.f;
+    for (int i = tid; i < d; i += NCW * 32) {
+        const float v = bf16_bits_to_float(row[i]);
+        __stcg(md.x + (size_t)m * d + i, v);
+        stream::store_split(op.lin.ys, d >> 7, m, i, op.lin.next_gain ? v * __ldg(op.lin.next_gain + i) : v);
+        ss = fmaf(v, v, ss);
+    }
+    ss = warp_sum(ss);
+    if (lane == 0) r.red_ss[32 + warp] = ss;
+    asm volatile("bar.sync 1, %0;" ::"n"(NCW * 32) : "memory");
+    if (tid == 0) {
+        float tot = 0.f;
+        for (int w = 0; w < NCW; ++w) tot += r.red_ss[32 + w];
+        __stcg(op.lin.ss_out + (size_t)m * n_cta, tot);
+    }
+    for (int c = 1 + tid; c < n_cta; c += NCW * 32) __stcg(op.lin.ss_out + (size_t)m * n_cta + c, 0.f);
+    asm volatile("bar.sync 1, %0;" ::"n"(NCW * 32) : "memory");
 }
 
 // ---- RMSNorm of the rows written out (hidden-state output) -------------------------------------------------
@@ -198,14 +216,12 @@ __device__ __forceinline__ void argmax_phase(const Model &md, const Params &pr, 
 
 // ---- attention over the KV cache ------------------------------------------------------------------------------
 // Rows m = 0..M-1 sit at positions P0 + m; row m attends to positions [0, P0 + m].  The context is cut at fixed
-// absolute boundaries into segments of SEGP positions; one warp handles one (query head, segment) for all rows:
-// it reads each K and V row of the segment once (8 bytes per lane, a whole 256-byte row per warp access), in
-// register batches of 16 positions with the next batch always in flight, takes the 16 dot products of a batch with
-// a transposed butterfly, keeps an online softmax per row over 32-position chunks and writes an un-normalised
-// partial (max, sum, o).  The warp that completes the last segment of a (row, head) merges the partials in segment
-// order.  K/V of the M new positions come from the projection buffer (rotated, rounded to bf16 exactly as they are
-// stored); the warp of the first query head of each KV group also writes them to the cache.  Loops over batches stay
-// rolled on purpose: the unrolled form of this code does not fit the instruction cache.
+// absolute boundaries into segments of SEGP positions; one warp handles one (query head, segment) for all rows: it
+// reads each K and V row of the segment once, keeps the segment's scores in registers, takes a plain softmax over
+// the segment and writes an un-normalised partial (max, sum, o).  The warp that completes the last segment of a
+// (row, head) merges the partials in segment order and writes the result pre-split for the output projection.
+// K/V of the M new positions come from the projection buffer (rotated, rounded to bf16 exactly as they are stored,
+// staged in shared memory); the warp of the first query head of each KV group also writes them to the cache.
 template <int HD> struct KVVec;
 template <> struct KVVec<128> { typedef uint2 T; };
 template <> struct KVVec<64> { typedef uint32_t T; };
@@ -230,206 +246,286 @@ template <int HD> __device__ __forceinline__ typename KVVec<HD>::T kv_zero();
 template <> __device__ __forceinline__ uint2 kv_zero<128>() { return make_uint2(0u, 0u); }
 template <> __device__ __forceinline__ uint32_t kv_zero<64>() { return 0u; }
 
-// Sum over lanes of v[i], delivered to every lane whose (lane & 15) == i (i = 0..15): 16 shuffles for 16 sums.
-__device__ __forceinline__ float transposed_sum16(float (&v)[16], int lane) {
-#pragma unroll
-    for (int step = 8; step >= 1; step >>= 1) {
-        const bool up = (lane & step) != 0;
-#pragma unroll
-        for (int i = 0; i < step; ++i) {
-            const float send = up ? v[i] : v[i + step];
-            const float keep = up ? v[i + step] : v[i];
-            v[i] = keep + __shfl_xor_sync(0xffffffffu, send, step);
-        }
-    }
-    return v[0] + __shfl_xor_sync(0xffffffffu, v[0], 16);
+__device__ __forceinline__ void mma_tf32(float (&c)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
+    // rows 8..15 of the 16-row operand are not used: their registers are zero
+    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void mma_bf16_top(float (&c)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
 }
 
-constexpr int ATT_B = 16;          // positions per register batch (one batch is always in flight ahead of the math)
+#ifndef KNNSSD_ATT_STAMP
+#define KNNSSD_ATT_STAMP(i)
+#endif
 
-// MR = rows the code is unrolled for (1: draft steps, 8: verification); rows >= M are skipped at run time.
-template <int HD, int MR>
+// Tensor-core form.  Lane (g8, t4) = (lane / 4, lane % 4).  The pass's rows are the rows 0..7 of the 16-row MMA
+// operand (row m = g8), so the cost does not depend on how many rows the pass carries.
+//   scores  S = Q K^T   m16n8k16 bf16: the 8 columns of a tile are 8 consecutive positions (column n = g8 of the K
+//           operand = position 8*nt + g8).  A dot product does not care in which order its terms are taken, so k-step
+//           s pairs k-indices with the dimensions (DL*t4 + 4s .. + 3): every lane then reads one contiguous run of
+//           DL = HD/4 dimensions of "its" K row (16-byte loads) and holds the same run of q, split into three bf16
+//           terms so that the products are exact.
+//   output  O += P V    m16n8k8 tf32: k-index t4 / t4 + 4 stands for positions 2*t4 / 2*t4 + 1 of the tile - exactly
+//           the two scores the lane already holds - and column n = g8 of V-tile j is dimension (HD/8)*g8 + j, so a lane
+//           reads HD/8 contiguous dimensions of two V rows.  bf16 values are exact tf32 values; p is split into two
+//           tf32 terms (22 bits).
+// A lane ends up with output dimensions [DL*t4, DL*t4 + DL) of row g8, the run it holds of q.
+template <int HD>
 __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const Params &pr, const Ring &r, int cta, int n_cta,
                                            int warp, int lane) {
-    constexpr int DPL = HD / 32, HALF = HD / 2;
-    typedef typename KVVec<HD>::T VT;
+    constexpr int DL = HD / 4;         // dimensions of q / o per lane
+    constexpr int NW = HD / 8;         // 32-bit words of a K row per lane
+    constexpr int KS = HD / 16;        // k-steps of Q K^T
+    constexpr int VW = HD / 16;        // 32-bit words of a V row per lane
+    constexpr int VJ = HD / 8;         // V tiles (8 dimensions each)
+    constexpr int HALF = HD / 2, DPL = HD / 32;
+    constexpr int NT = SEGP / 8;       // position tiles per segment
+    const int g8 = lane >> 2, t4 = lane & 3;
     const int M = pr.M, H = md.H, Hkv = md.Hkv, G = H / Hkv;
     const int P0 = md.state->len + pr.pos_off, Ttot = P0 + M;
     const int n_seg = (Ttot + SEGP - 1) / SEGP, n_tasks = H * n_seg;
     const int qstride = (H + 2 * Hkv) * HD;
     const float scale = 1.0f / sqrtf((float)HD);
-    const int d0 = DPL * lane, ci = d0 % HALF;
-    const bool upper = d0 >= HALF;
+    const bool upper = t4 >= 2;                              // this lane's run lies in the second half of the head
+    const int ci = DL * (t4 & 1);                            // its offset in the (cos, sin) table
     bf16_t *stash_k = reinterpret_cast<bf16_t *>(r.red) + (size_t)warp * (2 * MAXM * HD);   // [MAXM][HD] new K rows
     bf16_t *stash_v = stash_k + MAXM * HD;                                                  // [MAXM][HD] new V rows
+    const float2 *my_cs = md.rope_cs + (size_t)cta * MAXM * HALF;                           // this CTA's copy
 
     for (int t = warp * n_cta + cta; t < n_tasks; t += NCW * n_cta) {
         const int seg = t / H, h = t % H, kvh = h / G;
         const int p_begin = seg * SEGP, p_end = min(p_begin + SEGP, Ttot);
-        const int m_first = max(0, p_begin - P0);
+        const int m_first = max(0, p_begin - P0);           // first row that sees this segment
         const bool writer = (h % G) == 0;
         bf16_t *kbase = op.kc + (size_t)kvh * md.max_seq * HD;
         bf16_t *vbase = op.vc + (size_t)kvh * md.max_seq * HD;
+        const bool row_new = g8 < M && P0 + g8 >= p_begin && P0 + g8 < p_end;   // row g8's own position lies in this segment
+        const bool row_live = g8 < M && g8 >= m_first;
 
-        // new K/V rows that fall into this segment: rotate, round, stash (and store if this warp is the writer)
-        __syncwarp();
-        for (int mp = m_first; mp < M && P0 + mp < p_end; ++mp) {
-            const float *kraw = md.qkv + (size_t)mp * qstride + (size_t)(H + kvh) * HD + d0;
-            const float *vraw = md.qkv + (size_t)mp * qstride + (size_t)(H + Hkv + kvh) * HD + d0;
-            float kf[DPL], vf[DPL];
+        KNNSSD_ATT_STAMP(0);
+        // ---- this lane's run of q (row g8), of the new K row and of the new V row: load, rotate, round / split ----
+        float qf[DL], kf[DL];
+        {
+            const float *qraw = md.qkv + (size_t)min(g8, M - 1) * qstride + (size_t)h * HD + DL * t4;
+            const float *kraw = md.qkv + (size_t)min(g8, M - 1) * qstride + (size_t)(H + kvh) * HD + DL * t4;
 #pragma unroll
-            for (int e = 0; e < DPL; ++e) { kf[e] = __ldcg(kraw + e); vf[e] = __ldcg(vraw + e); }
-#pragma unroll
-            for (int e = 0; e < DPL; ++e) {
-                const float partner = __shfl_xor_sync(0xffffffffu, kf[e], 16);
-                const float2 cs = __ldcg(md.rope_cs + mp * HALF + ci + e);
-                kf[e] = upper ? (kf[e] * cs.x + partner * cs.y) : (kf[e] * cs.x - partner * cs.y);
+            for (int e = 0; e < DL; e += 4) {
+                const float4 a = row_live ? __ldcg(reinterpret_cast<const float4 *>(qraw + e)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                const float4 b = row_new ? __ldcg(reinterpret_cast<const float4 *>(kraw + e)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                qf[e] = a.x; qf[e + 1] = a.y; qf[e + 2] = a.z; qf[e + 3] = a.w;
+                kf[e] = b.x; kf[e + 1] = b.y; kf[e + 2] = b.z; kf[e + 3] = b.w;
             }
-            const VT kp = kv_pack<HD>(kf), vp = kv_pack<HD>(vf);
-            *reinterpret_cast<VT *>(stash_k + mp * HD + d0) = kp;
-            *reinterpret_cast<VT *>(stash_v + mp * HD + d0) = vp;
-            if (writer) {
-                *reinterpret_cast<VT *>(kbase + (size_t)(P0 + mp) * HD + d0) = kp;
-                *reinterpret_cast<VT *>(vbase + (size_t)(P0 + mp) * HD + d0) = vp;
+#pragma unroll
+            for (int e = 0; e < DL; ++e) {
+                const float qp = __shfl_xor_sync(0xffffffffu, qf[e], 2), kp = __shfl_xor_sync(0xffffffffu, kf[e], 2);
+                const float2 cs = (row_live || row_new) ? my_cs[g8 * HALF + ci + e] : make_float2(1.f, 0.f);
+                qf[e] = upper ? (qf[e] * cs.x + qp * cs.y) : (qf[e] * cs.x - qp * cs.y);
+                kf[e] = upper ? (kf[e] * cs.x + kp * cs.y) : (kf[e] * cs.x - kp * cs.y);
             }
         }
         __syncwarp();
-
-        // rotated queries of the rows that see this segment
-        float q[MR][DPL], o[MR][DPL], mx[MR], l[MR], sreg[MR];
+        if (row_new) {
+            const float *vraw = md.qkv + (size_t)g8 * qstride + (size_t)(H + Hkv + kvh) * HD + DL * t4;
 #pragma unroll
-        for (int m = 0; m < MR; ++m) {
-            mx[m] = -INFINITY; l[m] = 0.f; sreg[m] = 0.f;
-#pragma unroll
-            for (int e = 0; e < DPL; ++e) { q[m][e] = 0.f; o[m][e] = 0.f; }
-            if (m >= m_first && m < M) {
-                const float *qraw = md.qkv + (size_t)m * qstride + (size_t)h * HD + d0;
-#pragma unroll
-                for (int e = 0; e < DPL; ++e) q[m][e] = __ldcg(qraw + e);
-#pragma unroll
-                for (int e = 0; e < DPL; ++e) {
-                    const float partner = __shfl_xor_sync(0xffffffffu, q[m][e], 16);
-                    const float2 cs = __ldcg(md.rope_cs + m * HALF + ci + e);
-                    q[m][e] = upper ? (q[m][e] * cs.x + partner * cs.y) : (q[m][e] * cs.x - partner * cs.y);
+            for (int e = 0; e < DL; e += 8) {
+                const float4 a = __ldcg(reinterpret_cast<const float4 *>(vraw + e)), b = __ldcg(reinterpret_cast<const float4 *>(vraw + e + 4));
+                uint4 kp, vp;
+                kp.x = (uint32_t)float_to_bf16_rne(kf[e]) | ((uint32_t)float_to_bf16_rne(kf[e + 1]) << 16);
+                kp.y = (uint32_t)float_to_bf16_rne(kf[e + 2]) | ((uint32_t)float_to_bf16_rne(kf[e + 3]) << 16);
+                kp.z = (uint32_t)float_to_bf16_rne(kf[e + 4]) | ((uint32_t)float_to_bf16_rne(kf[e + 5]) << 16);
+                kp.w = (uint32_t)float_to_bf16_rne(kf[e + 6]) | ((uint32_t)float_to_bf16_rne(kf[e + 7]) << 16);
+                vp.x = (uint32_t)float_to_bf16_rne(a.x) | ((uint32_t)float_to_bf16_rne(a.y) << 16);
+                vp.y = (uint32_t)float_to_bf16_rne(a.z) | ((uint32_t)float_to_bf16_rne(a.w) << 16);
+                vp.z = (uint32_t)float_to_bf16_rne(b.x) | ((uint32_t)float_to_bf16_rne(b.y) << 16);
+                vp.w = (uint32_t)float_to_bf16_rne(b.z) | ((uint32_t)float_to_bf16_rne(b.w) << 16);
+                *reinterpret_cast<uint4 *>(stash_k + g8 * HD + DL * t4 + e) = kp;
+                *reinterpret_cast<uint4 *>(stash_v + g8 * HD + DL * t4 + e) = vp;
+                if (writer) {
+                    *reinterpret_cast<uint4 *>(kbase + (size_t)(P0 + g8) * HD + DL * t4 + e) = kp;
+                    *reinterpret_cast<uint4 *>(vbase + (size_t)(P0 + g8) * HD + DL * t4 + e) = vp;
                 }
             }
         }
-
-        // The segment as a flat list of register batches: per 32-position chunk, K rows 0-15, K rows 16-31, V rows
-        // 0-15, V rows 16-31.  Batch it + 1 is loading while batch it is being used.
-        auto load_batch = [&](int it, VT (&dst)[ATT_B]) {
-            const int sub = it & 3, pb = p_begin + (it >> 2) * 32 + (sub & 1) * ATT_B;
-            const bf16_t *cache = (sub >> 1) ? vbase : kbase;
-            const bf16_t *stash = (sub >> 1) ? stash_v : stash_k;
+        __syncwarp();
+        uint32_t qh[NW], qm[NW], ql[NW];                     // word w = dimensions (2w, 2w + 1) of the run
 #pragma unroll
-            for (int j = 0; j < ATT_B; ++j) {
-                const int p = pb + j;
-                const bf16_t *src = p < P0 ? cache + (size_t)p * HD + d0 : stash + (p - P0) * HD + d0;
-                dst[j] = p < p_end ? *reinterpret_cast<const VT *>(src) : kv_zero<HD>();
+        for (int w = 0; w < NW; ++w) {
+            uint32_t h0, m0, l0, h1, m1, l1;
+            stream::split3(qf[2 * w], h0, m0, l0);
+            stream::split3(qf[2 * w + 1], h1, m1, l1);
+            qh[w] = h0 | (h1 << 16); qm[w] = m0 | (m1 << 16); ql[w] = l0 | (l1 << 16);
+        }
+
+        KNNSSD_ATT_STAMP(1);
+        // ---- scores: one tile = 8 positions; K rows are fetched two tiles ahead ----
+        auto load_k = [&](int nt, uint4 (&dst)[NW / 4]) {
+            const int p = p_begin + 8 * nt + g8;
+            const bf16_t *src = p < P0 ? kbase + (size_t)p * HD + DL * t4 : stash_k + (p - P0) * HD + DL * t4;
+#pragma unroll
+            for (int q = 0; q < NW / 4; ++q)
+                dst[q] = p < p_end ? *reinterpret_cast<const uint4 *>(src + 8 * q) : make_uint4(0u, 0u, 0u, 0u);
+        };
+        float sc[NT][2];                                     // scores of (row g8, positions 8*nt + 2*t4 + {0, 1})
+        {
+            constexpr int KR = NT < 4 ? NT : 4;              // tiles in flight
+            uint4 kb[KR][NW / 4];
+#pragma unroll
+            for (int i = 0; i < KR; ++i) load_k(i, kb[i]);
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                uint4(&kq)[NW / 4] = kb[nt % KR];
+                float ch[4] = {}, cm[4] = {}, cl[4] = {};
+#pragma unroll
+                for (int q = 0; q < NW / 4; ++q) {
+                    // words 4q .. 4q+3 of the run: k-steps 2q (x, y) and 2q + 1 (z, w)
+                    mma_bf16_top(cl, ql[4 * q], ql[4 * q + 1], kq[q].x, kq[q].y);
+                    mma_bf16_top(cm, qm[4 * q], qm[4 * q + 1], kq[q].x, kq[q].y);
+                    mma_bf16_top(ch, qh[4 * q], qh[4 * q + 1], kq[q].x, kq[q].y);
+                    mma_bf16_top(cl, ql[4 * q + 2], ql[4 * q + 3], kq[q].z, kq[q].w);
+                    mma_bf16_top(cm, qm[4 * q + 2], qm[4 * q + 3], kq[q].z, kq[q].w);
+                    mma_bf16_top(ch, qh[4 * q + 2], qh[4 * q + 3], kq[q].z, kq[q].w);
+                }
+                sc[nt][0] = (cl[0] + cm[0]) + ch[0];
+                sc[nt][1] = (cl[1] + cm[1]) + ch[1];
+                if (nt + KR < NT) load_k(nt + KR, kq);
+            }
+        }
+        KNNSSD_ATT_STAMP(2);
+        // ---- V rows of the first tiles start moving while the softmax runs ----
+        auto load_v = [&](int nt, uint4 (&dst)[2][(VW + 3) / 4]) {
+#pragma unroll
+            for (int rr = 0; rr < 2; ++rr) {
+                const int p = p_begin + 8 * nt + 2 * t4 + rr;
+                const bf16_t *src = p < P0 ? vbase + (size_t)p * HD + 2 * VW * g8 : stash_v + (p - P0) * HD + 2 * VW * g8;
+                if (VW >= 4) {
+#pragma unroll
+                    for (int q = 0; q < VW / 4; ++q)
+                        dst[rr][q] = p < p_end ? *reinterpret_cast<const uint4 *>(src + 8 * q) : make_uint4(0u, 0u, 0u, 0u);
+                } else {
+                    const uint2 v = p < p_end ? *reinterpret_cast<const uint2 *>(src) : make_uint2(0u, 0u);
+                    dst[rr][0] = make_uint4(v.x, v.y, 0u, 0u);
+                }
             }
         };
-        const int n_it = 4 * ((p_end - p_begin + 31) >> 5);
-        VT cur[ATT_B], nxt[ATT_B];
-        load_batch(0, cur);
-        for (int it = 0; it < n_it; ++it) {
-            if (it + 1 < n_it) load_batch(it + 1, nxt);
-            const int sub = it & 3, half = sub & 1, p0 = p_begin + (it >> 2) * 32;
-            if (sub < 2) {
-                // ---- scores of 16 positions: lane (half * 16 + i) keeps position i's score ----
+        constexpr int VR = NT < 4 ? NT : 4;                  // tiles in flight
+        uint4 vb[VR][2][(VW + 3) / 4];
 #pragma unroll
-                for (int m = 0; m < MR; ++m) {
-                    if (m < m_first || m >= M || p0 > P0 + m) continue;      // row does not see this chunk
-                    float part[ATT_B];
+        for (int i = 0; i < VR; ++i) load_v(i, vb[i]);
+
+        KNNSSD_ATT_STAMP(3);
+        // ---- softmax over the segment for row g8 (the four lanes of a row share it) ----
+        float mx = -INFINITY;
 #pragma unroll
-                    for (int j = 0; j < ATT_B; ++j) {
-                        float kf[DPL];
-                        kv_unpack<HD>(cur[j], kf);
-                        float s = 0.f;
+        for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-                        for (int e = 0; e < DPL; ++e) s = fmaf(q[m][e], kf[e], s);
-                        part[j] = s;
-                    }
-                    const float tot = transposed_sum16(part, lane);
-                    if ((lane >> 4) == half) sreg[m] = tot;
-                }
-                if (sub == 1) {
-                    // ---- online softmax over the chunk's 32 positions (lane = position) ----
-#pragma unroll
-                    for (int m = 0; m < MR; ++m) {
-                        if (m < m_first || m >= M || p0 > P0 + m) continue;
-                        const bool valid = p0 + lane <= P0 + m;
-                        const float s = valid ? sreg[m] * scale : -INFINITY;
-                        const float mnew = fmaxf(mx[m], warp_max(s));
-                        const float corr = expf(mx[m] - mnew);
-                        const float pj = valid ? expf(s - mnew) : 0.f;
-                        l[m] = fmaf(l[m], corr, warp_sum(pj));
-#pragma unroll
-                        for (int e = 0; e < DPL; ++e) o[m][e] *= corr;
-                        mx[m] = mnew;
-                        sreg[m] = pj;
-                    }
-                }
-            } else {
-                // ---- o += p V over 16 positions ----
-#pragma unroll
-                for (int j = 0; j < ATT_B; ++j) {
-                    float vf[DPL];
-                    kv_unpack<HD>(cur[j], vf);
-#pragma unroll
-                    for (int m = 0; m < MR; ++m) {
-                        if (m < m_first || m >= M || p0 > P0 + m) continue;
-                        const float pj = __shfl_sync(0xffffffffu, sreg[m], half * ATT_B + j);
-#pragma unroll
-                        for (int e = 0; e < DPL; ++e) o[m][e] = fmaf(pj, vf[e], o[m][e]);
-                    }
-                }
+            for (int e = 0; e < 2; ++e) {
+                const int p = p_begin + 8 * nt + 2 * t4 + e;
+                const bool valid = row_live && p <= P0 + g8;             // causal; also excludes p >= p_end
+                sc[nt][e] = valid ? sc[nt][e] * scale : -INFINITY;
+                mx = fmaxf(mx, sc[nt][e]);
             }
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+        float lsum = 0.f;
 #pragma unroll
-            for (int j = 0; j < ATT_B; ++j) cur[j] = nxt[j];
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const float pj = sc[nt][e] == -INFINITY ? 0.f : expf(sc[nt][e] - mx);
+                sc[nt][e] = pj;
+                lsum += pj;
+            }
+        lsum += __shfl_xor_sync(0xffffffffu, lsum, 1);
+        lsum += __shfl_xor_sync(0xffffffffu, lsum, 2);
+
+        KNNSSD_ATT_STAMP(4);
+        // ---- o += p V ----
+        float o[VJ][4];
+#pragma unroll
+        for (int j = 0; j < VJ; ++j) { o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f; }
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            const uint32_t p0h = __float_as_uint(sc[nt][0]) & 0xFFFFE000u, p1h = __float_as_uint(sc[nt][1]) & 0xFFFFE000u;
+            const uint32_t p0l = __float_as_uint(sc[nt][0] - __uint_as_float(p0h)) & 0xFFFFE000u;
+            const uint32_t p1l = __float_as_uint(sc[nt][1] - __uint_as_float(p1h)) & 0xFFFFE000u;
+#pragma unroll
+            for (int j = 0; j < VJ; ++j) {
+                const uint4 &wa = vb[nt % VR][0][j / 8], &wb = vb[nt % VR][1][j / 8];
+                const int wi = (j >> 1) & 3;
+                const uint32_t xa = wi == 0 ? wa.x : wi == 1 ? wa.y : wi == 2 ? wa.z : wa.w;
+                const uint32_t xb = wi == 0 ? wb.x : wi == 1 ? wb.y : wi == 2 ? wb.z : wb.w;
+                const uint32_t b0 = (j & 1) ? (xa & 0xFFFF0000u) : (xa << 16);
+                const uint32_t b1 = (j & 1) ? (xb & 0xFFFF0000u) : (xb << 16);
+                mma_tf32(o[j], p0l, p1l, b0, b1);
+                mma_tf32(o[j], p0h, p1h, b0, b1);
+            }
+            if (nt + VR < NT) load_v(nt + VR, vb[nt % VR]);
         }
 
-        // ---- partials out; the last warp of a (row, head) merges ----
+        KNNSSD_ATT_STAMP(5);
+        // ---- partials out (row g8: dimensions DL*t4 + j and DL*t4 + VJ + j); the last warp of a (row, head) merges ----
+        if (row_live) {
+            const size_t pidx = ((size_t)g8 * H + h) * md.n_seg_max + seg;
+            if (t4 == 0) __stcg(md.part_ml + pidx, make_float2(mx, lsum));
+            float *po = md.part_o + pidx * HD + DL * t4;
 #pragma unroll
-        for (int m = 0; m < MR; ++m) {
-            if (m < m_first || m >= M) continue;
-            const size_t pidx = ((size_t)m * H + h) * md.n_seg_max + seg;
-            if (lane == 0) __stcg(md.part_ml + pidx, make_float2(mx[m], l[m]));
-#pragma unroll
-            for (int e = 0; e < DPL; ++e) __stcg(md.part_o + pidx * HD + d0 + e, o[m][e]);
+            for (int j = 0; j < VJ; j += 4) {
+                __stcg(reinterpret_cast<float4 *>(po + j), make_float4(o[j][0], o[j + 1][0], o[j + 2][0], o[j + 3][0]));
+                __stcg(reinterpret_cast<float4 *>(po + VJ + j), make_float4(o[j][1], o[j + 1][1], o[j + 2][1], o[j + 3][1]));
+            }
         }
         __threadfence();
         __syncwarp();
-        unsigned last_mask = 0;
-        if (lane == 0) {
-            for (int m = m_first; m < M; ++m) {
-                const int n_seg_m = (P0 + m + SEGP) / SEGP;              // segments row m sees
-                if (atomicAdd(md.attn_cnt + m * H + h, 1) == n_seg_m - 1) last_mask |= 1u << m;
-            }
+        KNNSSD_ATT_STAMP(6);
+        bool last = false;
+        if (row_live && t4 == 0) {
+            const int n_seg_m = (P0 + g8 + SEGP) / SEGP;                  // segments row g8 sees
+            last = atomicAdd(md.attn_cnt + g8 * H + h, 1) == n_seg_m - 1;
         }
-        last_mask = __shfl_sync(0xffffffffu, last_mask, 0);
+        KNNSSD_ATT_STAMP(7);
+        const unsigned last_mask = __ballot_sync(0xffffffffu, last);     // bit 4*m set: this warp finishes (row m, head h)
         if (last_mask) {
             __threadfence();
+            const int d0 = DPL * lane;
             for (int m = m_first; m < M; ++m) {
-                if (!((last_mask >> m) & 1u)) continue;
+                if (!((last_mask >> (4 * m)) & 1u)) continue;
                 const int n_seg_m = (P0 + m + SEGP) / SEGP;
                 const size_t base = ((size_t)m * H + h) * md.n_seg_max;
-                float gm = -INFINITY;
-                for (int s = 0; s < n_seg_m; ++s) gm = fmaxf(gm, __ldcg(md.part_ml + base + s).x);
-                float L = 0.f, acc[DPL];
+                // segment statistics: lane s holds segments s and s + 32 (contexts up to 4096); fixed-order warp reductions
+                const float2 ml0 = lane < n_seg_m ? __ldcg(md.part_ml + base + lane) : make_float2(-INFINITY, 0.f);
+                const float2 ml1 = lane + 32 < n_seg_m ? __ldcg(md.part_ml + base + lane + 32) : make_float2(-INFINITY, 0.f);
+                const float gm = warp_max(fmaxf(ml0.x, ml1.x));
+                const float w0 = ml0.x == -INFINITY ? 0.f : expf(ml0.x - gm), w1 = ml1.x == -INFINITY ? 0.f : expf(ml1.x - gm);
+                const float L = warp_sum(fmaf(ml1.y, w1, ml0.y * w0));
+                // weighted sum of the partial outputs in segment order, sixteen segments in flight at a time
+                float acc[DPL];
 #pragma unroll
                 for (int e = 0; e < DPL; ++e) acc[e] = 0.f;
-                for (int s = 0; s < n_seg_m; ++s) {
-                    const float2 ml = __ldcg(md.part_ml + base + s);
-                    const float w = expf(ml.x - gm);
-                    L = fmaf(ml.y, w, L);
+                for (int s0 = 0; s0 < n_seg_m; s0 += 16) {
+                    float pv[16][DPL];
 #pragma unroll
-                    for (int e = 0; e < DPL; ++e) acc[e] = fmaf(__ldcg(md.part_o + (base + s) * HD + d0 + e), w, acc[e]);
+                    for (int i = 0; i < 16; ++i)
+#pragma unroll
+                        for (int e = 0; e < DPL; ++e)
+                            pv[i][e] = s0 + i < n_seg_m ? __ldcg(md.part_o + (base + s0 + i) * HD + d0 + e) : 0.f;
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const int sg = s0 + i;
+                        const float w = __shfl_sync(0xffffffffu, sg < 32 ? w0 : w1, sg & 31);
+#pragma unroll
+                        for (int e = 0; e < DPL; ++e) acc[e] = fmaf(pv[i][e], w, acc[e]);
+                    }
                 }
 #pragma unroll
-                for (int e = 0; e < DPL; ++e) __stcg(md.attn + (size_t)m * H * HD + (size_t)h * HD + d0 + e, acc[e] / L);
+                for (int e = 0; e < DPL; ++e) stream::store_split(op.lin.ys, (H * HD) >> 7, m, h * HD + d0 + e, acc[e] / L);
                 if (lane == 0) md.attn_cnt[m * H + h] = 0;
             }
         }
+        KNNSSD_ATT_STAMP(8);
     }
 }
 
@@ -471,16 +567,14 @@ __global__ void __launch_bounds__(stream::NTHREADS, 1) pass_kernel(const Model m
             if (op.is_head) {
                 if (pr.head_row0 >= pr.M) ran = false;
                 lp.M = pr.M - pr.head_row0;
-                lp.x += (size_t)pr.head_row0 * lp.K;
+                lp.xs += (size_t)pr.head_row0 * (lp.K >> 7) * 192;
+                lp.ss_in += (size_t)pr.head_row0 * n_cta;
                 lp.y += (size_t)pr.head_row0 * lp.units;
             }
-            if (ran) stream::consume_linear(lp, r, cta, n_cta, warp, lane, w_use, alive);
+            if (ran) stream::consume_linear_pre(lp, r, cta, n_cta, warp, lane, w_use, alive);
         } else if (alive) {
-            if (op.type == OP_EMBED) embed_phase(md, pr, cta, tid);
-            else if (op.type == OP_ATTN) {
-                if (pr.M == 1) attn_phase<HD, 1>(md, op, pr, r, cta, n_cta, warp, lane);
-                else attn_phase<HD, MAXM>(md, op, pr, r, cta, n_cta, warp, lane);
-            }
+            if (op.type == OP_EMBED) embed_phase(md, op, pr, r, cta, n_cta, tid);
+            else if (op.type == OP_ATTN) attn_phase<HD>(md, op, pr, r, cta, n_cta, warp, lane);
             else if (op.type == OP_HIDDEN) { if (pr.want_hidden) hidden_phase(md, pr, r, cta, tid); else ran = false; }
             else if (op.type == OP_ARGMAX) { if (pr.head_row0 < pr.M) argmax_phase(md, pr, r, cta, n_cta, tid); else ran = false; }
         }
