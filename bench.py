@@ -334,7 +334,7 @@ def main():
     ap.add_argument("--workload", default="llama13b", choices=sorted(WORKLOADS))
     ap.add_argument("--k", type=int, default=4)
     ap.add_argument("--seed", type=int, default=0)
-    ap.add_argument("--gamma", type=float, default=0.05,
+    ap.add_argument("--gamma", type=float, default=0.0003,
                     help="scale of the output projections of mask-skipped sublayers (1 = plain random init)")
     ap.add_argument("--pass-iters", type=int, default=50)
     ap.add_argument("--cpu-prompt", type=int, default=16)

@@ -281,7 +281,7 @@ template <int HD> cudaError_t launch_pass_t(knnssd_ctx *c, const pass::Params &p
 
 // One pass through the persistent kernel.  Errors surface at the caller's next synchronisation.
 void run_pass_mega(knnssd_ctx *c, int M, const int *tok_dev, int pos_off, const unsigned char *mask, int head_row0,
-                   int *argmax_out, bool want_hidden) {
+                   int *argmax_out, bool want_hidden, int out_row0 = 0) {
     pass::Params pr{};
     int bars;
     if (!mask) {
@@ -298,6 +298,7 @@ void run_pass_mega(knnssd_ctx *c, int M, const int *tok_dev, int pos_off, const 
     }
     pr.M = M; pr.tok = tok_dev; pr.pos_off = pos_off; pr.head_row0 = head_row0; pr.argmax_out = argmax_out;
     pr.want_hidden = want_hidden ? 1 : 0;
+    pr.out_row0 = out_row0;
     pr.bar_base = c->bar_total;
     if (head_row0 < M) bars += 1;
     const cudaError_t e = c->cfg.head_dim == 128 ? launch_pass_t<128>(c, pr) : launch_pass_t<64>(c, pr);
@@ -381,6 +382,14 @@ void run_pass_t(knnssd_ctx *c, int M, const int *tok_dev, int pos_off, const uns
 void run_pass(knnssd_ctx *c, int M, const int *tok_dev, int pos_off, const unsigned char *mask, int head_row0,
               int *argmax_out, bool want_hidden) {
     if (c->mega_ok && M <= pass::MAXM) { run_pass_mega(c, M, tok_dev, pos_off, mask, head_row0, argmax_out, want_hidden); return; }
+    if (c->mega_ok && M <= 2 * pass::MAXM) {
+        // more rows than one launch of the persistent kernel carries: rows 0..7 first, then the rest as a second pass
+        // whose rows sit 8 positions further on (it finds the first eight rows' K/V in the cache like any earlier row)
+        const int A = pass::MAXM, hrA = head_row0 < A ? head_row0 : A, hrB = head_row0 > A ? head_row0 - A : 0;
+        run_pass_mega(c, A, tok_dev, pos_off, mask, hrA, argmax_out, want_hidden, 0);
+        run_pass_mega(c, M - A, tok_dev + A, pos_off + A, mask, hrB, argmax_out + (A + hrB - head_row0), want_hidden, A);
+        return;
+    }
     if (c->cfg.dtype) run_pass_t<bf16_t>(c, M, tok_dev, pos_off, mask, head_row0, argmax_out, want_hidden);
     else run_pass_t<float>(c, M, tok_dev, pos_off, mask, head_row0, argmax_out, want_hidden);
 }

@@ -68,6 +68,7 @@ struct Params {
     int head_row0;             // rows >= head_row0 get logits and an arg-max (== M: none)
     int *argmax_out;           // [M - head_row0]
     int want_hidden;
+    int out_row0;              // row of the logits / hidden-state buffers that this pass's row 0 goes to
     unsigned long long bar_base;   // value of *bar when this launch starts
 };
 
@@ -157,7 +158,7 @@ __device__ __forceinline__ void hidden_phase(const Model &md, const Params &pr, 
     float tot = 0.f;
     for (int w = 0; w < NCW; ++w) tot += r.red_ss[w];
     const float rinv = 1.0f / sqrtf(tot / (float)d + md.rms_eps);
-    for (int i = tid; i < d; i += NCW * 32) __stcg(md.hfinal + (size_t)m * d + i, __ldcg(xr + i) * rinv * md.final_norm[i]);
+    for (int i = tid; i < d; i += NCW * 32) __stcg(md.hfinal + (size_t)(pr.out_row0 + m) * d + i, __ldcg(xr + i) * rinv * md.final_norm[i]);
     asm volatile("bar.sync 1, %0;" ::"n"(NCW * 32) : "memory");
 }
 
@@ -170,7 +171,7 @@ __device__ __forceinline__ void argmax_phase(const Model &md, const Params &pr, 
     int *s_last = reinterpret_cast<int *>(r.red + 128);
     const int rows = pr.M - pr.head_row0;
     for (int m = 0; m < rows; ++m) {
-        const float *row = md.logits + (size_t)(pr.head_row0 + m) * V;
+        const float *row = md.logits + (size_t)(pr.out_row0 + pr.head_row0 + m) * V;
         float bv = -INFINITY;
         int bi = 0x7fffffff;
         for (int i = i0 + tid; i < i1; i += NCW * 32) argmax_fold(bv, bi, __ldcg(row + i), i);
@@ -569,7 +570,7 @@ __global__ void __launch_bounds__(stream::NTHREADS, 1) pass_kernel(const Model m
                 lp.M = pr.M - pr.head_row0;
                 lp.xs += (size_t)pr.head_row0 * (lp.K >> 7) * 192;
                 lp.ss_in += (size_t)pr.head_row0 * n_cta;
-                lp.y += (size_t)pr.head_row0 * lp.units;
+                lp.y += (size_t)(pr.out_row0 + pr.head_row0) * lp.units;
             }
             if (ran) stream::consume_linear_pre(lp, r, cta, n_cta, warp, lane, w_use, alive);
         } else if (alive) {

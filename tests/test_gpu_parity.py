@@ -190,6 +190,40 @@ def test_generate_matches_oracle_exactly(kb, shape_name, prompt_len, max_new, k)
     assert np.array_equal(plain["tokens"], got["tokens"])
 
 
+def test_full_width_13b_layers_match_oracle(kb):
+    """The widths of the LLaMA-2-13B-shaped workload (d 5120, 40 heads, FFN 13824, vocab 32000) on two layers, so that the
+    oracle finishes in seconds: the launch configuration the benchmark times (persistent pass kernel, 148 CTAs), a
+    prompt that spans several 64-position attention segments with a ragged tail, k = 4 and k = 8."""
+    shape = si.SHAPES["llama13b"].with_layers(2)
+    mask = np.array([1, 0, 0, 1], np.uint8)                    # skip attention of layer 0 and MLP of layer 1
+    damp = {0: 0.02, 3: 0.02}
+    w = si.make_model_weights(shape, 5, device="cuda", damp=damp, gain_spread=0.1)
+    wc = {k: ([t.cpu() for t in v] if isinstance(v, list) else v.cpu()) for k, v in w.items()}
+    om = oracle.OracleModel(shape, wc, 224)
+    sess = kb.Session.from_shape(shape, w, 224, max_draft=8)
+    prompt = si.uniform_tokens(7, 0, 150, shape.vocab).numpy()
+    pooled_o, first_o, _ = om.prefill(prompt)
+    first_g, pooled_g = sess.prefill(prompt, want_pooled=True)
+    assert first_g == first_o
+    assert np.abs(pooled_g.cpu().numpy() - pooled_o).max() < TOL["bf16"]
+    # teacher-forced rows: logits and hidden states of one verification pass
+    rows = si.uniform_tokens(8, 1, 4, shape.vocab).numpy()
+    o = om.forward(np.concatenate([[first_o], rows]).astype(np.int32), 150, want_hidden=True)
+    g = sess.verify(rows, want_logits=True, want_hidden=True)
+    assert np.abs(g["logits"].cpu().numpy() - o["logits"]).max() < TOL["bf16"]
+    assert np.abs(g["hidden"].cpu().numpy() - o["hidden"]).max() < TOL["bf16"]
+    assert (g["n_accepted"], g["next_token"]) == oracle.accept(rows, o["argmax"])
+    for k in (4, 8):
+        om.length = 150
+        sess.set_length(150)
+        sess.set_pending(first_o)
+        sess.set_skipmask(mask)
+        want = om.generate(first_o, 14, k, mask)
+        got = sess.decode(14, k)
+        assert np.array_equal(got["tokens"], want["tokens"]), f"k={k}: oracle min margin {want['min_margin']}"
+        assert np.array_equal(got["accepts"], want["accepts"])
+
+
 def test_config1_tiny_all_on_and_all_off_masks(kb):
     shape, om, sess = _pair(kb, "tiny", gain_spread=0.0)
     prompt = si.uniform_tokens(0, 0, 32, shape.vocab).numpy()
