@@ -151,13 +151,25 @@ def run_ours(args):
     torch.cuda.synchronize()
     t_weights = time.time() - t0
     max_seq = len(prompt) + max_new + 64
-    sess = kb.Session.from_shape(shape, w, max_seq, max_draft=max(k, 8), anchors=anchors.to(dev), skip_masks=masks,
+    # Domains are Gaussian clusters in hidden space and a request is a draw from its domain's cluster.  The request's
+    # pooled last-layer state is whatever this random-init model produces for the prompt, so the cluster of
+    # REQUEST_DOMAIN is centred there: a first session (no anchors) yields that state, then the anchors are drawn.
+    probe = kb.Session.from_shape(shape, w, max_seq, max_draft=max(k, 8))
+    _, pooled0 = probe.prefill(prompt, want_pooled=True)
+    probe.close()
+    anchors = anchors.to(dev).clone()
+    unit = pooled0 / pooled0.norm()
+    lo, hi = REQUEST_DOMAIN * PER_DOMAIN, (REQUEST_DOMAIN + 1) * PER_DOMAIN
+    noise = si.normal_f32(args.seed, si.TensorId.ANCHOR + 1000, torch.arange(PER_DOMAIN * shape.d_model, device=dev), 1.0)
+    own = unit[None, :] + 0.2 / (shape.d_model ** 0.5) * noise.view(PER_DOMAIN, shape.d_model)
+    anchors[lo:hi] = own / own.norm(dim=1, keepdim=True)
+    sess = kb.Session.from_shape(shape, w, max_seq, max_draft=max(k, 8), anchors=anchors.contiguous(), skip_masks=masks,
                                  anchors_per_domain=PER_DOMAIN)
-    # shift the request towards one domain's cluster as a labelled request of the mixed stream would be
-    cen = si.domain_centroids(args.seed, N_DOMAINS, shape.d_model).to(dev)
     first, pooled = sess.prefill(prompt, want_pooled=True)
-    query = (pooled + 4.0 * pooled.norm() / cen[REQUEST_DOMAIN].norm() * cen[REQUEST_DOMAIN]).contiguous()
+    query = pooled
     dom, anc, cos = sess.select_skipset(query)
+    if dom != REQUEST_DOMAIN:
+        raise SystemExit(f"selection picked domain {dom}, expected {REQUEST_DOMAIN}")
     mask = masks[dom]
     P = len(prompt)
 
