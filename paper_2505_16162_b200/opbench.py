@@ -1,9 +1,14 @@
-"""Per-kernel timing of the stand-alone operators, for tuning and for profiler captures.
+"""Per-kernel timing, for tuning and for profiler captures.
 
     python -m paper_2505_16162_b200.opbench linear --n-out 131072 --n-in 5120 --rows 5 --iters 20
 
 times ``knnssd_linear`` on seeded bf16 weights with CUDA events and prints GB/s (weight bytes / time).
 Several copies of the matrix are cycled through so that every launch reads from HBM, not from L2.
+
+    python -m paper_2505_16162_b200.opbench pass --shape llama13b --layers 4 --context 1280 --rows 5 --iters 10
+
+times the persistent pass kernel (rows 1 = a draft step under a seeded 45 % skip mask, rows k+1 = a verification pass)
+on a model of the named widths cut to ``--layers`` layers, small enough for a multi-pass profiler capture.
 """
 from __future__ import annotations
 
@@ -39,9 +44,41 @@ def bench_linear(n_out: int, n_in: int, rows: int, iters: int, warmup: int, dtyp
             "weight_bytes": nbytes, "gbs": nbytes / us / 1e3, "copies_cycled": copies}
 
 
+def bench_pass(shape_name: str, layers: int, context: int, rows: int, iters: int, seed: int = 0):
+    build.build()
+    from . import binding as kb
+    import numpy as np
+    torch.cuda.set_device(0)
+    shape = si.SHAPES[shape_name].with_layers(layers)
+    w = si.make_model_weights(shape, seed, device="cuda")
+    n_skip = int(round(0.45 * 2 * layers))
+    mask = si.skip_mask(seed + 102, 2 * layers, n_skip)
+    sess = kb.Session.from_shape(shape, w, context + 64, max_draft=8)
+    prompt = si.uniform_tokens(seed, 0, context, shape.vocab).numpy()
+    sess.prefill(prompt)
+    sess.set_skipmask(mask)
+    which, k = (0, 1) if rows == 1 else (1, rows - 1)
+    t = sess.time_pass(which, k, iters)
+    b = 2 if shape.dtype == "bf16" else 4
+    d, hd = shape.d_model, shape.head_dim
+    attn_w = (2 * d * shape.n_heads * hd + 2 * d * shape.n_kv_heads * hd) * b
+    mlp_w, head_w = 3 * d * shape.d_ff * b, shape.vocab * d * b
+    kv = 2 * shape.n_kv_heads * hd * b * (context + rows)
+    use = (lambda j: True) if rows > 1 else (lambda j: not mask[j])
+    n_attn = sum(1 for l in range(layers) if use(2 * l))
+    n_mlp = sum(1 for l in range(layers) if use(2 * l + 1))
+    nbytes = n_attn * (attn_w + kv) + n_mlp * mlp_w + head_w
+    return {"op": "pass", "shape": shape.name, "rows": rows, "context": context, "ms_per_pass": t["ms_per_pass"],
+            "algorithmic_bytes": nbytes, "gbs": nbytes / t["ms_per_pass"] / 1e6,
+            "attention_sublayers": n_attn, "mlp_sublayers": n_mlp}
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("op", choices=["linear"])
+    ap.add_argument("op", choices=["linear", "pass"])
+    ap.add_argument("--shape", default="llama13b")
+    ap.add_argument("--layers", type=int, default=4)
+    ap.add_argument("--context", type=int, default=1280)
     ap.add_argument("--n-out", type=int, default=131072)
     ap.add_argument("--n-in", type=int, default=5120)
     ap.add_argument("--rows", type=int, default=1)
@@ -49,7 +86,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp32"])
     a = ap.parse_args()
-    print(json.dumps(bench_linear(a.n_out, a.n_in, a.rows, a.iters, a.warmup, a.dtype)))
+    if a.op == "pass":
+        print(json.dumps(bench_pass(a.shape, a.layers, a.context, a.rows, a.iters)))
+    else:
+        print(json.dumps(bench_linear(a.n_out, a.n_in, a.rows, a.iters, a.warmup, a.dtype)))
 
 
 if __name__ == "__main__":
