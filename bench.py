@@ -244,11 +244,14 @@ def run_ours(args):
     round_bytes = k * (wd + kvd) + (wv + kvv)
     round_ms = k * t_draft["ms_per_pass"] + t_verify["ms_per_pass"]
     achieved = round_bytes / (round_ms * 1e-3) / 1e9
+    # DRAM traffic per launch: counters were taken on a 4-layer capture of the same kernel (profiles/); every weight
+    # byte is read once per pass, so the measured traffic / algorithmic ratio carries over to the full list
     traffic = None
     tp = os.path.join(ROOT, "profiles", "pass_kernel_traffic.json")
-    if os.path.exists(tp):
+    if os.path.exists(tp) and shape.dtype == "bf16":
         with open(tp) as f:
-            traffic = json.load(f).get(args.workload)
+            tr = json.load(f)
+        traffic = (k * (wd + kvd) * tr["ratio_rows1"] + (wv + kvv) * tr["ratio_rows5"]) / (k + 1)
     from paper_2505_16162_b200 import metrics
     n_skip = int(mask.sum())
     M_len = metrics.mean_generated_length(accepts) if len(accepts) else 1.0
