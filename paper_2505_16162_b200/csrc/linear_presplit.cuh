@@ -31,14 +31,7 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
     int ws = w_use % WS, it = w_use / WS;
     float *red = r.red, *red_ss = r.red_ss;
 
-    // RMSNorm scalar of every row from the producers' partial sums: warp w takes row w, lanes take CTAs lane, lane + 32, ...
-    if (normed && warp < p.M) {
-        float tot = 0.f;
-        for (int c = lane; c < n_cta; c += 32) tot += __ldcg(p.ss_in + (size_t)warp * n_cta + c);
-        tot = warp_sum(tot);
-        if (lane == 0) red_ss[warp] = 1.0f / sqrtf(tot / (float)p.K + p.eps);
-    }
-    float ss_acc = 0.f;                                     // token thread (tid < M): this CTA's sum of squares of y
+    float ss_acc = 0.f;                                     // lane 0 of warp n (n < M): this CTA's sum of squares of y row n
 
     for (int b = 0; b < s.n_batches; ++b) {
         const int g0 = b * GB, ng = min(s.n_groups - g0, GB);
@@ -56,6 +49,31 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
                     nx[t][q] = ld ? ld_frag4(xsrow + (size_t)slot * 192 + t * 64 + q * 4) : make_uint4(0u, 0u, 0u, 0u);
         };
         fetch(0);
+        if (b == 0 && normed && warp < p.M) {
+            // RMSNorm scalar of row `warp` from the producers' partial sums (lanes take CTAs lane, lane + 32, ...); issued
+            // after the first fragment fetch so that both round trips to L2 overlap
+            float tot = 0.f;
+            for (int c = lane; c < n_cta; c += 32) tot += __ldcg(p.ss_in + (size_t)warp * n_cta + c);
+            tot = warp_sum(tot);
+            if (lane == 0) red_ss[warp] = 1.0f / sqrtf(tot / (float)p.K + p.eps);
+        }
+        // this thread's epilogue items: (unit, token) pairs, token fastest among the M live tokens.  For a residual
+        // update the old value and the next gain are fetched now, long before the epilogue needs them.
+        const int gshift = s.swiglu ? 3 : 4, total = (ng << gshift) * p.M;
+        float xold[4], gnext[4];
+#pragma unroll
+        for (int it4 = 0; it4 < 4; ++it4) {
+            xold[it4] = 0.f; gnext[it4] = 1.f;
+            const int idx = tid + it4 * (NCW * 32);
+            if (p.epi == EPI_ADD && alive && idx < total) {
+                const int n = idx % p.M, ur = idx / p.M, gi = ur >> gshift, rr = ur & ((1 << gshift) - 1);
+                if (rr < s.group_size(g0 + gi)) {
+                    const int u = s.u_lo + s.group_lo(g0 + gi) + rr;
+                    xold[it4] = __ldcg(p.y + (size_t)n * p.units + u);
+                    if (p.next_gain) gnext[it4] = __ldg(p.next_gain + u);
+                }
+            }
+        }
         for (int kt = 0; kt < s.n_kt; ++kt) {
             const bool slot_valid = kt * NCW + warp < nslots;
             uint32_t bh[KSTEPS][2], bm[KSTEPS][2], bl[KSTEPS][2];
@@ -98,12 +116,13 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
             *reinterpret_cast<float4 *>(red + ((warp * GB + gi) * 32 + lane) * 4) =
                 make_float4(acc[gi][0], acc[gi][1], acc[gi][2], acc[gi][3]);
         asm volatile("bar.sync 1, %0;" ::"n"(NCW * 32) : "memory");
-        const int per_group = s.gsz * 8;                            // (unit, token) pairs per group
         if (alive) {
-            for (int idx = tid; idx < ng * per_group; idx += NCW * 32) {
-                const int gi = idx / per_group, rem = idx % per_group;
-                const int rr = rem >> 3, n = rem & 7;                 // unit within group, token
-                if (rr >= s.group_size(g0 + gi) || n >= p.M) continue;
+#pragma unroll
+            for (int it4 = 0; it4 < 4; ++it4) {
+                const int idx = tid + it4 * (NCW * 32);
+                if (idx >= total) break;
+                const int n = idx % p.M, ur = idx / p.M, gi = ur >> gshift, rr = ur & ((1 << gshift) - 1);
+                if (rr >= s.group_size(g0 + gi)) continue;
                 // rows 0..7 of the tile: regs 0,1; rows 8..15: regs 2,3
                 const int src_lane = (rr & 7) * 4 + (n >> 1), reg = n & 1;
                 const int e0 = s.swiglu ? reg : (rr >> 3) * 2 + reg;
@@ -122,10 +141,10 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
                     const float a = gt / (1.0f + expf(-gt)) * up;
                     if (p.ys) store_split(p.ys, p.units >> 7, n, u, a); else __stcg(yp, a);
                 } else if (p.epi == EPI_ADD) {
-                    const float v = __ldcg(yp) + s0 * ri;
+                    const float v = xold[it4] + s0 * ri;
                     __stcg(yp, v);
-                    if (p.ys) store_split(p.ys, p.units >> 7, n, u, p.next_gain ? v * __ldg(p.next_gain + u) : v);
-                    // leave v^2 where this thread alone read its first partial: the token thread adds them up below
+                    if (p.ys) store_split(p.ys, p.units >> 7, n, u, v * gnext[it4]);
+                    // leave v^2 where this thread alone read its first partial: warp n adds them up below
                     red[((0 * GB + gi) * 32 + src_lane) * 4 + e0] = v * v;
                 } else {
                     __stcg(yp, s0 * ri);
@@ -134,18 +153,21 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
         }
         if (p.ss_out) {
             asm volatile("bar.sync 1, %0;" ::"n"(NCW * 32) : "memory");
-            if (alive && tid < p.M) {
-                const int n = tid;
-                for (int gi = 0; gi < ng; ++gi) {
-                    const int gs = s.group_size(g0 + gi);
-                    for (int rr = 0; rr < gs; ++rr)
-                        ss_acc += red[((0 * GB + gi) * 32 + (rr & 7) * 4 + (n >> 1)) * 4 + (rr >> 3) * 2 + (n & 1)];
+            if (alive && warp < p.M) {
+                const int n = warp;
+                float part = 0.f;
+                for (int i = lane; i < (ng << gshift); i += 32) {
+                    const int gi = i >> gshift, rr = i & ((1 << gshift) - 1);
+                    if (rr < s.group_size(g0 + gi))
+                        part += red[((0 * GB + gi) * 32 + (rr & 7) * 4 + (n >> 1)) * 4 + (rr >> 3) * 2 + (n & 1)];
                 }
+                part = warp_sum(part);
+                ss_acc += part;
             }
         }
         asm volatile("bar.sync 1, %0;" ::"n"(NCW * 32) : "memory");
     }
-    if (p.ss_out && alive && tid < p.M) __stcg(p.ss_out + (size_t)tid * n_cta + cta, ss_acc);
+    if (p.ss_out && alive && warp < p.M && lane == 0) __stcg(p.ss_out + (size_t)warp * n_cta + cta, ss_acc);
 }
 
 }  // namespace stream

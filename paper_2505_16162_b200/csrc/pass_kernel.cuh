@@ -102,7 +102,6 @@ __device__ __forceinline__ bool grid_barrier(const Model &md, const Ring &r, uns
             }
             __nanosleep(32);
         }
-        __threadfence();
     }
     asm volatile("bar.sync 1, %0;" ::"n"(NCW * 32) : "memory");
     return alive && !*r.abort_flag;
