@@ -643,9 +643,9 @@ knnssd_status knnssd_init(const knnssd_config *cfg, const knnssd_weights *w, con
         ok2 &= dev_alloc(&c->mamax_v, (size_t)pass::MAXM * c->n_sms) == cudaSuccess;
         ok2 &= dev_alloc(&c->mamax_i, (size_t)pass::MAXM * c->n_sms) == cudaSuccess;
         ok2 &= dev_alloc(&c->trace, (size_t)2 * n_ops_cap) == cudaSuccess;
-        ok2 &= dev_alloc(&c->xs_x, (size_t)pass::MAXM * (d / 128) * 192) == cudaSuccess;
-        ok2 &= dev_alloc(&c->xs_attn, (size_t)pass::MAXM * (nq / 128) * 192) == cudaSuccess;
-        ok2 &= dev_alloc(&c->xs_act, (size_t)pass::MAXM * (g.d_ff / 128) * 192) == cudaSuccess;
+        ok2 &= dev_alloc(&c->xs_x, (size_t)pass::MAXM * (d / 128) * stream::SLOT_WORDS) == cudaSuccess;
+        ok2 &= dev_alloc(&c->xs_attn, (size_t)pass::MAXM * (nq / 128) * stream::SLOT_WORDS) == cudaSuccess;
+        ok2 &= dev_alloc(&c->xs_act, (size_t)pass::MAXM * (g.d_ff / 128) * stream::SLOT_WORDS) == cudaSuccess;
         ok2 &= dev_alloc(&c->ssp, (size_t)pass::MAXM * c->n_sms) == cudaSuccess;
         if (!ok2) { cudaGetLastError(); return bail(KNNSSD_ERR_CUDA); }
         pass::Model &md = c->model;

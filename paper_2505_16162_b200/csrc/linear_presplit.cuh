@@ -3,7 +3,7 @@
 // Same ring, same tiles, same sum order per output as consume_linear, but the activation operand arrives already
 // split into its three bf16 terms and laid out fragment by fragment (LinPhase::xs), written once by whoever produced
 // the activation.  The consumer therefore spends no arithmetic on the split that every CTA would otherwise repeat:
-// per column tile a lane loads twelve 16-byte pieces, one tile ahead of the tensor-core work.  RMSNorm's scalar comes
+// per column tile a lane loads four 16-byte pieces per term, one tile ahead of the tensor-core work.  RMSNorm's scalar comes
 // from per-CTA partial sums of squares that the producer of the row left in LinPhase::ss_in.
 //
 // The epilogue writes what the NEXT map needs: the fp32 result where something reads it as fp32 (projection buffer,
@@ -26,8 +26,8 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
     const bool normed = p.ss_in != nullptr;
     const bool row_live = g8 < p.M;
     const int nslots = p.K >> 7;
-    // this lane's 16-word runs: row g8, lane group t4; + slot * 192 + term * 64
-    const uint32_t *xsrow = p.xs + (((size_t)min(g8, p.M - 1) * nslots * 3) * 4 + t4) * 16;
+    // this lane's 16-word runs: row g8, lane group t4; + slot * SLOT_WORDS + term * 64
+    const uint32_t *xsrow = p.xs + (((size_t)min(g8, p.M - 1) * nslots * NTERM) * 4 + t4) * 16;
     int ws = w_use % WS, it = w_use / WS;
     float *red = r.red, *red_ss = r.red_ss;
 
@@ -38,15 +38,15 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
         float acc[GB][4];
 #pragma unroll
         for (int i = 0; i < GB; ++i) { acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f; }
-        uint4 nx[3][4];                                      // fragments of the next column tile (hi, mid, lo)
+        uint4 nx[NTERM][4];                                  // fragments of the next column tile, term by term
         auto fetch = [&](int kt) {
             const int slot = kt * NCW + warp;
             const bool ld = alive && row_live && slot < nslots;
 #pragma unroll
-            for (int t = 0; t < 3; ++t)
+            for (int t = 0; t < NTERM; ++t)
 #pragma unroll
                 for (int q = 0; q < 4; ++q)
-                    nx[t][q] = ld ? ld_frag4(xsrow + (size_t)slot * 192 + t * 64 + q * 4) : make_uint4(0u, 0u, 0u, 0u);
+                    nx[t][q] = ld ? ld_frag4(xsrow + (size_t)slot * SLOT_WORDS + t * 64 + q * 4) : make_uint4(0u, 0u, 0u, 0u);
         };
         fetch(0);
         if (b == 0 && normed && warp < p.M) {
@@ -76,13 +76,14 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
         }
         for (int kt = 0; kt < s.n_kt; ++kt) {
             const bool slot_valid = kt * NCW + warp < nslots;
-            uint32_t bh[KSTEPS][2], bm[KSTEPS][2], bl[KSTEPS][2];
+            uint32_t bf[NTERM][KSTEPS][2];                    // operand registers: term, k-step, (b0, b1)
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                bh[2 * q][0] = nx[0][q].x; bh[2 * q][1] = nx[0][q].y; bh[2 * q + 1][0] = nx[0][q].z; bh[2 * q + 1][1] = nx[0][q].w;
-                bm[2 * q][0] = nx[1][q].x; bm[2 * q][1] = nx[1][q].y; bm[2 * q + 1][0] = nx[1][q].z; bm[2 * q + 1][1] = nx[1][q].w;
-                bl[2 * q][0] = nx[2][q].x; bl[2 * q][1] = nx[2][q].y; bl[2 * q + 1][0] = nx[2][q].z; bl[2 * q + 1][1] = nx[2][q].w;
-            }
+            for (int t = 0; t < NTERM; ++t)
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    bf[t][2 * q][0] = nx[t][q].x; bf[t][2 * q][1] = nx[t][q].y;
+                    bf[t][2 * q + 1][0] = nx[t][q].z; bf[t][2 * q + 1][1] = nx[t][q].w;
+                }
             if (kt + 1 < s.n_kt) fetch(kt + 1);
 #pragma unroll
             for (int gi = 0; gi < GB; ++gi) {
@@ -90,19 +91,22 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
                 if (alive) alive = mbar_wait(&r.full_w[ws], it & 1, r.abort_flag, r.err, 5);
                 if (alive && slot_valid) {
                     const uint32_t base = smem_u32(r.wring + ws * WSTAGE) + lm_row * WPITCH + (warp * SLOT + lm_col) * 2;
-                    // six independent accumulator chains: term x parity of the k-step
-                    float tl[2][4] = {}, tm[2][4] = {}, th[2][4] = {};
+                    // independent accumulator chains: term x parity of the k-step; smallest terms are added first
+                    float tc[NTERM][2][4] = {};
 #pragma unroll
                     for (int j = 0; j < KSTEPS; ++j) {
                         uint32_t a0, a1, a2, a3;
                         ldmatrix_x4(base + j * 32, a0, a1, a2, a3);
-                        mma_bf16(tl[j & 1], a0, a1, a2, a3, bl[j][0], bl[j][1]);
-                        mma_bf16(tm[j & 1], a0, a1, a2, a3, bm[j][0], bm[j][1]);
-                        mma_bf16(th[j & 1], a0, a1, a2, a3, bh[j][0], bh[j][1]);
+#pragma unroll
+                        for (int t = NTERM - 1; t >= 0; --t) mma_bf16(tc[t][j & 1], a0, a1, a2, a3, bf[t][j][0], bf[t][j][1]);
                     }
 #pragma unroll
-                    for (int e = 0; e < 4; ++e)
-                        acc[gi][e] += ((tl[0][e] + tl[1][e]) + (tm[0][e] + tm[1][e])) + (th[0][e] + th[1][e]);
+                    for (int e = 0; e < 4; ++e) {
+                        float sum = tc[NTERM - 1][0][e] + tc[NTERM - 1][1][e];
+#pragma unroll
+                        for (int t = NTERM - 2; t >= 0; --t) sum += tc[t][0][e] + tc[t][1][e];
+                        acc[gi][e] += sum;
+                    }
                 }
                 __syncwarp();
                 if (alive && lane == 0) mbar_arrive(&r.empty_w[ws]);

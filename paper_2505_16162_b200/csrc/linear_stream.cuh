@@ -47,6 +47,8 @@ constexpr int MAX_SMEM = 232448;             // 227 KB
 constexpr int WS = (MAX_SMEM - RED_BYTES - SS_BYTES - BAR_BYTES) / WSTAGE;   // ring stages
 constexpr int SMEM_BYTES = WS * WSTAGE + RED_BYTES + SS_BYTES + BAR_BYTES;
 constexpr unsigned SPIN_LIMIT = 20000000u;
+constexpr int NTERM = 2;                     // bf16 terms a pre-split activation is carried in (2: hi + lo, 16-17 significant bits)
+constexpr int SLOT_WORDS = NTERM * 64;       // 32-bit words of one row's 128-column slot in a pre-split buffer
 static_assert(WS >= 4 && 2 * WS * 8 + 16 <= BAR_BYTES, "ring layout");
 
 // One linear map  y[m][u] = epilogue( sum_i W[u][i] * gain[i] * x[m][i] ).
@@ -63,7 +65,7 @@ struct LinPhase {
     int M;              // 1..8
     // Pre-split form (persistent pass kernel): the producer of an activation writes it already split into the three
     // bf16 terms, in the order the tensor-core operand wants, so the consuming map only loads fragments.
-    const uint32_t *xs;      // input  [M][K/128][3 terms][4][16] words (see split_index); nullptr = read x / gain
+    const uint32_t *xs;      // input  [M][K/128][NTERM terms][4][16] words (see split_index); nullptr = read x / gain
     const float *ss_in;      // [M][n_cta] partial sums of squares of the input rows (maps behind an RMSNorm); or nullptr
     uint32_t *ys;            // output in the same form for the next map (EPI_ADD: y * next_gain, SWIGLU: y); or nullptr
     const float *next_gain;  // [units] RMSNorm gain of the next map that reads y (EPI_ADD); nullptr = none
@@ -71,12 +73,12 @@ struct LinPhase {
 };
 
 // Word index of term 0 of column `col` of row m in a pre-split buffer with nslots = K / 128 column slots; the terms
-// of one value sit 64 words apart.  Inside a slot the words are ordered (lane group t4, k-step j, half h) so that the
+// of one value sit 64 words apart (NTERM terms per value).  Inside a slot the words are ordered (lane group t4, k-step j, half h) so that the
 // 16 words a lane needs for one term of one slot are contiguous: word 2j + h of group t4 packs columns
 // (16j + 8h + 2t4, 16j + 8h + 2t4 + 1) of the slot - the pair an m16n8k16 "col" operand register holds.
 __host__ __device__ __forceinline__ size_t split_index(int nslots, int m, int col) {
     const int s = col >> 7, within = col & 127, j = within >> 4, r = within & 15, h = r >> 3, t4 = (r & 7) >> 1;
-    return ((((size_t)m * nslots + s) * 3) * 4 + t4) * 16 + 2 * j + h;
+    return ((((size_t)m * nslots + s) * NTERM) * 4 + t4) * 16 + 2 * j + h;
 }
 
 // Shared-memory ring and its barriers, carved out of the CTA's dynamic shared memory.
@@ -147,14 +149,16 @@ __device__ __forceinline__ void split3(float v, uint32_t &hi, uint32_t &mid, uin
     lo = float_to_bf16_rne(r2);
 }
 
-// Write one activation value in pre-split form.
+// Write one activation value in pre-split form: hi = bf16(v), then the bf16 roundings of the successive residuals
+// (each residual is exact in fp32).
 __device__ __forceinline__ void store_split(uint32_t *buf, int nslots, int m, int col, float v) {
-    uint32_t hi, mid, lo;
-    split3(v, hi, mid, lo);
     bf16_t *b = reinterpret_cast<bf16_t *>(buf) + 2 * split_index(nslots, m, col) + (col & 1);
-    __stcg(b, (bf16_t)hi);
-    __stcg(b + 128, (bf16_t)mid);
-    __stcg(b + 256, (bf16_t)lo);
+#pragma unroll
+    for (int t = 0; t < NTERM; ++t) {
+        const uint32_t h = float_to_bf16_rne(v);
+        __stcg(b + 128 * t, (bf16_t)h);
+        v -= __uint_as_float(h << 16);
+    }
 }
 
 // The CTA's share of a linear map: units [u_lo, u_lo + n_units) in n_groups groups whose sizes differ by at

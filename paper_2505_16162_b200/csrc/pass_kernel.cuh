@@ -567,7 +567,7 @@ __global__ void __launch_bounds__(stream::NTHREADS, 1) pass_kernel(const Model m
             if (op.is_head) {
                 if (pr.head_row0 >= pr.M) ran = false;
                 lp.M = pr.M - pr.head_row0;
-                lp.xs += (size_t)pr.head_row0 * (lp.K >> 7) * 192;
+                lp.xs += (size_t)pr.head_row0 * (lp.K >> 7) * stream::SLOT_WORDS;
                 lp.ss_in += (size_t)pr.head_row0 * n_cta;
                 lp.y += (size_t)(pr.out_row0 + pr.head_row0) * lp.units;
             }
