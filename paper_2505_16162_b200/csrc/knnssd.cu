@@ -64,6 +64,7 @@ struct knnssd_ctx {
     pass::Model model{};
     pass::Op *ops_full = nullptr, *ops_draft = nullptr;     // device op lists
     int n_ops_full = 0, n_ops_draft = 0, bar_full = 0, bar_draft = 0;   // ops and barriers (without head / hidden parts)
+    int attn_full = 0, attn_draft = 0;                                  // attention sublayers in each list
     std::vector<unsigned char> ops_draft_mask;              // the mask ops_draft was built for
     unsigned long long *bar = nullptr, bar_total = 0;
     int *gabort = nullptr, *attn_cnt = nullptr, *amax_cnt = nullptr;
@@ -190,11 +191,11 @@ LinearArgs make_args(const void *W0, int rows0, int n_in, const float *x, const 
 // ---- persistent pass kernel: op lists and launch ----------------------------------------------------------------
 // The list of one pass under a skip mask (nullptr = full model).  n_bar receives the number of grid barriers of the
 // body; the head part (when rows get logits) adds one more.
-std::vector<pass::Op> build_ops(const knnssd_ctx *c, const unsigned char *mask, int *n_bar) {
+std::vector<pass::Op> build_ops(const knnssd_ctx *c, const unsigned char *mask, int *n_bar, int *n_attn) {
     const knnssd_config &g = c->cfg;
     const int d = g.d_model, hd = g.head_dim, nq = g.n_heads * hd, nkv = g.n_kv_heads * hd, F = g.d_ff, V = g.vocab;
     std::vector<pass::Op> ops;
-    int bars = 0;
+    int bars = 0, attn = 0;
     auto lin = [&](const void *W0, int rows0, int K, const float *x, const float *gain, float *y, int epi) {
         pass::Op o{};
         o.type = pass::OP_LINEAR; o.barrier_after = 1;
@@ -222,6 +223,10 @@ std::vector<pass::Op> build_ops(const knnssd_ctx *c, const unsigned char *mask, 
             a.vc = reinterpret_cast<bf16_t *>(c->vcache) + (size_t)l * layer_stride;
             a.lin.ys = c->xs_attn;
             ops.push_back(a);
+            pass::Op mg{};                               // runs (and its barrier counts) only in passes of >= MERGE_ROWS rows
+            mg.type = pass::OP_ATTN_MERGE; mg.barrier_after = 1; mg.layer = l; mg.lin.ys = c->xs_attn;
+            ops.push_back(mg);
+            ++attn;
             pass::Op o = lin(ly.wo, d, nq, c->attn, nullptr, c->x, EPI_ADD);
             o.layer = l;
             o.lin.xs = c->xs_attn; o.lin.ys = c->xs_x; o.lin.ss_out = c->ssp;
@@ -258,6 +263,7 @@ std::vector<pass::Op> build_ops(const knnssd_ctx *c, const unsigned char *mask, 
         if (o.type == pass::OP_LINEAR && o.lin.gain) next_gain = o.lin.gain;
     }
     *n_bar = bars;
+    *n_attn = attn;
     return ops;
 }
 
@@ -283,24 +289,25 @@ template <int HD> cudaError_t launch_pass_t(knnssd_ctx *c, const pass::Params &p
 void run_pass_mega(knnssd_ctx *c, int M, const int *tok_dev, int pos_off, const unsigned char *mask, int head_row0,
                    int *argmax_out, bool want_hidden, int out_row0 = 0) {
     pass::Params pr{};
-    int bars;
+    int bars, n_attn;
     if (!mask) {
-        pr.ops = c->ops_full; pr.n_ops = c->n_ops_full; bars = c->bar_full;
+        pr.ops = c->ops_full; pr.n_ops = c->n_ops_full; bars = c->bar_full; n_attn = c->attn_full;
     } else {
         const size_t n = 2 * (size_t)c->cfg.n_layers;
         if (c->ops_draft_mask.size() != n || std::memcmp(c->ops_draft_mask.data(), mask, n) != 0) {
-            const std::vector<pass::Op> ops = build_ops(c, mask, &c->bar_draft);
+            const std::vector<pass::Op> ops = build_ops(c, mask, &c->bar_draft, &c->attn_draft);
             c->n_ops_draft = (int)ops.size();
             if (upload_ops(c, ops, c->ops_draft) != KNNSSD_OK) return;
             c->ops_draft_mask.assign(mask, mask + n);
         }
-        pr.ops = c->ops_draft; pr.n_ops = c->n_ops_draft; bars = c->bar_draft;
+        pr.ops = c->ops_draft; pr.n_ops = c->n_ops_draft; bars = c->bar_draft; n_attn = c->attn_draft;
     }
     pr.M = M; pr.tok = tok_dev; pr.pos_off = pos_off; pr.head_row0 = head_row0; pr.argmax_out = argmax_out;
     pr.want_hidden = want_hidden ? 1 : 0;
     pr.out_row0 = out_row0;
     pr.bar_base = c->bar_total;
     if (head_row0 < M) bars += 1;
+    if (M >= pass::MERGE_ROWS) bars += n_attn;
     const cudaError_t e = c->cfg.head_dim == 128 ? launch_pass_t<128>(c, pr) : launch_pass_t<64>(c, pr);
     if (e == cudaSuccess) c->bar_total += (unsigned long long)bars * (unsigned long long)c->n_sms;
     c->launches++;
@@ -630,7 +637,7 @@ knnssd_status knnssd_init(const knnssd_config *cfg, const knnssd_weights *w, con
     if (g.dtype == 1 && coop && d % 128 == 0 && nq % 128 == 0 && g.d_ff % 128 == 0 && d >= 256 && nq >= 256 && g.d_ff >= 256 &&
         g.max_seq <= 64 * pass::SEGP) {            // the attention merge keeps at most 64 segment statistics per warp
         const int n_seg_max = (g.max_seq + pass::SEGP - 1) / pass::SEGP;
-        const int n_ops_cap = 5 * g.n_layers + 8;
+        const int n_ops_cap = 6 * g.n_layers + 8;
         bool ok2 = true;
         ok2 &= dev_alloc(&c->ops_full, (size_t)n_ops_cap) == cudaSuccess;
         ok2 &= dev_alloc(&c->ops_draft, (size_t)n_ops_cap) == cudaSuccess;
@@ -657,7 +664,7 @@ knnssd_status knnssd_init(const knnssd_config *cfg, const knnssd_weights *w, con
         md.amax_cnt = c->amax_cnt; md.state = c->state; md.bar = c->bar; md.gabort = c->gabort; md.err = stream_err_ptr();
         c->mega_ok = true;
         reset_mega_state(c);
-        const std::vector<pass::Op> ops = build_ops(c, nullptr, &c->bar_full);
+        const std::vector<pass::Op> ops = build_ops(c, nullptr, &c->bar_full, &c->attn_full);
         c->n_ops_full = (int)ops.size();
         if (upload_ops(c, ops, c->ops_full) != KNNSSD_OK) return bail(KNNSSD_ERR_CUDA);
     }
@@ -956,7 +963,8 @@ knnssd_status knnssd_trace_pass(knnssd_ctx *c, int which, int k, int cap, int *o
     if (st != KNNSSD_OK) return st;
     std::vector<pass::Op> ops;
     int bars = 0;
-    ops = build_ops(c, which == 0 ? c->active_mask.data() : nullptr, &bars);
+    int n_attn_unused = 0;
+    ops = build_ops(c, which == 0 ? c->active_mask.data() : nullptr, &bars, &n_attn_unused);
     const int n = (int)ops.size();
     CUDA_TRY(c, cudaMemsetAsync(c->trace, 0, sizeof(unsigned long long) * 2 * n, s));
     c->model.trace = c->trace;

@@ -27,7 +27,8 @@ constexpr int MAXM = 8;            // rows per pass this kernel handles
 constexpr int SEGP = 64;           // attention: positions per segment (fixed absolute boundaries)
 constexpr unsigned BAR_SPIN_LIMIT = 4000000u;
 
-enum { OP_EMBED = 0, OP_LINEAR = 1, OP_ATTN = 2, OP_HIDDEN = 3, OP_ARGMAX = 4 };
+enum { OP_EMBED = 0, OP_LINEAR = 1, OP_ATTN = 2, OP_HIDDEN = 3, OP_ARGMAX = 4, OP_ATTN_MERGE = 5 };
+constexpr int MERGE_ROWS = 3;      // passes with at least this many rows merge attention partials in a separate operation
 
 struct Op {
     int type;
@@ -258,6 +259,42 @@ __device__ __forceinline__ void mma_bf16_top(float (&c)[4], uint32_t a0, uint32_
                  : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
 }
 
+// Merge the segment partials of one (row m, head h) in segment order and write the result pre-split (one warp).
+template <int HD>
+__device__ __forceinline__ void attn_merge_row(const Model &md, const Op &op, int P0, int m, int h, int lane) {
+    constexpr int DPL = HD / 32;
+    const int H = md.H, d0 = DPL * lane;
+    const int n_seg_m = (P0 + m + SEGP) / SEGP;
+    const size_t base = ((size_t)m * H + h) * md.n_seg_max;
+    // segment statistics: lane s holds segments s and s + 32 (contexts up to 4096); fixed-order warp reductions
+    const float2 ml0 = lane < n_seg_m ? __ldcg(md.part_ml + base + lane) : make_float2(-INFINITY, 0.f);
+    const float2 ml1 = lane + 32 < n_seg_m ? __ldcg(md.part_ml + base + lane + 32) : make_float2(-INFINITY, 0.f);
+    const float gm = warp_max(fmaxf(ml0.x, ml1.x));
+    const float w0 = ml0.x == -INFINITY ? 0.f : expf(ml0.x - gm), w1 = ml1.x == -INFINITY ? 0.f : expf(ml1.x - gm);
+    const float L = warp_sum(fmaf(ml1.y, w1, ml0.y * w0));
+    // weighted sum of the partial outputs in segment order, sixteen segments in flight at a time
+    float acc[DPL];
+#pragma unroll
+    for (int e = 0; e < DPL; ++e) acc[e] = 0.f;
+    for (int s0 = 0; s0 < n_seg_m; s0 += 16) {
+        float pv[16][DPL];
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+#pragma unroll
+            for (int e = 0; e < DPL; ++e)
+                pv[i][e] = s0 + i < n_seg_m ? __ldcg(md.part_o + (base + s0 + i) * HD + d0 + e) : 0.f;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const int sg = s0 + i;
+            const float w = __shfl_sync(0xffffffffu, sg < 32 ? w0 : w1, sg & 31);
+#pragma unroll
+            for (int e = 0; e < DPL; ++e) acc[e] = fmaf(pv[i][e], w, acc[e]);
+        }
+    }
+#pragma unroll
+    for (int e = 0; e < DPL; ++e) stream::store_split(op.lin.ys, (H * HD) >> 7, m, h * HD + d0 + e, acc[e] / L);
+}
+
 #ifndef KNNSSD_ATT_STAMP
 #define KNNSSD_ATT_STAMP(i)
 #endif
@@ -276,7 +313,7 @@ __device__ __forceinline__ void mma_bf16_top(float (&c)[4], uint32_t a0, uint32_
 // A lane ends up with output dimensions [DL*t4, DL*t4 + DL) of row g8, the run it holds of q.
 template <int HD>
 __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const Params &pr, const Ring &r, int cta, int n_cta,
-                                           int warp, int lane) {
+                                           int warp, int lane, bool defer_merge) {
     constexpr int DL = HD / 4;         // dimensions of q / o per lane
     constexpr int NW = HD / 8;         // 32-bit words of a K row per lane
     constexpr int KS = HD / 16;        // k-steps of Q K^T
@@ -478,6 +515,7 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
                 __stcg(reinterpret_cast<float4 *>(po + VJ + j), make_float4(o[j][1], o[j + 1][1], o[j + 2][1], o[j + 3][1]));
             }
         }
+        if (defer_merge) continue;                            // a separate merge operation follows a grid barrier
         __threadfence();
         __syncwarp();
         KNNSSD_ATT_STAMP(6);
@@ -490,43 +528,23 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
         const unsigned last_mask = __ballot_sync(0xffffffffu, last);     // bit 4*m set: this warp finishes (row m, head h)
         if (last_mask) {
             __threadfence();
-            const int d0 = DPL * lane;
             for (int m = m_first; m < M; ++m) {
                 if (!((last_mask >> (4 * m)) & 1u)) continue;
-                const int n_seg_m = (P0 + m + SEGP) / SEGP;
-                const size_t base = ((size_t)m * H + h) * md.n_seg_max;
-                // segment statistics: lane s holds segments s and s + 32 (contexts up to 4096); fixed-order warp reductions
-                const float2 ml0 = lane < n_seg_m ? __ldcg(md.part_ml + base + lane) : make_float2(-INFINITY, 0.f);
-                const float2 ml1 = lane + 32 < n_seg_m ? __ldcg(md.part_ml + base + lane + 32) : make_float2(-INFINITY, 0.f);
-                const float gm = warp_max(fmaxf(ml0.x, ml1.x));
-                const float w0 = ml0.x == -INFINITY ? 0.f : expf(ml0.x - gm), w1 = ml1.x == -INFINITY ? 0.f : expf(ml1.x - gm);
-                const float L = warp_sum(fmaf(ml1.y, w1, ml0.y * w0));
-                // weighted sum of the partial outputs in segment order, sixteen segments in flight at a time
-                float acc[DPL];
-#pragma unroll
-                for (int e = 0; e < DPL; ++e) acc[e] = 0.f;
-                for (int s0 = 0; s0 < n_seg_m; s0 += 16) {
-                    float pv[16][DPL];
-#pragma unroll
-                    for (int i = 0; i < 16; ++i)
-#pragma unroll
-                        for (int e = 0; e < DPL; ++e)
-                            pv[i][e] = s0 + i < n_seg_m ? __ldcg(md.part_o + (base + s0 + i) * HD + d0 + e) : 0.f;
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        const int sg = s0 + i;
-                        const float w = __shfl_sync(0xffffffffu, sg < 32 ? w0 : w1, sg & 31);
-#pragma unroll
-                        for (int e = 0; e < DPL; ++e) acc[e] = fmaf(pv[i][e], w, acc[e]);
-                    }
-                }
-#pragma unroll
-                for (int e = 0; e < DPL; ++e) stream::store_split(op.lin.ys, (H * HD) >> 7, m, h * HD + d0 + e, acc[e] / L);
+                attn_merge_row<HD>(md, op, P0, m, h, lane);
                 if (lane == 0) md.attn_cnt[m * H + h] = 0;
             }
         }
         KNNSSD_ATT_STAMP(8);
     }
+}
+
+// With several rows the warp that finishes a head last would merge all its rows one after the other; the merges
+// then run as an operation of their own instead, one (row, head) per warp across the whole grid.
+template <int HD>
+__device__ __forceinline__ void attn_merge_phase(const Model &md, const Op &op, const Params &pr, int cta, int n_cta, int warp,
+                                                 int lane) {
+    const int P0 = md.state->len + pr.pos_off, jobs = pr.M * md.H;
+    for (int j = warp * n_cta + cta; j < jobs; j += NCW * n_cta) attn_merge_row<HD>(md, op, P0, j / md.H, j % md.H, lane);
 }
 
 // ---- the pass ---------------------------------------------------------------------------------------------------
@@ -574,7 +592,8 @@ __global__ void __launch_bounds__(stream::NTHREADS, 1) pass_kernel(const Model m
             if (ran) stream::consume_linear_pre(lp, r, cta, n_cta, warp, lane, w_use, alive);
         } else if (alive) {
             if (op.type == OP_EMBED) embed_phase(md, op, pr, r, cta, n_cta, tid);
-            else if (op.type == OP_ATTN) attn_phase<HD>(md, op, pr, r, cta, n_cta, warp, lane);
+            else if (op.type == OP_ATTN) attn_phase<HD>(md, op, pr, r, cta, n_cta, warp, lane, pr.M >= MERGE_ROWS);
+            else if (op.type == OP_ATTN_MERGE) { if (pr.M >= MERGE_ROWS) attn_merge_phase<HD>(md, op, pr, cta, n_cta, warp, lane); else ran = false; }
             else if (op.type == OP_HIDDEN) { if (pr.want_hidden) hidden_phase(md, pr, r, cta, tid); else ran = false; }
             else if (op.type == OP_ARGMAX) { if (pr.head_row0 < pr.M) argmax_phase(md, pr, r, cta, n_cta, tid); else ran = false; }
         }
