@@ -26,8 +26,8 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
     const bool normed = p.ss_in != nullptr;
     const bool row_live = g8 < p.M;
     const int nslots = p.K >> 7;
-    // this lane's 16-word runs: row g8, lane group t4; + slot * SLOT_WORDS + term * 64
-    const uint32_t *xsrow = p.xs + (((size_t)min(g8, p.M - 1) * nslots * NTERM) * 4 + t4) * 16;
+    // this lane's 16-byte pieces: row g8, lane group t4; + slot * SLOT_WORDS + term * 64 + piece * 16
+    const uint32_t *xsrow = p.xs + (size_t)min(g8, p.M - 1) * nslots * SLOT_WORDS + t4 * 4;
     int ws = w_use % WS, it = w_use / WS;
     float *red = r.red, *red_ss = r.red_ss;
 
@@ -46,7 +46,7 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
             for (int t = 0; t < NTERM; ++t)
 #pragma unroll
                 for (int q = 0; q < 4; ++q)
-                    nx[t][q] = ld ? ld_frag4(xsrow + (size_t)slot * SLOT_WORDS + t * 64 + q * 4) : make_uint4(0u, 0u, 0u, 0u);
+                    nx[t][q] = ld ? ld_frag4(xsrow + (size_t)slot * SLOT_WORDS + t * 64 + q * 16) : make_uint4(0u, 0u, 0u, 0u);
         };
         fetch(0);
         if (b == 0 && normed && warp < p.M) {

@@ -73,12 +73,14 @@ struct LinPhase {
 };
 
 // Word index of term 0 of column `col` of row m in a pre-split buffer with nslots = K / 128 column slots; the terms
-// of one value sit 64 words apart (NTERM terms per value).  Inside a slot the words are ordered (lane group t4, k-step j, half h) so that the
-// 16 words a lane needs for one term of one slot are contiguous: word 2j + h of group t4 packs columns
-// (16j + 8h + 2t4, 16j + 8h + 2t4 + 1) of the slot - the pair an m16n8k16 "col" operand register holds.
+// of one value sit 64 words apart (NTERM terms per value).  A lane (group t4) needs 16 words per term and slot: word
+// 2j + h packs columns (16j + 8h + 2t4, 16j + 8h + 2t4 + 1) of the slot - the pair an m16n8k16 "col" operand register
+// holds for k-step j.  They are stored as four 16-byte pieces q = 0..3, and piece q of the four lane groups is
+// contiguous (64 bytes), so one warp-wide 16-byte load touches whole 32-byte sectors only.
 __host__ __device__ __forceinline__ size_t split_index(int nslots, int m, int col) {
     const int s = col >> 7, within = col & 127, j = within >> 4, r = within & 15, h = r >> 3, t4 = (r & 7) >> 1;
-    return ((((size_t)m * nslots + s) * NTERM) * 4 + t4) * 16 + 2 * j + h;
+    const int wr = 2 * j + h;                 // word of the lane's 16-word run: q = wr / 4 is the 16-byte piece it lies in
+    return (((size_t)m * nslots + s) * NTERM) * 64 + (wr >> 2) * 16 + t4 * 4 + (wr & 3);
 }
 
 // Shared-memory ring and its barriers, carved out of the CTA's dynamic shared memory.
