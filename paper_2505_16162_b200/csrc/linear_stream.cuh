@@ -37,10 +37,10 @@ constexpr int WSTAGE = WROWS * WPITCH;
 constexpr int NCW = 8;                       // consumer warps
 constexpr int SLOT = SEG / NCW;              // columns per consumer warp per tile (128 = 8 k16 steps)
 constexpr int KSTEPS = SLOT / 16;
-constexpr int GB = 8;                        // groups per batch
+constexpr int GB = 4;                        // groups per batch
 constexpr int NTHREADS = (NCW + 4) * 32;      // two consumer warpgroups + the producer's warpgroup (one warp of it works)
 constexpr int REGS_PRODUCER = 40, REGS_CONSUMER = 232;
-constexpr int RED_BYTES = NCW * GB * 32 * 4 * 4;
+constexpr int RED_BYTES = NCW * 8 * 32 * 4 * 4;  // reduction buffer (sized for 8 groups; attention keeps its K/V stash here)
 constexpr int SS_BYTES = NCW * 8 * 4;
 constexpr int BAR_BYTES = 1024;
 constexpr int MAX_SMEM = 232448;             // 227 KB
