@@ -122,6 +122,19 @@ def build_inputs(workload: str, seed: int, device, gamma: float):
     return shape, masks, anchors, prompt, max_new
 
 
+def reduce_over_replicas(ms, e2e_s, tokens, e2e_tokens, launches, device, world):
+    """Whole-job figures of N independent replicas (one per GPU, no traffic between them while they work): the slowest
+    replica sets the time (MAX over ranks), work adds up (SUM over ranks)."""
+    if world <= 1:
+        return ms, e2e_s, tokens, e2e_tokens, launches
+    import torch.distributed as dist
+    t = torch.tensor([ms, e2e_s], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    c = torch.tensor([tokens, e2e_tokens, launches], device=device, dtype=torch.float64)
+    dist.all_reduce(c, op=dist.ReduceOp.SUM)
+    return float(t[0]), float(t[1]), int(c[0]), int(c[1]), int(c[2])
+
+
 def run_ours(args):
     from paper_2505_16162_b200 import build
     build.build()
@@ -225,14 +238,7 @@ def run_ours(args):
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - te
 
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([ms, e2e_s], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, e2e_s = float(t[0]), float(t[1])
-        c = torch.tensor([tokens, e2e_tokens, launches], device=dev, dtype=torch.float64)
-        dist.all_reduce(c, op=dist.ReduceOp.SUM)
-        tokens, e2e_tokens, launches = int(c[0]), int(c[1]), int(c[2])
+    ms, e2e_s, tokens, e2e_tokens, launches = reduce_over_replicas(ms, e2e_s, tokens, e2e_tokens, launches, dev, world)
 
     if rank != 0:
         return
