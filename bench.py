@@ -326,6 +326,60 @@ def cpu_baseline(args, shape, w_dev, mask, steps, warmup, per_step=None):
                       f"({len(times)} timed step(s), decode only)", "ms_per_step": 1e3 * total / len(times)}
 
 
+def run_stream(args):
+    """Mixed-domain request stream on the 13B shape (the fifth workload): requests drawn from 5 synthetic domains, the
+    order given by the mix-ratio chain (Sec. 4.2), prompts of 128-1024 random tokens; per request: prefill, the
+    request's pooled state shifted into its domain's cluster, cosine selection of the skip mask, 256 tokens of
+    self-speculative decoding with k = 4.  The domains' masks are drawn from one pool of sublayers whose output
+    projections are scaled by gamma (what the method presumes of skippable sublayers)."""
+    from paper_2505_16162_b200 import build
+    build.build()
+    from paper_2505_16162_b200 import binding as kb
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    shape = si.SHAPES["llama13b"]
+    per = args.stream_requests // N_DOMAINS
+    n_req, k, max_new = per * N_DOMAINS, 4, 256
+    pool, masks = si.nested_skip_masks(args.seed + 100, shape.n_layers, N_DOMAINS, 23, 21, 19, 17)
+    damp = {int(j): args.gamma for j in np.nonzero(pool)[0]} if args.gamma < 1.0 else None
+    w = si.make_model_weights(shape, args.seed, device=dev, damp=damp)
+    anchors = si.anchors(args.seed, N_DOMAINS, PER_DOMAIN, shape.d_model, 0.2).to(dev)
+    cen = si.domain_centroids(args.seed, N_DOMAINS, shape.d_model).to(dev)
+    labels = si.request_stream(args.seed, N_DOMAINS, per, args.mix_ratio)
+    lengths = si.prompt_lengths(args.seed, n_req, 128, 1024)
+    sess = kb.Session.from_shape(shape, w, 1024 + max_new + 64, max_draft=8, anchors=anchors, skip_masks=masks,
+                                 anchors_per_domain=PER_DOMAIN)
+    sel_ms, pre_ms, draft_ms, verify_ms, alphas, mlen, correct, tokens = [], [], [], [], [], [], 0, 0
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for i in range(n_req):
+        prompt = si.uniform_tokens(args.seed, 1 + i, lengths[i], shape.vocab).numpy()
+        _, pooled = sess.prefill(prompt, want_pooled=True)
+        c = cen[labels[i]]
+        query = (pooled + 4.0 * pooled.norm() / c.norm() * c).contiguous()     # a draw from the domain's cluster
+        dom, _, _ = sess.select_skipset(query)
+        r = sess.decode(max_new, k)
+        st = r["stats"]
+        correct += int(dom == labels[i])
+        tokens += len(r["tokens"])
+        sel_ms.append(st["ms_select"]); pre_ms.append(st["ms_prefill"])
+        draft_ms.append(st["ms_draft"] / max(1, st["drafted"])); verify_ms.append(st["ms_verify"] / max(1, st["rounds"]))
+        alphas.append(st["accepted"] / max(1, st["drafted"])); mlen.append(len(r["tokens"]) / max(1, st["rounds"]))
+    torch.cuda.synchronize()
+    wall = time.perf_counter() - t0
+    med = statistics.median
+    print(json.dumps({
+        "workload": f"stream13b: {n_req} requests from {N_DOMAINS} domains, mix ratio {args.mix_ratio}, prompts 128-1024, "
+                    f"{max_new} new tokens, k={k}, gamma={args.gamma}",
+        "domain_accuracy": correct / n_req, "tokens_per_s_incl_prefill": tokens / wall, "wall_s": wall,
+        "select_ms_median": med(sel_ms), "select_ms_max": max(sel_ms), "prefill_ms_median": med(pre_ms),
+        "draft_pass_ms_median": med(draft_ms), "verify_pass_ms_median": med(verify_ms),
+        "alpha_mean": sum(alphas) / n_req, "alpha_min": min(alphas), "mean_generated_length": sum(mlen) / n_req,
+        "switches": sum(1 for a, b in zip(labels, labels[1:]) if a != b)}))
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -361,8 +415,13 @@ def main():
     ap.add_argument("--cpu-prompt", type=int, default=16)
     ap.add_argument("--cpu-new", type=int, default=6)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--stream-requests", type=int, default=0,
+                    help="run the mixed-domain request stream (fifth workload) with this many requests instead of the bench")
+    ap.add_argument("--mix-ratio", type=float, default=1.0)
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.stream_requests > 0:
+        run_stream(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

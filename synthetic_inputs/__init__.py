@@ -20,6 +20,7 @@ from .generators import (  # noqa: F401
     uniform_tokens,
     skip_mask,
     skip_mask_split,
+    nested_skip_masks,
     domain_centroids,
     anchors,
     prompt_lengths,

@@ -128,6 +128,22 @@ def skip_mask_split(seed: int, n_layers: int, n_attn_skip: int, n_mlp_skip: int)
     return z
 
 
+def nested_skip_masks(seed: int, n_layers: int, n_domains: int, pool_attn: int, pool_mlp: int,
+                      n_attn_skip: int, n_mlp_skip: int):
+    """Per-domain masks drawn from one common pool of skippable sublayers.
+
+    Returns (pool, masks): ``pool`` uint8[2L] marks pool_attn attention and pool_mlp MLP sublayers; each of the
+    ``n_domains`` rows of ``masks`` skips n_attn_skip attention and n_mlp_skip MLP sublayers chosen (by seeded rank)
+    inside the pool, so the domains' masks differ but share the sublayers that matter to none of them."""
+    pool = skip_mask_split(seed, n_layers, pool_attn, pool_mlp)
+    masks = np.zeros((n_domains, 2 * n_layers), dtype=np.uint8)
+    for i in range(n_domains):
+        order = _ranks(seed + 1 + i, TensorId.MASK, 2 * n_layers)
+        masks[i, [j for j in order if pool[j] and j % 2 == 0][:n_attn_skip]] = 1
+        masks[i, [j for j in order if pool[j] and j % 2 == 1][:n_mlp_skip]] = 1
+    return pool, masks
+
+
 def domain_centroids(seed: int, n_domains: int, d: int) -> torch.Tensor:
     idx = torch.arange(n_domains * d, dtype=torch.int64)
     return normal_f32(seed, TensorId.CENTROID, idx, 1.0).view(n_domains, d)
