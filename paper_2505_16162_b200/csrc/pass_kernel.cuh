@@ -304,12 +304,13 @@ __device__ __forceinline__ void attn_merge_row(const Model &md, const Op &op, in
 //   scores  S = Q K^T   m16n8k16 bf16: the 8 columns of a tile are 8 consecutive positions (column n = g8 of the K
 //           operand = position 8*nt + g8).  A dot product does not care in which order its terms are taken, so k-step
 //           s pairs k-indices with the dimensions (DL*t4 + 4s .. + 3): every lane then reads one contiguous run of
-//           DL = HD/4 dimensions of "its" K row (16-byte loads) and holds the same run of q, split into three bf16
-//           terms so that the products are exact.
-//   output  O += P V    m16n8k8 tf32: k-index t4 / t4 + 4 stands for positions 2*t4 / 2*t4 + 1 of the tile - exactly
-//           the two scores the lane already holds - and column n = g8 of V-tile j is dimension (HD/8)*g8 + j, so a lane
-//           reads HD/8 contiguous dimensions of two V rows.  bf16 values are exact tf32 values; p is split into two
-//           tf32 terms (22 bits).
+//           DL = HD/4 dimensions of "its" K row (16-byte loads) and holds the same run of q, split into two bf16
+//           terms (hi + lo, 16-17 bits); products are exact.
+//   output  O += P V    m16n8k16 bf16 over pairs of tiles: k-indices 2t4, 2t4+1 stand for positions 2t4, 2t4+1 of the
+//           first tile and 2t4+8, 2t4+9 for the same positions of the second - exactly the four scores the lane already
+//           holds - and column n = g8 of V-tile j is dimension (HD/8)*g8 + j, so a lane reads HD/8 contiguous
+//           dimensions of four V rows; an operand register (two positions of one dimension) is one byte-permute of two
+//           loaded words.  p is split into two bf16 terms.
 // A lane ends up with output dimensions [DL*t4, DL*t4 + DL) of row g8, the run it holds of q.
 template <int HD>
 __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const Params &pr, const Ring &r, int cta, int n_cta,
@@ -388,13 +389,13 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
             }
         }
         __syncwarp();
-        uint32_t qh[NW], qm[NW], ql[NW];                     // word w = dimensions (2w, 2w + 1) of the run
+        uint32_t qh[NW], ql[NW];                             // word w = dimensions (2w, 2w + 1) of the run; q = hi + lo
 #pragma unroll
         for (int w = 0; w < NW; ++w) {
-            uint32_t h0, m0, l0, h1, m1, l1;
-            stream::split3(qf[2 * w], h0, m0, l0);
-            stream::split3(qf[2 * w + 1], h1, m1, l1);
-            qh[w] = h0 | (h1 << 16); qm[w] = m0 | (m1 << 16); ql[w] = l0 | (l1 << 16);
+            const uint32_t h0 = float_to_bf16_rne(qf[2 * w]), h1 = float_to_bf16_rne(qf[2 * w + 1]);
+            const uint32_t l0 = float_to_bf16_rne(qf[2 * w] - __uint_as_float(h0 << 16));
+            const uint32_t l1 = float_to_bf16_rne(qf[2 * w + 1] - __uint_as_float(h1 << 16));
+            qh[w] = h0 | (h1 << 16); ql[w] = l0 | (l1 << 16);
         }
 
         KNNSSD_ATT_STAMP(1);
@@ -415,19 +416,17 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
                 uint4(&kq)[NW / 4] = kb[nt % KR];
-                float ch[4] = {}, cm[4] = {}, cl[4] = {};
+                float ch[4] = {}, cl[4] = {};
 #pragma unroll
                 for (int q = 0; q < NW / 4; ++q) {
                     // words 4q .. 4q+3 of the run: k-steps 2q (x, y) and 2q + 1 (z, w)
                     mma_bf16_top(cl, ql[4 * q], ql[4 * q + 1], kq[q].x, kq[q].y);
-                    mma_bf16_top(cm, qm[4 * q], qm[4 * q + 1], kq[q].x, kq[q].y);
                     mma_bf16_top(ch, qh[4 * q], qh[4 * q + 1], kq[q].x, kq[q].y);
                     mma_bf16_top(cl, ql[4 * q + 2], ql[4 * q + 3], kq[q].z, kq[q].w);
-                    mma_bf16_top(cm, qm[4 * q + 2], qm[4 * q + 3], kq[q].z, kq[q].w);
                     mma_bf16_top(ch, qh[4 * q + 2], qh[4 * q + 3], kq[q].z, kq[q].w);
                 }
-                sc[nt][0] = (cl[0] + cm[0]) + ch[0];
-                sc[nt][1] = (cl[1] + cm[1]) + ch[1];
+                sc[nt][0] = cl[0] + ch[0];
+                sc[nt][1] = cl[1] + ch[1];
                 if (nt + KR < NT) load_k(nt + KR, kq);
             }
         }
@@ -485,22 +484,32 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
 #pragma unroll
         for (int j = 0; j < VJ; ++j) { o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f; }
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-            const uint32_t p0h = __float_as_uint(sc[nt][0]) & 0xFFFFE000u, p1h = __float_as_uint(sc[nt][1]) & 0xFFFFE000u;
-            const uint32_t p0l = __float_as_uint(sc[nt][0] - __uint_as_float(p0h)) & 0xFFFFE000u;
-            const uint32_t p1l = __float_as_uint(sc[nt][1] - __uint_as_float(p1h)) & 0xFFFFE000u;
+        for (int np = 0; np < NT; np += 2) {
+            // k-indices 2t4, 2t4+1 stand for this lane's two positions of tile np, 2t4+8, 2t4+9 for those of tile np + 1
+            uint32_t ah[2], al[2];
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                const uint32_t h0 = float_to_bf16_rne(sc[np + i][0]), h1 = float_to_bf16_rne(sc[np + i][1]);
+                const uint32_t l0 = float_to_bf16_rne(sc[np + i][0] - __uint_as_float(h0 << 16));
+                const uint32_t l1 = float_to_bf16_rne(sc[np + i][1] - __uint_as_float(h1 << 16));
+                ah[i] = h0 | (h1 << 16); al[i] = l0 | (l1 << 16);
+            }
 #pragma unroll
             for (int j = 0; j < VJ; ++j) {
-                const uint4 &wa = vb[nt % VR][0][j / 8], &wb = vb[nt % VR][1][j / 8];
                 const int wi = (j >> 1) & 3;
-                const uint32_t xa = wi == 0 ? wa.x : wi == 1 ? wa.y : wi == 2 ? wa.z : wa.w;
-                const uint32_t xb = wi == 0 ? wb.x : wi == 1 ? wb.y : wi == 2 ? wb.z : wb.w;
-                const uint32_t b0 = (j & 1) ? (xa & 0xFFFF0000u) : (xa << 16);
-                const uint32_t b1 = (j & 1) ? (xb & 0xFFFF0000u) : (xb << 16);
-                mma_tf32(o[j], p0l, p1l, b0, b1);
-                mma_tf32(o[j], p0h, p1h, b0, b1);
+                uint32_t b[2];
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+                    const uint4 &wa = vb[(np + i) % VR][0][j / 8], &wb = vb[(np + i) % VR][1][j / 8];
+                    const uint32_t xa = wi == 0 ? wa.x : wi == 1 ? wa.y : wi == 2 ? wa.z : wa.w;
+                    const uint32_t xb = wi == 0 ? wb.x : wi == 1 ? wb.y : wi == 2 ? wb.z : wb.w;
+                    b[i] = __byte_perm(xa, xb, (j & 1) ? 0x7632 : 0x5410);     // dimension j of the two positions' rows
+                }
+                mma_bf16_top(o[j], al[0], al[1], b[0], b[1]);
+                mma_bf16_top(o[j], ah[0], ah[1], b[0], b[1]);
             }
-            if (nt + VR < NT) load_v(nt + VR, vb[nt % VR]);
+            if (np + VR < NT) load_v(np + VR, vb[np % VR]);
+            if (np + 1 + VR < NT) load_v(np + 1 + VR, vb[(np + 1) % VR]);
         }
 
         KNNSSD_ATT_STAMP(5);
