@@ -1,10 +1,13 @@
 // Consumer half of the weight-streaming linear engine for PRE-SPLIT activations (persistent pass kernel).
 //
 // Same ring, same tiles, same sum order per output as consume_linear, but the activation operand arrives already
-// split into its three bf16 terms and laid out fragment by fragment (LinPhase::xs), written once by whoever produced
-// the activation.  The consumer therefore spends no arithmetic on the split that every CTA would otherwise repeat:
-// per column tile a lane loads four 16-byte pieces per term, one tile ahead of the tensor-core work.  RMSNorm's scalar comes
-// from per-CTA partial sums of squares that the producer of the row left in LinPhase::ss_in.
+// split into its bf16 terms and laid out fragment by fragment (LinPhase::xs), written once by whoever produced the
+// activation.  The consumer therefore spends no arithmetic on the split that every CTA would otherwise repeat:
+// per column tile a lane loads four 16-byte pieces per term and row block, one tile ahead of the tensor-core work.
+// RMSNorm's scalar comes from per-CTA partial sums of squares that the producer of the row left in LinPhase::ss_in.
+//
+// NB = row blocks of eight: 1 for passes of up to 8 rows, 2 for 9..16 rows (the second block is a second 8-column
+// operand for the same weight fragments; every row is computed exactly as it would be in a one-row pass).
 //
 // The epilogue writes what the NEXT map needs: the fp32 result where something reads it as fp32 (projection buffer,
 // residual stream, logits) and, for the residual update and the SwiGLU product, the pre-split form (times the next
@@ -17,6 +20,7 @@ namespace stream {
 
 __device__ __forceinline__ uint4 ld_frag4(const uint32_t *p) { return __ldcg(reinterpret_cast<const uint4 *>(p)); }
 
+template <int NB>
 __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring &r, int cta, int n_cta, int warp, int lane,
                                                    int &w_use, bool &alive) {
     const Share s = make_share(p, cta, n_cta);
@@ -24,45 +28,64 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
     const int g8 = lane >> 2, t4 = lane & 3;
     const int lm_row = (lane & 7) + ((lane >> 3) & 1) * 8, lm_col = (lane >> 4) * 8;   // ldmatrix source of this lane
     const bool normed = p.ss_in != nullptr;
-    const bool row_live = g8 < p.M;
     const int nslots = p.K >> 7;
-    // this lane's 16-byte pieces: row g8, lane group t4; + slot * SLOT_WORDS + term * 64 + piece * 16
-    const uint32_t *xsrow = p.xs + (size_t)min(g8, p.M - 1) * nslots * SLOT_WORDS + t4 * 4;
+    // this lane's 16-byte pieces: row nb*8 + g8, lane group t4; + slot * SLOT_WORDS + term * 64 + piece * 16
+    const uint32_t *xsrow[NB];
+    bool row_live[NB];
+#pragma unroll
+    for (int nb = 0; nb < NB; ++nb) {
+        row_live[nb] = nb * 8 + g8 < p.M;
+        xsrow[nb] = p.xs + (size_t)min(nb * 8 + g8, p.M - 1) * nslots * SLOT_WORDS + t4 * 4;
+    }
     int ws = w_use % WS, it = w_use / WS;
     float *red = r.red, *red_ss = r.red_ss;
 
-    float ss_acc = 0.f;                                     // lane 0 of warp n (n < M): this CTA's sum of squares of y row n
+    float ss_acc[NB];                                       // lane 0 of warp w: this CTA's sum of squares of y rows w, w + 8
+#pragma unroll
+    for (int nb = 0; nb < NB; ++nb) ss_acc[nb] = 0.f;
 
     for (int b = 0; b < s.n_batches; ++b) {
         const int g0 = b * GB, ng = min(s.n_groups - g0, GB);
-        float acc[GB][4];
+        float acc[GB][NB][4];
 #pragma unroll
-        for (int i = 0; i < GB; ++i) { acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f; }
-        uint4 nx[NTERM][4];                                  // fragments of the next column tile, term by term
+        for (int i = 0; i < GB; ++i)
+#pragma unroll
+            for (int nb = 0; nb < NB; ++nb) { acc[i][nb][0] = acc[i][nb][1] = acc[i][nb][2] = acc[i][nb][3] = 0.f; }
+        uint4 nx[NB][NTERM][4];                              // fragments of the next column tile, block by block, term by term
         auto fetch = [&](int kt) {
             const int slot = kt * NCW + warp;
-            const bool ld = alive && row_live && slot < nslots;
 #pragma unroll
-            for (int t = 0; t < NTERM; ++t)
+            for (int nb = 0; nb < NB; ++nb) {
+                const bool ld = alive && row_live[nb] && slot < nslots;
 #pragma unroll
-                for (int q = 0; q < 4; ++q)
-                    nx[t][q] = ld ? ld_frag4(xsrow + (size_t)slot * SLOT_WORDS + t * 64 + q * 16) : make_uint4(0u, 0u, 0u, 0u);
+                for (int t = 0; t < NTERM; ++t)
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        nx[nb][t][q] = ld ? ld_frag4(xsrow[nb] + (size_t)slot * SLOT_WORDS + t * 64 + q * 16) : make_uint4(0u, 0u, 0u, 0u);
+            }
         };
         fetch(0);
-        if (b == 0 && normed && warp < p.M) {
-            // RMSNorm scalar of row `warp` from the producers' partial sums (lanes take CTAs lane, lane + 32, ...); issued
-            // after the first fragment fetch so that both round trips to L2 overlap
-            float tot = 0.f;
-            for (int c = lane; c < n_cta; c += 32) tot += __ldcg(p.ss_in + (size_t)warp * n_cta + c);
-            tot = warp_sum(tot);
-            if (lane == 0) red_ss[warp] = 1.0f / sqrtf(tot / (float)p.K + p.eps);
+        if (b == 0 && normed) {
+            // RMSNorm scalar of rows `warp` (and warp + 8) from the producers' partial sums (lanes take CTAs lane,
+            // lane + 32, ...); issued after the first fragment fetch so that both round trips to L2 overlap
+#pragma unroll
+            for (int nb = 0; nb < NB; ++nb) {
+                const int row = nb * 8 + warp;
+                if (row < p.M) {
+                    float tot = 0.f;
+                    for (int c = lane; c < n_cta; c += 32) tot += __ldcg(p.ss_in + (size_t)row * n_cta + c);
+                    tot = warp_sum(tot);
+                    if (lane == 0) red_ss[row] = 1.0f / sqrtf(tot / (float)p.K + p.eps);
+                }
+            }
         }
         // this thread's epilogue items: (unit, token) pairs, token fastest among the M live tokens.  For a residual
         // update the old value and the next gain are fetched now, long before the epilogue needs them.
         const int gshift = s.swiglu ? 3 : 4, total = (ng << gshift) * p.M;
-        float xold[4], gnext[4];
+        constexpr int ITEMS = GB * 16 * 8 * NB / (NCW * 32);
+        float xold[ITEMS], gnext[ITEMS];
 #pragma unroll
-        for (int it4 = 0; it4 < 4; ++it4) {
+        for (int it4 = 0; it4 < ITEMS; ++it4) {
             xold[it4] = 0.f; gnext[it4] = 1.f;
             const int idx = tid + it4 * (NCW * 32);
             if (p.epi == EPI_ADD && alive && idx < total) {
@@ -76,14 +99,16 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
         }
         for (int kt = 0; kt < s.n_kt; ++kt) {
             const bool slot_valid = kt * NCW + warp < nslots;
-            uint32_t bf[NTERM][KSTEPS][2];                    // operand registers: term, k-step, (b0, b1)
+            uint32_t bf[NB][NTERM][KSTEPS][2];                // operand registers: block, term, k-step, (b0, b1)
 #pragma unroll
-            for (int t = 0; t < NTERM; ++t)
+            for (int nb = 0; nb < NB; ++nb)
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    bf[t][2 * q][0] = nx[t][q].x; bf[t][2 * q][1] = nx[t][q].y;
-                    bf[t][2 * q + 1][0] = nx[t][q].z; bf[t][2 * q + 1][1] = nx[t][q].w;
-                }
+                for (int t = 0; t < NTERM; ++t)
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        bf[nb][t][2 * q][0] = nx[nb][t][q].x; bf[nb][t][2 * q][1] = nx[nb][t][q].y;
+                        bf[nb][t][2 * q + 1][0] = nx[nb][t][q].z; bf[nb][t][2 * q + 1][1] = nx[nb][t][q].w;
+                    }
             if (kt + 1 < s.n_kt) fetch(kt + 1);
 #pragma unroll
             for (int gi = 0; gi < GB; ++gi) {
@@ -91,22 +116,27 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
                 if (alive) alive = mbar_wait(&r.full_w[ws], it & 1, r.abort_flag, r.err, 5);
                 if (alive && slot_valid) {
                     const uint32_t base = smem_u32(r.wring + ws * WSTAGE) + lm_row * WPITCH + (warp * SLOT + lm_col) * 2;
-                    // independent accumulator chains: term x parity of the k-step; smallest terms are added first
-                    float tc[NTERM][2][4] = {};
+                    // independent accumulator chains: block x term x parity of the k-step; smallest terms are added first
+                    float tc[NB][NTERM][2][4] = {};
 #pragma unroll
                     for (int j = 0; j < KSTEPS; ++j) {
                         uint32_t a0, a1, a2, a3;
                         ldmatrix_x4(base + j * 32, a0, a1, a2, a3);
 #pragma unroll
-                        for (int t = NTERM - 1; t >= 0; --t) mma_bf16(tc[t][j & 1], a0, a1, a2, a3, bf[t][j][0], bf[t][j][1]);
+                        for (int nb = 0; nb < NB; ++nb)
+#pragma unroll
+                            for (int t = NTERM - 1; t >= 0; --t)
+                                mma_bf16(tc[nb][t][j & 1], a0, a1, a2, a3, bf[nb][t][j][0], bf[nb][t][j][1]);
                     }
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        float sum = tc[NTERM - 1][0][e] + tc[NTERM - 1][1][e];
+                    for (int nb = 0; nb < NB; ++nb)
 #pragma unroll
-                        for (int t = NTERM - 2; t >= 0; --t) sum += tc[t][0][e] + tc[t][1][e];
-                        acc[gi][e] += sum;
-                    }
+                        for (int e = 0; e < 4; ++e) {
+                            float sum = tc[nb][NTERM - 1][0][e] + tc[nb][NTERM - 1][1][e];
+#pragma unroll
+                            for (int t = NTERM - 2; t >= 0; --t) sum += tc[nb][t][0][e] + tc[nb][t][1][e];
+                            acc[gi][nb][e] += sum;
+                        }
                 }
                 __syncwarp();
                 if (alive && lane == 0) mbar_arrive(&r.empty_w[ws]);
@@ -117,23 +147,26 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
         // ---- batch end: partial sums of the 8 column slots meet in shared memory, in warp order ----
 #pragma unroll
         for (int gi = 0; gi < GB; ++gi)
-            *reinterpret_cast<float4 *>(red + ((warp * GB + gi) * 32 + lane) * 4) =
-                make_float4(acc[gi][0], acc[gi][1], acc[gi][2], acc[gi][3]);
+#pragma unroll
+            for (int nb = 0; nb < NB; ++nb)
+                *reinterpret_cast<float4 *>(red + ((((warp * GB + gi) * NB + nb) * 32) + lane) * 4) =
+                    make_float4(acc[gi][nb][0], acc[gi][nb][1], acc[gi][nb][2], acc[gi][nb][3]);
         asm volatile("bar.sync 1, %0;" ::"n"(NCW * 32) : "memory");
         if (alive) {
 #pragma unroll
-            for (int it4 = 0; it4 < 4; ++it4) {
+            for (int it4 = 0; it4 < ITEMS; ++it4) {
                 const int idx = tid + it4 * (NCW * 32);
                 if (idx >= total) break;
                 const int n = idx % p.M, ur = idx / p.M, gi = ur >> gshift, rr = ur & ((1 << gshift) - 1);
                 if (rr >= s.group_size(g0 + gi)) continue;
-                // rows 0..7 of the tile: regs 0,1; rows 8..15: regs 2,3
-                const int src_lane = (rr & 7) * 4 + (n >> 1), reg = n & 1;
+                // token n sits in block n / 8, column n % 8; rows 0..7 of the tile: regs 0,1; rows 8..15: regs 2,3
+                const int nb = n >> 3, n8 = n & 7;
+                const int src_lane = (rr & 7) * 4 + (n8 >> 1), reg = n8 & 1;
                 const int e0 = s.swiglu ? reg : (rr >> 3) * 2 + reg;
                 float s0 = 0.f, s1 = 0.f;
 #pragma unroll
                 for (int w = 0; w < NCW; ++w) {
-                    const float *q = red + ((w * GB + gi) * 32 + src_lane) * 4;
+                    const float *q = red + ((((w * GB + gi) * NB + nb) * 32) + src_lane) * 4;
                     s0 += q[e0];
                     if (s.swiglu) s1 += q[2 + reg];
                 }
@@ -148,8 +181,8 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
                     const float v = xold[it4] + s0 * ri;
                     __stcg(yp, v);
                     if (p.ys) store_split(p.ys, p.units >> 7, n, u, v * gnext[it4]);
-                    // leave v^2 where this thread alone read its first partial: warp n adds them up below
-                    red[((0 * GB + gi) * 32 + src_lane) * 4 + e0] = v * v;
+                    // leave v^2 where this thread alone read its first partial: warp n % 8 adds them up below
+                    red[((((0 * GB + gi) * NB + nb) * 32) + src_lane) * 4 + e0] = v * v;
                 } else {
                     __stcg(yp, s0 * ri);
                 }
@@ -157,21 +190,29 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
         }
         if (p.ss_out) {
             asm volatile("bar.sync 1, %0;" ::"n"(NCW * 32) : "memory");
-            if (alive && warp < p.M) {
-                const int n = warp;
-                float part = 0.f;
-                for (int i = lane; i < (ng << gshift); i += 32) {
-                    const int gi = i >> gshift, rr = i & ((1 << gshift) - 1);
-                    if (rr < s.group_size(g0 + gi))
-                        part += red[((0 * GB + gi) * 32 + (rr & 7) * 4 + (n >> 1)) * 4 + (rr >> 3) * 2 + (n & 1)];
+            if (alive) {
+#pragma unroll
+                for (int nb = 0; nb < NB; ++nb) {
+                    if (nb * 8 + warp >= p.M) continue;
+                    const int n8 = warp;
+                    float part = 0.f;
+                    for (int i = lane; i < (ng << gshift); i += 32) {
+                        const int gi = i >> gshift, rr = i & ((1 << gshift) - 1);
+                        if (rr < s.group_size(g0 + gi))
+                            part += red[((((0 * GB + gi) * NB + nb) * 32) + (rr & 7) * 4 + (n8 >> 1)) * 4 + (rr >> 3) * 2 + (n8 & 1)];
+                    }
+                    part = warp_sum(part);
+                    ss_acc[nb] += part;
                 }
-                part = warp_sum(part);
-                ss_acc += part;
             }
         }
         asm volatile("bar.sync 1, %0;" ::"n"(NCW * 32) : "memory");
     }
-    if (p.ss_out && alive && warp < p.M && lane == 0) __stcg(p.ss_out + (size_t)warp * n_cta + cta, ss_acc);
+    if (p.ss_out && alive && lane == 0) {
+#pragma unroll
+        for (int nb = 0; nb < NB; ++nb)
+            if (nb * 8 + warp < p.M) __stcg(p.ss_out + (size_t)(nb * 8 + warp) * n_cta + cta, ss_acc[nb]);
+    }
 }
 
 }  // namespace stream

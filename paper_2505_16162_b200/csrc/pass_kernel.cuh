@@ -598,7 +598,7 @@ __global__ void __launch_bounds__(stream::NTHREADS, 1) pass_kernel(const Model m
                 lp.ss_in += (size_t)pr.head_row0 * n_cta;
                 lp.y += (size_t)(pr.out_row0 + pr.head_row0) * lp.units;
             }
-            if (ran) stream::consume_linear_pre(lp, r, cta, n_cta, warp, lane, w_use, alive);
+            if (ran) stream::consume_linear_pre<1>(lp, r, cta, n_cta, warp, lane, w_use, alive);
         } else if (alive) {
             if (op.type == OP_EMBED) embed_phase(md, op, pr, r, cta, n_cta, tid);
             else if (op.type == OP_ATTN) attn_phase<HD>(md, op, pr, r, cta, n_cta, warp, lane, pr.M >= MERGE_ROWS);
