@@ -217,6 +217,11 @@ std::vector<pass::Op> build_ops(const knnssd_ctx *c, const unsigned char *mask, 
             q.lin.units = nq + 2 * nkv; q.layer = l;
             q.lin.xs = c->xs_x; q.lin.ss_in = c->ssp;
             ops.push_back(q);
+            pass::Op ap{};                               // runs (and its barrier counts) only in passes of > BLKM rows
+            ap.type = pass::OP_KV_APPEND; ap.barrier_after = 1; ap.layer = l;
+            ap.kc = reinterpret_cast<bf16_t *>(c->kcache) + (size_t)l * layer_stride;
+            ap.vc = reinterpret_cast<bf16_t *>(c->vcache) + (size_t)l * layer_stride;
+            ops.push_back(ap);
             pass::Op a{};
             a.type = pass::OP_ATTN; a.barrier_after = 1; a.layer = l;
             a.kc = reinterpret_cast<bf16_t *>(c->kcache) + (size_t)l * layer_stride;
@@ -274,15 +279,15 @@ knnssd_status upload_ops(knnssd_ctx *c, const std::vector<pass::Op> &ops, pass::
     return KNNSSD_OK;
 }
 
-template <int HD> cudaError_t launch_pass_t(knnssd_ctx *c, const pass::Params &pr) {
+template <int HD, int NB> cudaError_t launch_pass_t(knnssd_ctx *c, const pass::Params &pr) {
     static bool configured = false;
     if (!configured) {
-        cudaFuncSetAttribute(pass::pass_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, stream::SMEM_BYTES);
+        cudaFuncSetAttribute(pass::pass_kernel<HD, NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, stream::SMEM_BYTES);
         configured = true;
     }
     void *args[] = {const_cast<pass::Model *>(&c->model), const_cast<pass::Params *>(&pr)};
-    return cudaLaunchCooperativeKernel(reinterpret_cast<void *>(pass::pass_kernel<HD>), dim3(c->n_sms), dim3(stream::NTHREADS),
-                                       args, stream::SMEM_BYTES, c->stream);
+    return cudaLaunchCooperativeKernel(reinterpret_cast<void *>(pass::pass_kernel<HD, NB>), dim3(c->n_sms),
+                                       dim3(stream::NTHREADS), args, stream::SMEM_BYTES, c->stream);
 }
 
 // One pass through the persistent kernel.  Errors surface at the caller's next synchronisation.
@@ -308,7 +313,10 @@ void run_pass_mega(knnssd_ctx *c, int M, const int *tok_dev, int pos_off, const 
     pr.bar_base = c->bar_total;
     if (head_row0 < M) bars += 1;
     if (M >= pass::MERGE_ROWS) bars += n_attn;
-    const cudaError_t e = c->cfg.head_dim == 128 ? launch_pass_t<128>(c, pr) : launch_pass_t<64>(c, pr);
+    if (M > pass::BLKM) bars += n_attn;
+    cudaError_t e;
+    if (M > pass::BLKM) e = c->cfg.head_dim == 128 ? launch_pass_t<128, 2>(c, pr) : launch_pass_t<64, 2>(c, pr);
+    else e = c->cfg.head_dim == 128 ? launch_pass_t<128, 1>(c, pr) : launch_pass_t<64, 1>(c, pr);
     if (e == cudaSuccess) c->bar_total += (unsigned long long)bars * (unsigned long long)c->n_sms;
     c->launches++;
 }
@@ -389,14 +397,6 @@ void run_pass_t(knnssd_ctx *c, int M, const int *tok_dev, int pos_off, const uns
 void run_pass(knnssd_ctx *c, int M, const int *tok_dev, int pos_off, const unsigned char *mask, int head_row0,
               int *argmax_out, bool want_hidden) {
     if (c->mega_ok && M <= pass::MAXM) { run_pass_mega(c, M, tok_dev, pos_off, mask, head_row0, argmax_out, want_hidden); return; }
-    if (c->mega_ok && M <= 2 * pass::MAXM) {
-        // more rows than one launch of the persistent kernel carries: rows 0..7 first, then the rest as a second pass
-        // whose rows sit 8 positions further on (it finds the first eight rows' K/V in the cache like any earlier row)
-        const int A = pass::MAXM, hrA = head_row0 < A ? head_row0 : A, hrB = head_row0 > A ? head_row0 - A : 0;
-        run_pass_mega(c, A, tok_dev, pos_off, mask, hrA, argmax_out, want_hidden, 0);
-        run_pass_mega(c, M - A, tok_dev + A, pos_off + A, mask, hrB, argmax_out + (A + hrB - head_row0), want_hidden, A);
-        return;
-    }
     if (c->cfg.dtype) run_pass_t<bf16_t>(c, M, tok_dev, pos_off, mask, head_row0, argmax_out, want_hidden);
     else run_pass_t<float>(c, M, tok_dev, pos_off, mask, head_row0, argmax_out, want_hidden);
 }
@@ -637,7 +637,7 @@ knnssd_status knnssd_init(const knnssd_config *cfg, const knnssd_weights *w, con
     if (g.dtype == 1 && coop && d % 128 == 0 && nq % 128 == 0 && g.d_ff % 128 == 0 && d >= 256 && nq >= 256 && g.d_ff >= 256 &&
         g.max_seq <= 64 * pass::SEGP) {            // the attention merge keeps at most 64 segment statistics per warp
         const int n_seg_max = (g.max_seq + pass::SEGP - 1) / pass::SEGP;
-        const int n_ops_cap = 6 * g.n_layers + 8;
+        const int n_ops_cap = 7 * g.n_layers + 8;
         bool ok2 = true;
         ok2 &= dev_alloc(&c->ops_full, (size_t)n_ops_cap) == cudaSuccess;
         ok2 &= dev_alloc(&c->ops_draft, (size_t)n_ops_cap) == cudaSuccess;

@@ -23,11 +23,12 @@ using stream::LinPhase;
 using stream::Ring;
 using stream::NCW;
 
-constexpr int MAXM = 8;            // rows per pass this kernel handles
+constexpr int MAXM = 16;           // rows per pass this kernel handles
+constexpr int BLKM = 8;            // rows per tensor-core row block (linear maps take two blocks at once, attention one at a time)
 constexpr int SEGP = 64;           // attention: positions per segment (fixed absolute boundaries)
 constexpr unsigned BAR_SPIN_LIMIT = 4000000u;
 
-enum { OP_EMBED = 0, OP_LINEAR = 1, OP_ATTN = 2, OP_HIDDEN = 3, OP_ARGMAX = 4, OP_ATTN_MERGE = 5 };
+enum { OP_EMBED = 0, OP_LINEAR = 1, OP_ATTN = 2, OP_HIDDEN = 3, OP_ARGMAX = 4, OP_ATTN_MERGE = 5, OP_KV_APPEND = 6 };
 constexpr int MERGE_ROWS = 3;      // passes with at least this many rows merge attention partials in a separate operation
 
 struct Op {
@@ -314,7 +315,7 @@ __device__ __forceinline__ void attn_merge_row(const Model &md, const Op &op, in
 // A lane ends up with output dimensions [DL*t4, DL*t4 + DL) of row g8, the run it holds of q.
 template <int HD>
 __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const Params &pr, const Ring &r, int cta, int n_cta,
-                                           int warp, int lane, bool defer_merge) {
+                                           int warp, int lane, bool defer_merge, int row0, bool all_cached) {
     constexpr int DL = HD / 4;         // dimensions of q / o per lane
     constexpr int NW = HD / 8;         // 32-bit words of a K row per lane
     constexpr int KS = HD / 16;        // k-steps of Q K^T
@@ -325,13 +326,15 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
     const int g8 = lane >> 2, t4 = lane & 3;
     const int M = pr.M, H = md.H, Hkv = md.Hkv, G = H / Hkv;
     const int P0 = md.state->len + pr.pos_off, Ttot = P0 + M;
+    const int Pc = all_cached ? Ttot : P0;                   // positions below Pc are read from the cache
+    const int rm = row0 + g8;                                // the pass row this lane's MMA row stands for
     const int n_seg = (Ttot + SEGP - 1) / SEGP, n_tasks = H * n_seg;
     const int qstride = (H + 2 * Hkv) * HD;
     const float scale = 1.0f / sqrtf((float)HD);
     const bool upper = t4 >= 2;                              // this lane's run lies in the second half of the head
     const int ci = DL * (t4 & 1);                            // its offset in the (cos, sin) table
-    bf16_t *stash_k = reinterpret_cast<bf16_t *>(r.red) + (size_t)warp * (2 * MAXM * HD);   // [MAXM][HD] new K rows
-    bf16_t *stash_v = stash_k + MAXM * HD;                                                  // [MAXM][HD] new V rows
+    bf16_t *stash_k = reinterpret_cast<bf16_t *>(r.red) + (size_t)warp * (2 * BLKM * HD);   // [BLKM][HD] new K rows
+    bf16_t *stash_v = stash_k + BLKM * HD;                                                  // [BLKM][HD] new V rows
     const float2 *my_cs = md.rope_cs + (size_t)cta * MAXM * HALF;                           // this CTA's copy
 
     for (int t = warp * n_cta + cta; t < n_tasks; t += NCW * n_cta) {
@@ -341,15 +344,17 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
         const bool writer = (h % G) == 0;
         bf16_t *kbase = op.kc + (size_t)kvh * md.max_seq * HD;
         bf16_t *vbase = op.vc + (size_t)kvh * md.max_seq * HD;
-        const bool row_new = g8 < M && P0 + g8 >= p_begin && P0 + g8 < p_end;   // row g8's own position lies in this segment
-        const bool row_live = g8 < M && g8 >= m_first;
+        if (row0 + BLKM <= m_first) continue;               // none of this block's rows sees the segment
+        // row rm's own position lies in this segment and is not in the cache yet
+        const bool row_new = !all_cached && rm < M && P0 + rm >= p_begin && P0 + rm < p_end;
+        const bool row_live = rm < M && rm >= m_first;
 
         KNNSSD_ATT_STAMP(0);
         // ---- this lane's run of q (row g8), of the new K row and of the new V row: load, rotate, round / split ----
         float qf[DL], kf[DL];
         {
-            const float *qraw = md.qkv + (size_t)min(g8, M - 1) * qstride + (size_t)h * HD + DL * t4;
-            const float *kraw = md.qkv + (size_t)min(g8, M - 1) * qstride + (size_t)(H + kvh) * HD + DL * t4;
+            const float *qraw = md.qkv + (size_t)min(rm, M - 1) * qstride + (size_t)h * HD + DL * t4;
+            const float *kraw = md.qkv + (size_t)min(rm, M - 1) * qstride + (size_t)(H + kvh) * HD + DL * t4;
 #pragma unroll
             for (int e = 0; e < DL; e += 4) {
                 const float4 a = row_live ? __ldcg(reinterpret_cast<const float4 *>(qraw + e)) : make_float4(0.f, 0.f, 0.f, 0.f);
@@ -360,14 +365,14 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
 #pragma unroll
             for (int e = 0; e < DL; ++e) {
                 const float qp = __shfl_xor_sync(0xffffffffu, qf[e], 2), kp = __shfl_xor_sync(0xffffffffu, kf[e], 2);
-                const float2 cs = (row_live || row_new) ? my_cs[g8 * HALF + ci + e] : make_float2(1.f, 0.f);
+                const float2 cs = (row_live || row_new) ? my_cs[rm * HALF + ci + e] : make_float2(1.f, 0.f);
                 qf[e] = upper ? (qf[e] * cs.x + qp * cs.y) : (qf[e] * cs.x - qp * cs.y);
                 kf[e] = upper ? (kf[e] * cs.x + kp * cs.y) : (kf[e] * cs.x - kp * cs.y);
             }
         }
         __syncwarp();
         if (row_new) {
-            const float *vraw = md.qkv + (size_t)g8 * qstride + (size_t)(H + Hkv + kvh) * HD + DL * t4;
+            const float *vraw = md.qkv + (size_t)rm * qstride + (size_t)(H + Hkv + kvh) * HD + DL * t4;
 #pragma unroll
             for (int e = 0; e < DL; e += 8) {
                 const float4 a = __ldcg(reinterpret_cast<const float4 *>(vraw + e)), b = __ldcg(reinterpret_cast<const float4 *>(vraw + e + 4));
@@ -402,7 +407,7 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
         // ---- scores: one tile = 8 positions; K rows are fetched two tiles ahead ----
         auto load_k = [&](int nt, uint4 (&dst)[NW / 4]) {
             const int p = p_begin + 8 * nt + g8;
-            const bf16_t *src = p < P0 ? kbase + (size_t)p * HD + DL * t4 : stash_k + (p - P0) * HD + DL * t4;
+            const bf16_t *src = p < Pc ? kbase + (size_t)p * HD + DL * t4 : stash_k + (p - P0) * HD + DL * t4;
 #pragma unroll
             for (int q = 0; q < NW / 4; ++q)
                 dst[q] = p < p_end ? *reinterpret_cast<const uint4 *>(src + 8 * q) : make_uint4(0u, 0u, 0u, 0u);
@@ -436,7 +441,7 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
 #pragma unroll
             for (int rr = 0; rr < 2; ++rr) {
                 const int p = p_begin + 8 * nt + 2 * t4 + rr;
-                const bf16_t *src = p < P0 ? vbase + (size_t)p * HD + 2 * VW * g8 : stash_v + (p - P0) * HD + 2 * VW * g8;
+                const bf16_t *src = p < Pc ? vbase + (size_t)p * HD + 2 * VW * g8 : stash_v + (p - P0) * HD + 2 * VW * g8;
                 if (VW >= 4) {
 #pragma unroll
                     for (int q = 0; q < VW / 4; ++q)
@@ -460,7 +465,7 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
                 const int p = p_begin + 8 * nt + 2 * t4 + e;
-                const bool valid = row_live && p <= P0 + g8;             // causal; also excludes p >= p_end
+                const bool valid = row_live && p <= P0 + rm;             // causal; also excludes p >= p_end
                 sc[nt][e] = valid ? sc[nt][e] * scale : -INFINITY;
                 mx = fmaxf(mx, sc[nt][e]);
             }
@@ -515,7 +520,7 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
         KNNSSD_ATT_STAMP(5);
         // ---- partials out (row g8: dimensions DL*t4 + j and DL*t4 + VJ + j); the last warp of a (row, head) merges ----
         if (row_live) {
-            const size_t pidx = ((size_t)g8 * H + h) * md.n_seg_max + seg;
+            const size_t pidx = ((size_t)rm * H + h) * md.n_seg_max + seg;
             if (t4 == 0) __stcg(md.part_ml + pidx, make_float2(mx, lsum));
             float *po = md.part_o + pidx * HD + DL * t4;
 #pragma unroll
@@ -530,8 +535,8 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
         KNNSSD_ATT_STAMP(6);
         bool last = false;
         if (row_live && t4 == 0) {
-            const int n_seg_m = (P0 + g8 + SEGP) / SEGP;                  // segments row g8 sees
-            last = atomicAdd(md.attn_cnt + g8 * H + h, 1) == n_seg_m - 1;
+            const int n_seg_m = (P0 + rm + SEGP) / SEGP;                  // segments row rm sees
+            last = atomicAdd(md.attn_cnt + rm * H + h, 1) == n_seg_m - 1;
         }
         KNNSSD_ATT_STAMP(7);
         const unsigned last_mask = __ballot_sync(0xffffffffu, last);     // bit 4*m set: this warp finishes (row m, head h)
@@ -547,6 +552,36 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
     }
 }
 
+// Passes of more than BLKM rows first put the K/V rows of all their new positions into the cache (rotated, rounded),
+// one (row, KV head) per warp, so that the attention operation - which then takes the rows one block at a time - reads
+// every position from the cache.  Lane l holds dimensions [DPL*l, DPL*l + DPL); its rotation partner is lane l ^ 16.
+template <int HD>
+__device__ __forceinline__ void kv_append_phase(const Model &md, const Op &op, const Params &pr, int cta, int n_cta, int warp,
+                                                int lane) {
+    constexpr int DPL = HD / 32, HALF = HD / 2;
+    typedef typename KVVec<HD>::T VT;
+    const int H = md.H, Hkv = md.Hkv, P0 = md.state->len + pr.pos_off, jobs = pr.M * Hkv;
+    const int qstride = (H + 2 * Hkv) * HD, d0 = DPL * lane, ci = d0 % HALF;
+    const bool upper = d0 >= HALF;
+    const float2 *my_cs = md.rope_cs + (size_t)cta * MAXM * HALF;
+    for (int j = warp * n_cta + cta; j < jobs; j += NCW * n_cta) {
+        const int m = j / Hkv, kvh = j % Hkv;
+        const float *kraw = md.qkv + (size_t)m * qstride + (size_t)(H + kvh) * HD + d0;
+        const float *vraw = md.qkv + (size_t)m * qstride + (size_t)(H + Hkv + kvh) * HD + d0;
+        float kf[DPL], vf[DPL];
+#pragma unroll
+        for (int e = 0; e < DPL; ++e) { kf[e] = __ldcg(kraw + e); vf[e] = __ldcg(vraw + e); }
+#pragma unroll
+        for (int e = 0; e < DPL; ++e) {
+            const float partner = __shfl_xor_sync(0xffffffffu, kf[e], 16);
+            const float2 cs = my_cs[m * HALF + ci + e];
+            kf[e] = upper ? (kf[e] * cs.x + partner * cs.y) : (kf[e] * cs.x - partner * cs.y);
+        }
+        *reinterpret_cast<VT *>(op.kc + ((size_t)kvh * md.max_seq + P0 + m) * HD + d0) = kv_pack<HD>(kf);
+        *reinterpret_cast<VT *>(op.vc + ((size_t)kvh * md.max_seq + P0 + m) * HD + d0) = kv_pack<HD>(vf);
+    }
+}
+
 // With several rows the warp that finishes a head last would merge all its rows one after the other; the merges
 // then run as an operation of their own instead, one (row, head) per warp across the whole grid.
 template <int HD>
@@ -557,7 +592,8 @@ __device__ __forceinline__ void attn_merge_phase(const Model &md, const Op &op, 
 }
 
 // ---- the pass ---------------------------------------------------------------------------------------------------
-template <int HD>
+// NB = 1: passes of up to BLKM rows; NB = 2: 9..16 rows (a kernel of its own, so that the common one stays small).
+template <int HD, int NB>
 __global__ void __launch_bounds__(stream::NTHREADS, 1) pass_kernel(const Model md, const Params pr) {
     extern __shared__ __align__(128) unsigned char smem[];
     Ring r;
@@ -598,10 +634,17 @@ __global__ void __launch_bounds__(stream::NTHREADS, 1) pass_kernel(const Model m
                 lp.ss_in += (size_t)pr.head_row0 * n_cta;
                 lp.y += (size_t)(pr.out_row0 + pr.head_row0) * lp.units;
             }
-            if (ran) stream::consume_linear_pre<1>(lp, r, cta, n_cta, warp, lane, w_use, alive);
+            if (ran) stream::consume_linear_pre<NB>(lp, r, cta, n_cta, warp, lane, w_use, alive);
         } else if (alive) {
             if (op.type == OP_EMBED) embed_phase(md, op, pr, r, cta, n_cta, tid);
-            else if (op.type == OP_ATTN) attn_phase<HD>(md, op, pr, r, cta, n_cta, warp, lane, pr.M >= MERGE_ROWS);
+            else if (op.type == OP_KV_APPEND) { if (NB > 1) kv_append_phase<HD>(md, op, pr, cta, n_cta, warp, lane); else ran = false; }
+            else if (op.type == OP_ATTN) {
+                if (NB == 1) {
+                    attn_phase<HD>(md, op, pr, r, cta, n_cta, warp, lane, pr.M >= MERGE_ROWS, 0, false);
+                } else {
+                    for (int blk = 0; blk < NB; ++blk) attn_phase<HD>(md, op, pr, r, cta, n_cta, warp, lane, true, blk * BLKM, true);
+                }
+            }
             else if (op.type == OP_ATTN_MERGE) { if (pr.M >= MERGE_ROWS) attn_merge_phase<HD>(md, op, pr, cta, n_cta, warp, lane); else ran = false; }
             else if (op.type == OP_HIDDEN) { if (pr.want_hidden) hidden_phase(md, pr, r, cta, tid); else ran = false; }
             else if (op.type == OP_ARGMAX) { if (pr.head_row0 < pr.M) argmax_phase(md, pr, r, cta, n_cta, tid); else ran = false; }
