@@ -23,6 +23,9 @@ __device__ __forceinline__ uint4 ld_frag4(const uint32_t *p) { return __ldcg(rei
 template <int NB>
 __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring &r, int cta, int n_cta, int warp, int lane,
                                                    int &w_use, bool &alive) {
+    // groups per batch: the tile loop is unrolled over them and has to stay small (instruction cache), so two row
+    // blocks take half as many groups; the producer is told the same number through LinPhase::gb
+    constexpr int GBN = GB / NB;
     const Share s = make_share(p, cta, n_cta);
     const int tid = warp * 32 + lane;
     const int g8 = lane >> 2, t4 = lane & 3;
@@ -45,10 +48,10 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
     for (int nb = 0; nb < NB; ++nb) ss_acc[nb] = 0.f;
 
     for (int b = 0; b < s.n_batches; ++b) {
-        const int g0 = b * GB, ng = min(s.n_groups - g0, GB);
-        float acc[GB][NB][4];
+        const int g0 = b * GBN, ng = min(s.n_groups - g0, GBN);
+        float acc[GBN][NB][4];
 #pragma unroll
-        for (int i = 0; i < GB; ++i)
+        for (int i = 0; i < GBN; ++i)
 #pragma unroll
             for (int nb = 0; nb < NB; ++nb) { acc[i][nb][0] = acc[i][nb][1] = acc[i][nb][2] = acc[i][nb][3] = 0.f; }
         uint4 nx[NB][NTERM][4];                              // fragments of the next column tile, block by block, term by term
@@ -82,7 +85,7 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
         // this thread's epilogue items: (unit, token) pairs, token fastest among the M live tokens.  For a residual
         // update the old value and the next gain are fetched now, long before the epilogue needs them.
         const int gshift = s.swiglu ? 3 : 4, total = (ng << gshift) * p.M;
-        constexpr int ITEMS = GB * 16 * 8 * NB / (NCW * 32);
+        constexpr int ITEMS = GBN * 16 * 8 * NB / (NCW * 32);
         float xold[ITEMS], gnext[ITEMS];
 #pragma unroll
         for (int it4 = 0; it4 < ITEMS; ++it4) {
@@ -111,7 +114,7 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
                     }
             if (kt + 1 < s.n_kt) fetch(kt + 1);
 #pragma unroll
-            for (int gi = 0; gi < GB; ++gi) {
+            for (int gi = 0; gi < GBN; ++gi) {
                 if (gi >= ng) break;
                 if (alive) alive = mbar_wait(&r.full_w[ws], it & 1, r.abort_flag, r.err, 5);
                 if (alive && slot_valid) {
@@ -146,10 +149,10 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
         }
         // ---- batch end: partial sums of the 8 column slots meet in shared memory, in warp order ----
 #pragma unroll
-        for (int gi = 0; gi < GB; ++gi)
+        for (int gi = 0; gi < GBN; ++gi)
 #pragma unroll
             for (int nb = 0; nb < NB; ++nb)
-                *reinterpret_cast<float4 *>(red + ((((warp * GB + gi) * NB + nb) * 32) + lane) * 4) =
+                *reinterpret_cast<float4 *>(red + ((((warp * GBN + gi) * NB + nb) * 32) + lane) * 4) =
                     make_float4(acc[gi][nb][0], acc[gi][nb][1], acc[gi][nb][2], acc[gi][nb][3]);
         asm volatile("bar.sync 1, %0;" ::"n"(NCW * 32) : "memory");
         if (alive) {
@@ -166,7 +169,7 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
                 float s0 = 0.f, s1 = 0.f;
 #pragma unroll
                 for (int w = 0; w < NCW; ++w) {
-                    const float *q = red + ((((w * GB + gi) * NB + nb) * 32) + src_lane) * 4;
+                    const float *q = red + ((((w * GBN + gi) * NB + nb) * 32) + src_lane) * 4;
                     s0 += q[e0];
                     if (s.swiglu) s1 += q[2 + reg];
                 }
@@ -182,7 +185,7 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
                     __stcg(yp, v);
                     if (p.ys) store_split(p.ys, p.units >> 7, n, u, v * gnext[it4]);
                     // leave v^2 where this thread alone read its first partial: warp n % 8 adds them up below
-                    red[((((0 * GB + gi) * NB + nb) * 32) + src_lane) * 4 + e0] = v * v;
+                    red[((((0 * GBN + gi) * NB + nb) * 32) + src_lane) * 4 + e0] = v * v;
                 } else {
                     __stcg(yp, s0 * ri);
                 }
@@ -199,7 +202,7 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
                     for (int i = lane; i < (ng << gshift); i += 32) {
                         const int gi = i >> gshift, rr = i & ((1 << gshift) - 1);
                         if (rr < s.group_size(g0 + gi))
-                            part += red[((((0 * GB + gi) * NB + nb) * 32) + (rr & 7) * 4 + (n8 >> 1)) * 4 + (rr >> 3) * 2 + (n8 & 1)];
+                            part += red[((((0 * GBN + gi) * NB + nb) * 32) + (rr & 7) * 4 + (n8 >> 1)) * 4 + (rr >> 3) * 2 + (n8 & 1)];
                     }
                     part = warp_sum(part);
                     ss_acc[nb] += part;

@@ -62,7 +62,8 @@ struct LinPhase {
     float eps;
     float *y;           // [M][units]
     int epi;
-    int M;              // 1..8
+    int M;              // 1..8 (stand-alone kernel), 1..16 (pass kernel)
+    int gb;             // groups per batch, 1..GB (0 = GB); producer and consumers must use the same value
     // Pre-split form (persistent pass kernel): the producer of an activation writes it already split into the three
     // bf16 terms, in the order the tensor-core operand wants, so the consuming map only loads fragments.
     const uint32_t *xs;      // input  [M][K/128][NTERM terms][4][16] words (see split_index); nullptr = read x / gain
@@ -166,7 +167,7 @@ __device__ __forceinline__ void store_split(uint32_t *buf, int nslots, int m, in
 // The CTA's share of a linear map: units [u_lo, u_lo + n_units) in n_groups groups whose sizes differ by at
 // most one (the first g_rem groups hold g_base + 1 units).
 struct Share {
-    int u_lo, n_units, n_groups, g_base, g_rem, n_batches, n_kt, gsz;
+    int u_lo, n_units, n_groups, g_base, g_rem, n_batches, n_kt, gsz, gb;
     bool swiglu;
     __device__ __forceinline__ int group_lo(int g) const { return g * g_base + min(g, g_rem); }
     __device__ __forceinline__ int group_size(int g) const { return g_base + (g < g_rem ? 1 : 0); }
@@ -182,7 +183,8 @@ __device__ __forceinline__ Share make_share(const LinPhase &p, int cta, int n_ct
     s.n_groups = (s.n_units + s.gsz - 1) / s.gsz;
     s.g_base = s.n_groups ? s.n_units / s.n_groups : 0;
     s.g_rem = s.n_groups ? s.n_units % s.n_groups : 0;
-    s.n_batches = (s.n_groups + GB - 1) / GB;
+    s.gb = p.gb > 0 && p.gb < GB ? p.gb : GB;
+    s.n_batches = (s.n_groups + s.gb - 1) / s.gb;
     s.n_kt = (p.K + SEG - 1) / SEG;
     return s;
 }
@@ -212,7 +214,7 @@ __device__ __forceinline__ void produce_linear(const LinPhase &p, const Ring &r,
     const Share s = make_share(p, cta, n_cta);
     int ws = w_use % WS, it = w_use / WS;
     for (int b = 0; b < s.n_batches && alive; ++b) {
-        const int g0 = b * GB, ng = min(s.n_groups - g0, GB);
+        const int g0 = b * s.gb, ng = min(s.n_groups - g0, s.gb);
         // source row of this lane in each group of the batch, and the row count of each group
         const bf16_t *src[GB];
         int nrows[GB];
@@ -275,7 +277,7 @@ __device__ __forceinline__ void consume_linear(const LinPhase &p, const Ring &r,
     int ws = w_use % WS, it = w_use / WS;
     float *red = r.red, *red_ss = r.red_ss;
     for (int b = 0; b < s.n_batches; ++b) {
-        const int g0 = b * GB, ng = min(s.n_groups - g0, GB);
+        const int g0 = b * s.gb, ng = min(s.n_groups - g0, s.gb);
         float acc[GB][4];
 #pragma unroll
         for (int i = 0; i < GB; ++i) { acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f; }
