@@ -224,6 +224,32 @@ def test_full_width_13b_layers_match_oracle(kb):
         assert np.array_equal(got["accepts"], want["accepts"])
 
 
+@pytest.mark.parametrize("shape_name,prompt_len", [("qwen14b", 186), ("llama7b", 120)])
+def test_full_width_other_shapes_match_oracle(kb, shape_name, prompt_len):
+    """Full widths of the Qwen-2.5-14B-shaped (GQA 40/8, vocab 152064, theta 1e6) and LLaMA-2-7B-shaped workloads on two
+    layers; the Qwen case starts six positions before a 64-position segment boundary, so drafted and verified rows
+    straddle it."""
+    shape = si.SHAPES[shape_name].with_layers(2)
+    mask = np.array([0, 1, 1, 0], np.uint8)                    # skip MLP of layer 0 and attention of layer 1
+    damp = {1: 0.02, 2: 0.02}
+    w = si.make_model_weights(shape, 6, device="cuda", damp=damp, gain_spread=0.1)
+    wc = {k: ([t.cpu() for t in v] if isinstance(v, list) else v.cpu()) for k, v in w.items()}
+    om = oracle.OracleModel(shape, wc, prompt_len + 40)
+    sess = kb.Session.from_shape(shape, w, prompt_len + 40, max_draft=8)
+    prompt = si.uniform_tokens(11, 0, prompt_len, shape.vocab).numpy()
+    _, first_o, _ = om.prefill(prompt)
+    assert sess.prefill(prompt) == first_o
+    sess.set_skipmask(mask)
+    for k in (4, 8):
+        om.length = prompt_len
+        sess.set_length(prompt_len)
+        sess.set_pending(first_o)
+        want = om.generate(first_o, 12, k, mask)
+        got = sess.decode(12, k)
+        assert np.array_equal(got["tokens"], want["tokens"]), f"k={k}: oracle min margin {want['min_margin']}"
+        assert np.array_equal(got["accepts"], want["accepts"])
+
+
 def test_config1_tiny_all_on_and_all_off_masks(kb):
     shape, om, sess = _pair(kb, "tiny", gain_spread=0.0)
     prompt = si.uniform_tokens(0, 0, 32, shape.vocab).numpy()
