@@ -298,12 +298,13 @@ def run_ours(args):
         "clocks": clocks,
     }
     if not args.no_cpu_baseline and world == 1:
-        out["cpu_baseline"] = cpu_baseline(args, shape, w, masks[dom], steps=1, warmup=0)
+        out["cpu_baseline"] = cpu_baseline(args, shape, w, masks[dom], steps=1, warmup=0, sess=sess)
     print(json.dumps(out))
 
 
-def cpu_baseline(args, shape, w_dev, mask, steps, warmup, per_step=None):
-    """The oracle as it stands, on this host's cores, on a bounded sample: a short prompt and a few rounds."""
+def cpu_baseline(args, shape, w_dev, mask, steps, warmup, per_step=None, sess=None):
+    """The oracle as it stands, on this host's cores, on a bounded sample: a short prompt and a few rounds.  With a
+    session given, the CUDA path runs the same sample at full model size and the two token streams are compared."""
     import oracle
     w = {kname: ([t.cpu() for t in v] if isinstance(v, list) else v.cpu()) for kname, v in w_dev.items()}
     sp, sn = args.cpu_prompt, args.cpu_new
@@ -321,9 +322,16 @@ def cpu_baseline(args, shape, w_dev, mask, steps, warmup, per_step=None):
         if per_step:
             per_step(dt)
     total = sum(times)
-    return {"value": sn * len(times) / total, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
-            "sample": f"same shape and mask, {sp}-token prompt, {sn} new tokens per step with k={args.k} "
-                      f"({len(times)} timed step(s), decode only)", "ms_per_step": 1e3 * total / len(times)}
+    out = {"value": sn * len(times) / total, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
+           "sample": f"same shape and mask, {sp}-token prompt, {sn} new tokens per step with k={args.k} "
+                     f"({len(times)} timed step(s), decode only)", "ms_per_step": 1e3 * total / len(times)}
+    if sess is not None and warmup == 0 and steps == 1:
+        # full-size parity on the sample: same prompt, mask and k through the CUDA path
+        sess.set_skipmask(mask)
+        g = sess.generate(prompt, sn, args.k)
+        out["gpu_matches_oracle_on_sample"] = bool(np.array_equal(g["tokens"], r["tokens"]) and
+                                                   np.array_equal(g["accepts"], r["accepts"]))
+    return out
 
 
 def run_stream(args):
