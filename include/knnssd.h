@@ -208,6 +208,21 @@ knnssd_status knnssd_linear(const void *W_dev, int dtype, int n_out, int n_in, c
                             float *y_dev, void *cuda_stream);
 
 /*
+ * The contraction of the prompt pass (Sec. 4.2: the model's pass over the whole sample, T rows at once), on the
+ * tensor cores: x is split into two bf16 terms (hi + lo) and multiplied with the bf16 weights, fp32 accumulation.
+ *   mode 0   y[t][o]  = sum_i W0[o][i] x[t][i]
+ *   mode 1   y[t][o] += sum_i W0[o][i] x[t][i]                      (residual add)
+ *   mode 2   y[t][o]  = silu(sum_i W0[o][i] x[t][i]) * (sum_i W1[o][i] x[t][i]), rounded to hi + lo bf16 terms as
+ *            the prompt pass hands it to the next map
+ *   W0, W1 DEVICE bf16 [n_out][n_in], 16-byte aligned (W1 only for mode 2); x DEVICE fp32 [T][n_in];
+ *   y DEVICE fp32 [T][n_out]; n_in % 64 == 0, n_out % 8 == 0, T >= 1.
+ * Allocates and frees its temporary planes, and synchronises the stream before it returns.  KNNSSD_ERR_SHAPE for
+ * sizes outside the rules above, KNNSSD_ERR_TIMEOUT if a device-side wait gave up.
+ */
+knnssd_status knnssd_gemm_split(const void *W0_dev, const void *W1_dev, int n_out, int n_in, const float *x_dev, int T,
+                                int mode, float *y_dev, void *cuda_stream);
+
+/*
  * Cosine top-1 (Sec. 4.2, Eq. (4)) of one query against n anchors of dimension d, all DEVICE fp32; HOST outputs.
  * KNNSSD_ERR_DEGENERATE for a zero / non-finite query or anchor.
  */

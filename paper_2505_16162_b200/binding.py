@@ -23,7 +23,7 @@ STATUS = {0: "OK", 1: "ERR_INVALID_ARG", 2: "ERR_SHAPE", 3: "ERR_CAPACITY", 4: "
 EXPORTS = ["knnssd_init", "knnssd_destroy", "knnssd_prefill", "knnssd_select_skipset", "knnssd_set_skipmask",
            "knnssd_draft", "knnssd_verify", "knnssd_generate", "knnssd_decode", "knnssd_get_launch_count", "knnssd_get_length", "knnssd_set_length",
            "knnssd_set_pending", "knnssd_get_stats", "knnssd_last_error", "knnssd_time_pass", "knnssd_trace_pass", "knnssd_linear",
-           "knnssd_cosine_top1", "knnssd_cosine_top1_static"]
+           "knnssd_gemm_split", "knnssd_cosine_top1", "knnssd_cosine_top1_static"]
 
 
 class KnnssdError(RuntimeError):
@@ -76,6 +76,7 @@ def _load():
         "knnssd_time_pass": (I, [P, I, I, I, PF, PI, PF, PI]),
         "knnssd_trace_pass": (I, [P, I, I, I, PI, PI, PF, PF, PI]),
         "knnssd_linear": (I, [P, I, I, I, P, I, P, P]),
+        "knnssd_gemm_split": (I, [P, P, I, I, P, I, I, P, P]),
         "knnssd_cosine_top1": (I, [P, P, I, I, PI, PF, P]),
         "knnssd_cosine_top1_static": (I, [P, P, I, I, PI, PF, P]),
     }
@@ -118,6 +119,23 @@ def knnssd_linear(W: torch.Tensor, x: torch.Tensor, stream: Optional[torch.cuda.
                                 cur.cuda_stream)
     if rc:
         raise KnnssdError(rc, "knnssd_linear")
+    return y
+
+
+def knnssd_gemm_split(W0: torch.Tensor, x: torch.Tensor, mode: int = 0, W1: Optional[torch.Tensor] = None,
+                      y: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """The prompt pass's tensor-core contraction over T rows.  W0 (and W1 for mode 2) bf16 [n_out][n_in], x fp32 [T][n_in].
+    mode 0: y = x W0^T; 1: y += x W0^T (y given); 2: silu(x W0^T) * (x W1^T), rounded to two bf16 terms."""
+    T, n_in = x.shape
+    n_out = W0.shape[0]
+    if y is None:
+        y = torch.zeros((T, n_out), dtype=torch.float32, device=x.device)
+    with torch.cuda.device(x.device):
+        rc = _lib.knnssd_gemm_split(_dev_ptr(W0, torch.bfloat16), None if W1 is None else _dev_ptr(W1, torch.bfloat16), n_out, n_in,
+                                    _dev_ptr(x, torch.float32), T, mode, _dev_ptr(y, torch.float32),
+                                    torch.cuda.current_stream().cuda_stream)
+    if rc:
+        raise KnnssdError(rc, "knnssd_gemm_split")
     return y
 
 

@@ -5,6 +5,7 @@
 #include "kernels.cuh"
 #include "linear_stream.cuh"
 #include "pass_kernel.cuh"
+#include "prefill_host.cuh"
 
 #include <cmath>
 #include <cstdio>
@@ -1005,6 +1006,42 @@ knnssd_status knnssd_linear(const void *W_dev, int dtype, int n_out, int n_in, c
     LinearArgs a = make_args(W_dev, n_out, n_in, x_dev, nullptr, 0.f, y_dev, EPI_STORE, M);
     launch_linear(dtype, a, n_sms, reinterpret_cast<cudaStream_t>(cuda_stream));
     return cudaGetLastError() == cudaSuccess ? KNNSSD_OK : KNNSSD_ERR_CUDA;
+}
+
+knnssd_status knnssd_gemm_split(const void *W0_dev, const void *W1_dev, int n_out, int n_in, const float *x_dev, int T,
+                                int mode, float *y_dev, void *cuda_stream) {
+    if (!W0_dev || !x_dev || !y_dev || T < 1 || n_out < 1 || n_in < 1 || mode < 0 || mode > 2 || (mode == 2 && !W1_dev))
+        return KNNSSD_ERR_INVALID_ARG;
+    if (n_in % prefill::BK != 0 || n_out % 8 != 0 || (reinterpret_cast<uintptr_t>(W0_dev) & 15u) ||
+        (reinterpret_cast<uintptr_t>(W1_dev) & 15u) || (reinterpret_cast<uintptr_t>(x_dev) & 15u) ||
+        (reinterpret_cast<uintptr_t>(y_dev) & 15u))
+        return KNNSSD_ERR_SHAPE;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+    const int cap = (T + prefill::BM - 1) / prefill::BM * prefill::BM;
+    bf16_t *planes = nullptr, *outp = nullptr;
+    const size_t plane = (size_t)cap * n_in, oplane = (size_t)T * n_out;
+    if (dev_alloc(&planes, 2 * plane) != cudaSuccess) { cudaGetLastError(); return KNNSSD_ERR_CUDA; }
+    if (mode == 2 && dev_alloc(&outp, 2 * oplane) != cudaSuccess) { cudaGetLastError(); cudaFree(planes); return KNNSSD_ERR_CUDA; }
+    knnssd_status st = KNNSSD_OK;
+    cudaMemsetAsync(planes, 0, 2 * plane * sizeof(bf16_t), s);
+    prefill::split_rows_kernel<<<T, 256, 0, s>>>(x_dev, n_in, planes, planes + plane);
+    CUtensorMap ta;
+    if (!prefill::make_map(&ta, planes, (size_t)2 * cap, (size_t)n_in) ||
+        !prefill::launch_gemm(ta, cap, W0_dev, W1_dev, n_out, n_in, T, mode, y_dev, n_out, 0, outp, outp ? outp + oplane : nullptr,
+                              n_out, stream_err_ptr(), s))
+        st = KNNSSD_ERR_CUDA;
+    if (st == KNNSSD_OK && mode == 2) prefill::join_planes_kernel<<<T, 256, 0, s>>>(outp, outp + oplane, n_out, y_dev);
+    cudaError_t e = cudaStreamSynchronize(s);
+    if (e == cudaSuccess) e = cudaGetLastError();
+    if (e != cudaSuccess) st = KNNSSD_ERR_CUDA;
+    if (st == KNNSSD_OK) {
+        int code = 0;
+        if (cudaMemcpy(&code, stream_err_ptr(), sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) st = KNNSSD_ERR_CUDA;
+        else if (code) { cudaMemset(stream_err_ptr(), 0, sizeof(int)); st = KNNSSD_ERR_TIMEOUT; }
+    }
+    cudaFree(planes);
+    if (outp) cudaFree(outp);
+    return st;
 }
 
 knnssd_status knnssd_cosine_top1(const float *query_dev, const float *anchors_dev, int n, int d, int *best, float *cosine,

@@ -1,0 +1,564 @@
+// Prompt pass on the 5th-generation tensor cores.
+//
+// The prompt pass is the full model over all T prompt tokens at once (Section 4.2: the sample's last hidden vector
+// comes from a pass of the model over the sample; the same pass fills the K/V cache that drafting and verification
+// read).  With T in the hundreds or thousands every linear map is a real contraction [T x K] . [K x N], so it runs on
+// tcgen05.mma with the accumulator in tensor memory, operands staged in shared memory by TMA:
+//
+//   gemm_split_kernel   Y[T][N] (+)= A[T][K] . W[N][K]^T, A given as two bf16 planes (hi + lo of the fp32
+//                       activation, so that the product with the bf16 weights carries 16 mantissa bits of A, as in
+//                       the decode passes), accumulator fp32.  Epilogues: store, add to the residual stream,
+//                       SwiGLU of a gate tile and an up tile.
+//   norm_split_kernel   RMSNorm of each row, written as the two bf16 planes the next map reads.
+//   rope_kv_kernel      rotary embedding of q and k, K/V rows rounded to bf16 into the cache.
+//   attn_prompt_kernel  causal attention of 8 query rows per warp over the cached K/V, on mma.sync (the sizes are
+//                       small next to the linear maps), output written as bf16 planes for the O projection.
+//
+// Every wait in these kernels is bounded; a wait that gives up sets the error word and the kernel returns after
+// releasing its tensor memory.
+#pragma once
+
+#include <cuda.h>
+
+#include "linear_stream.cuh"
+
+namespace knnssd {
+namespace prefill {
+
+using stream::mbar_init;
+using stream::mbar_try_wait;
+using stream::smem_u32;
+
+constexpr int BM = 128;                               // tokens per tile: rows of the accumulator = lanes of tensor memory
+constexpr int BN = 256;                               // accumulator columns per tile: two boxes of 128 weight rows
+constexpr int BK = 64;                                // input columns per stage: 128 bytes of bf16 = one swizzle row
+constexpr int STAGES = 3;
+constexpr int A_BYTES = BM * BK * 2;                  // one term of the activation tile
+constexpr int B_BYTES = BN * BK * 2;
+constexpr int STAGE_BYTES = 2 * A_BYTES + B_BYTES;    // hi plane, lo plane, weights
+constexpr int GEMM_THREADS = 192;                     // warp 0: TMA; warp 1: MMA issue + tensor-memory owner; warps 2..5: epilogue
+constexpr int GEMM_SMEM = STAGES * STAGE_BYTES + 1024 + 128;   // + slack to align the tiles to 1024 bytes + barriers
+constexpr unsigned WAIT_LIMIT = 4000000u;           // polls of one wait (a whole tile takes well under a millisecond)
+
+enum { PF_STORE = 0, PF_ADD = 1, PF_SWIGLU = 2 };
+
+struct GemmArgs {
+    int T;             // live rows
+    int K;             // input width, a multiple of BK
+    int N;             // output units (per matrix)
+    float *y;          // STORE: y[t * ldy + col0 + n] = sum;  ADD: y[t * ldy + n] += sum
+    int ldy, col0;
+    bf16_t *out_hi;    // SWIGLU: silu(gate) * up as two bf16 planes, [t * ldo + n]
+    bf16_t *out_lo;
+    int ldo;
+    int *err;          // set non-zero if a bounded wait gave up
+};
+
+__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int x, int y, uint64_t *bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(
+                     smem_u32(dst)),
+                 "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y)
+                 : "memory");
+}
+
+// Shared-memory operand descriptor of tcgen05.mma for a K-major tile whose rows are 128 bytes, written by TMA with the
+// 128-byte swizzle: start address / 16 in bits 0..13, leading-dimension offset (unused for this layout) in 16..29,
+// stride between groups of 8 rows (1024 bytes) / 16 in 32..45, descriptor version 1 in 46..47, swizzle mode 2
+// (128 bytes) in 61..63.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr) {
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) |
+           ((uint64_t)2 << 61);
+}
+// Instruction descriptor, kind::f16: fp32 accumulator (bits 4..5 = 1), A and B bf16 (bits 7..9 and 10..12 = 1), both
+// K-major (bits 15, 16 = 0), N / 8 in bits 17..22, M / 16 in bits 24..28.
+constexpr uint32_t UMMA_IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t"
+        "}\n" ::"r"(tmem_d),
+        "l"(da), "l"(db), "r"(UMMA_IDESC), "r"(accumulate)
+        : "memory");
+}
+// The barrier gets one arrival once every MMA this thread issued before has finished.
+__device__ __forceinline__ void umma_commit(uint64_t *bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// 32 consecutive accumulator columns of this thread's lane (lane = 32 * (warp % 4) + lane id).
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, "
+        "%18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+          "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+          "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+          "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Bounded wait on an mbarrier phase; false once the limit is reached or another thread of the CTA has given up.
+__device__ __forceinline__ bool pf_wait(uint64_t *b, uint32_t parity, volatile int *cta_abort, int *err, int code) {
+    unsigned spins = 0;
+    while (!mbar_try_wait(b, parity)) {
+        if (*cta_abort) return false;
+        if (++spins > WAIT_LIMIT) {
+            *cta_abort = 1;
+            atomicExch(err, code);
+            return false;
+        }
+    }
+    return true;
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(uint32_t lo16, uint32_t hi16) { return lo16 | (hi16 << 16); }
+
+// One CTA per tile of 128 tokens x 256 accumulator columns.  EPI = PF_SWIGLU: columns 0..127 are units n0..n0+127 of
+// the gate matrix (map tb0) and columns 128..255 the same units of the up matrix (map tb1); otherwise the columns are
+// units n0..n0+255 of one matrix (tb0 = tb1).  ta covers both activation planes: rows [0, Tpad) the hi terms, rows
+// [Tpad, 2 Tpad) the lo terms.
+template <int EPI>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+gemm_split_kernel(const __grid_constant__ CUtensorMap ta, const __grid_constant__ CUtensorMap tb0,
+                  const __grid_constant__ CUtensorMap tb1, GemmArgs g, int Tpad) {
+    extern __shared__ unsigned char pf_smem_raw[];
+    unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(pf_smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint64_t *full = reinterpret_cast<uint64_t *>(smem + STAGES * STAGE_BYTES);
+    uint64_t *empty = full + STAGES;
+    uint64_t *acc_full = empty + STAGES;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_full + 1);
+    volatile int *cta_abort = reinterpret_cast<volatile int *>(tmem_slot + 1);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int t0 = blockIdx.x * BM;
+    const int n0 = blockIdx.y * (EPI == PF_SWIGLU ? BN / 2 : BN);
+    const int nkb = g.K / BK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        mbar_init(acc_full, 1);
+        *cta_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(BN) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // ---- TMA producer: a stage is refilled once the MMAs that read it have finished ----
+            int armed = 0;
+            for (int kb = 0; kb < nkb; ++kb) {
+                const int s = kb % STAGES;
+                const uint32_t ph = (uint32_t)(kb / STAGES) & 1u;
+                if (!pf_wait(&empty[s], ph ^ 1u, cta_abort, g.err, 21)) break;
+                unsigned char *st = smem + s * STAGE_BYTES;
+                stream::mbar_expect_tx(&full[s], STAGE_BYTES);
+                tma_load_2d(st, &ta, kb * BK, t0, &full[s]);
+                tma_load_2d(st + A_BYTES, &ta, kb * BK, Tpad + t0, &full[s]);
+                tma_load_2d(st + 2 * A_BYTES, &tb0, kb * BK, n0, &full[s]);
+                tma_load_2d(st + 2 * A_BYTES + B_BYTES / 2, &tb1, kb * BK, EPI == PF_SWIGLU ? n0 : n0 + BN / 2, &full[s]);
+                armed = kb + 1;
+            }
+            if (*cta_abort) {
+                // copies in flight land in this CTA's shared memory: let them finish before the CTA goes away
+                for (int kb = (armed > STAGES ? armed - STAGES : 0); kb < armed; ++kb) {
+                    unsigned spins = 0;
+                    while (!mbar_try_wait(&full[kb % STAGES], (uint32_t)(kb / STAGES) & 1u) && ++spins < WAIT_LIMIT) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // ---- MMA issue: 4 k-steps of 16 columns per stage, hi and lo term into the same accumulator ----
+            bool ok = true;
+            for (int kb = 0; kb < nkb && ok; ++kb) {
+                const int s = kb % STAGES;
+                const uint32_t ph = (uint32_t)(kb / STAGES) & 1u;
+                ok = pf_wait(&full[s], ph, cta_abort, g.err, 22);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t a_hi = smem_u32(smem + s * STAGE_BYTES), a_lo = a_hi + A_BYTES, b = a_hi + 2 * A_BYTES;
+#pragma unroll
+                for (int k = 0; k < BK / 16; ++k) {
+                    const uint64_t db = umma_desc(b + 32 * k);
+                    umma_bf16(tmem, umma_desc(a_hi + 32 * k), db, (kb | k) != 0 ? 1u : 0u);
+                    umma_bf16(tmem, umma_desc(a_lo + 32 * k), db, 1u);
+                }
+                umma_commit(&empty[s]);
+            }
+            umma_commit(acc_full);         // on the abort path too: it releases the epilogue warps' wait
+        }
+    } else {
+        // ---- epilogue: warp w reads lanes 32 (w % 4) .. + 31 of tensor memory = tokens t0 + 32 (w % 4) + lane ----
+        // the loads from tensor memory are warp-wide: the warp goes on only if all of its threads saw the accumulator
+        const bool ok = __all_sync(0xffffffffu, pf_wait(acc_full, 0u, cta_abort, g.err, 23) && !*cta_abort);
+        tc_fence_after();
+        const int q = warp & 3;
+        const int t = t0 + 32 * q + lane;
+        const uint32_t trow = tmem + ((uint32_t)(32 * q) << 16);
+        if (ok) {
+            if (EPI == PF_SWIGLU) {
+                for (int c0 = 0; c0 < BN / 2 && n0 + c0 < g.N; c0 += 32) {
+                    float gt[32], up[32];
+                    tmem_ld32(trow + c0, gt);
+                    tmem_ld32(trow + BN / 2 + c0, up);
+                    if (t < g.T) {
+                        uint32_t hi[16], lo[16];
+#pragma unroll
+                        for (int i = 0; i < 32; i += 2) {
+                            uint32_t h2[2], l2[2];
+#pragma unroll
+                            for (int e = 0; e < 2; ++e) {
+                                const float a = gt[i + e] / (1.0f + expf(-gt[i + e])) * up[i + e];
+                                h2[e] = float_to_bf16_rne(a);
+                                l2[e] = float_to_bf16_rne(a - __uint_as_float(h2[e] << 16));
+                            }
+                            hi[i >> 1] = pack_bf16(h2[0], h2[1]);
+                            lo[i >> 1] = pack_bf16(l2[0], l2[1]);
+                        }
+                        bf16_t *ph = g.out_hi + (size_t)t * g.ldo + n0 + c0, *pl = g.out_lo + (size_t)t * g.ldo + n0 + c0;
+                        if (n0 + c0 + 32 <= g.N) {
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                reinterpret_cast<uint4 *>(ph)[i] = make_uint4(hi[4 * i], hi[4 * i + 1], hi[4 * i + 2], hi[4 * i + 3]);
+                                reinterpret_cast<uint4 *>(pl)[i] = make_uint4(lo[4 * i], lo[4 * i + 1], lo[4 * i + 2], lo[4 * i + 3]);
+                            }
+                        } else {
+                            for (int i = 0; n0 + c0 + i < g.N; ++i) {
+                                ph[i] = (bf16_t)((hi[i >> 1] >> (16 * (i & 1))) & 0xFFFFu);
+                                pl[i] = (bf16_t)((lo[i >> 1] >> (16 * (i & 1))) & 0xFFFFu);
+                            }
+                        }
+                    }
+                }
+            } else {
+                for (int c0 = 0; c0 < BN && n0 + c0 < g.N; c0 += 32) {
+                    float v[32];
+                    tmem_ld32(trow + c0, v);
+                    if (t < g.T) {
+                        float *yp = g.y + (size_t)t * g.ldy + g.col0 + n0 + c0;
+                        if (n0 + c0 + 32 <= g.N) {
+#pragma unroll
+                            for (int i = 0; i < 32; i += 4) {
+                                float4 o = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+                                if (EPI == PF_ADD) {
+                                    const float4 x = *reinterpret_cast<const float4 *>(yp + i);
+                                    o.x += x.x; o.y += x.y; o.z += x.z; o.w += x.w;
+                                }
+                                *reinterpret_cast<float4 *>(yp + i) = o;
+                            }
+                        } else {
+                            for (int i = 0; n0 + c0 + i < g.N; ++i) yp[i] = EPI == PF_ADD ? yp[i] + v[i] : v[i];
+                        }
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(BN) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Row-wise kernels around the contractions
+// ---------------------------------------------------------------------------------------------
+
+// x[t][:] = embedding row of token t (bf16 -> fp32).  grid = T.
+__global__ void embed_rows_kernel(const bf16_t *__restrict__ table, const int *__restrict__ tok, int d, float *__restrict__ x) {
+    const bf16_t *row = table + (size_t)tok[blockIdx.x] * d;
+    float *xr = x + (size_t)blockIdx.x * d;
+    for (int i = threadIdx.x; i < d; i += blockDim.x) xr[i] = bf16_bits_to_float(row[i]);
+}
+
+// RMSNorm of row t (gain g, epsilon eps), written as hi = bf16(v) and lo = bf16(v - hi).  grid = T, 256 threads.
+__global__ void __launch_bounds__(256) norm_split_kernel(const float *__restrict__ x, int d, const float *__restrict__ gain, float eps,
+                                                         bf16_t *__restrict__ hi, bf16_t *__restrict__ lo) {
+    __shared__ float part[8];
+    const float *xr = x + (size_t)blockIdx.x * d;
+    float ss = 0.f;
+    for (int i = threadIdx.x * 4; i < d; i += 1024) {
+        const float4 v = *reinterpret_cast<const float4 *>(xr + i);
+        ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+    }
+    ss = warp_sum(ss);
+    if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) tot += part[w];
+    const float rinv = 1.0f / sqrtf(tot / (float)d + eps);
+    bf16_t *hr = hi + (size_t)blockIdx.x * d, *lr = lo + (size_t)blockIdx.x * d;
+    for (int i = threadIdx.x * 4; i < d; i += 1024) {
+        const float4 v = *reinterpret_cast<const float4 *>(xr + i);
+        const float4 g = *reinterpret_cast<const float4 *>(gain + i);
+        const float a[4] = {v.x * rinv * g.x, v.y * rinv * g.y, v.z * rinv * g.z, v.w * rinv * g.w};
+        uint32_t h[4], l[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            h[e] = float_to_bf16_rne(a[e]);
+            l[e] = float_to_bf16_rne(a[e] - __uint_as_float(h[e] << 16));
+        }
+        *reinterpret_cast<uint2 *>(hr + i) = make_uint2(pack_bf16(h[0], h[1]), pack_bf16(h[2], h[3]));
+        *reinterpret_cast<uint2 *>(lr + i) = make_uint2(pack_bf16(l[0], l[1]), pack_bf16(l[2], l[3]));
+    }
+}
+
+// Rotary embedding of the q and k heads of row t at position pos0 + t (q in place, fp32); K and V rows rounded to
+// bf16 into the cache.  grid = (H + 2 Hkv, T), hd / 2 threads: thread i owns the pair (i, i + hd / 2).
+__global__ void rope_kv_rows_kernel(float *__restrict__ qkv, int H, int Hkv, int hd, const double *__restrict__ inv_freq,
+                                    bf16_t *__restrict__ kc, bf16_t *__restrict__ vc, int max_seq, int pos0) {
+    const int slot = blockIdx.x, t = blockIdx.y, i = threadIdx.x, half = hd / 2;
+    float *row = qkv + (size_t)t * (H + 2 * Hkv) * hd + (size_t)slot * hd;
+    const int pos = pos0 + t;
+    if (slot < H + Hkv) {
+        double sn, cs;
+        sincos((double)pos * inv_freq[i], &sn, &cs);
+        const float c = (float)cs, s = (float)sn;
+        const float a = row[i], b = row[i + half];
+        const float ra = a * c - b * s, rb = b * c + a * s;
+        if (slot < H) {
+            row[i] = ra;
+            row[i + half] = rb;
+        } else {
+            bf16_t *dst = kc + ((size_t)(slot - H) * max_seq + pos) * hd;
+            dst[i] = float_to_bf16_rne(ra);
+            dst[i + half] = float_to_bf16_rne(rb);
+        }
+    } else {
+        bf16_t *dst = vc + ((size_t)(slot - H - Hkv) * max_seq + pos) * hd;
+        dst[i] = float_to_bf16_rne(row[i]);
+        dst[i + half] = float_to_bf16_rne(row[i + half]);
+    }
+}
+
+// y[t][n] = hi[t][n] + lo[t][n] (the value a pair of planes stands for).  grid = T.
+__global__ void join_planes_kernel(const bf16_t *__restrict__ hi, const bf16_t *__restrict__ lo, int n, float *__restrict__ y) {
+    const size_t base = (size_t)blockIdx.x * n;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) y[base + i] = bf16_bits_to_float(hi[base + i]) + bf16_bits_to_float(lo[base + i]);
+}
+// The two planes of plain fp32 rows (no norm).  grid = T.
+__global__ void split_rows_kernel(const float *__restrict__ x, int n, bf16_t *__restrict__ hi, bf16_t *__restrict__ lo) {
+    const size_t base = (size_t)blockIdx.x * n;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+        const float v = x[base + i];
+        const uint32_t h = float_to_bf16_rne(v);
+        hi[base + i] = (bf16_t)h;
+        lo[base + i] = float_to_bf16_rne(v - __uint_as_float(h << 16));
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Causal attention over the prompt
+// ---------------------------------------------------------------------------------------------
+
+// m16n8k16 with only rows 0..7 of the 16-row operand in use (registers of rows 8..15 are zero).
+__device__ __forceinline__ void mma_rows8(float (&c)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
+}
+
+// One warp per (head, block of 8 consecutive prompt rows); it walks the positions 0 .. (its last row's position) in
+// segments of 64 with a running maximum and sum (the softmax of a row is taken over all its positions at once in
+// exact arithmetic; the running form differs from it by rounding only).  K and V, this chunk's rows included, are
+// already in the cache in bf16; q is rotated fp32 and is split into hi + lo here, as are the probabilities.
+// Lane (g8, t4) = (lane / 4, lane % 4): row g8 of the block.  Index conventions of the two products:
+//   scores  column n = g8 of a tile is position 8 nt + g8; k-step s of the lane covers dimensions DL t4 + 4 s .. + 3
+//           for q and K alike (a dot product may take its terms in any order), so a lane reads one contiguous run of
+//           DL = HD / 4 dimensions of a K row;
+//   output  over pairs of tiles, k-indices (2 t4, 2 t4 + 1) = the lane's two positions of the first tile and
+//           (2 t4 + 8, 2 t4 + 9) those of the second; column n = g8 of V-tile j is dimension (HD / 8) g8 + j.
+// grid = (ceil(T / 8), ceil(H / 4)), 128 threads; the last row blocks (longest walks) are scheduled first.
+template <int HD>
+__global__ void __launch_bounds__(128) attn_prompt_kernel(const float *__restrict__ qkv, int H, int Hkv, const bf16_t *__restrict__ kc,
+                                                          const bf16_t *__restrict__ vc, int max_seq, int pos0, int T,
+                                                          bf16_t *__restrict__ out_hi, bf16_t *__restrict__ out_lo) {
+    constexpr int DL = HD / 4, NW = HD / 8, VW = HD / 16, VJ = HD / 8, SEG = 64, NT = SEG / 8;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g8 = lane >> 2, t4 = lane & 3;
+    const int h = blockIdx.y * 4 + warp;
+    if (h >= H) return;
+    const int rb = gridDim.x - 1 - blockIdx.x;
+    const int t_row = rb * 8 + g8;
+    const bool live = t_row < T;
+    const int p_row = pos0 + t_row;
+    const int p_last = pos0 + min(rb * 8 + 7, T - 1);
+    const int n_seg = p_last / SEG + 1;
+    const int kvh = h / (H / Hkv);
+    const int qstride = (H + 2 * Hkv) * HD;
+    const bf16_t *kbase = kc + (size_t)kvh * max_seq * HD, *vbase = vc + (size_t)kvh * max_seq * HD;
+    const float scale = 1.0f / sqrtf((float)HD);
+
+    uint32_t qh[NW], ql[NW];                                 // word w = dimensions (2w, 2w + 1) of the lane's run
+    {
+        const float *qr = qkv + (size_t)min(t_row, T - 1) * qstride + (size_t)h * HD + DL * t4;
+#pragma unroll
+        for (int e = 0; e < DL; e += 4) {
+            const float4 a = live ? *reinterpret_cast<const float4 *>(qr + e) : make_float4(0.f, 0.f, 0.f, 0.f);
+            const float v[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+            for (int i = 0; i < 4; i += 2) {
+                const uint32_t h0 = float_to_bf16_rne(v[i]), h1 = float_to_bf16_rne(v[i + 1]);
+                const uint32_t l0 = float_to_bf16_rne(v[i] - __uint_as_float(h0 << 16));
+                const uint32_t l1 = float_to_bf16_rne(v[i + 1] - __uint_as_float(h1 << 16));
+                qh[(e + i) >> 1] = pack_bf16(h0, h1);
+                ql[(e + i) >> 1] = pack_bf16(l0, l1);
+            }
+        }
+    }
+    float o[VJ][4];
+#pragma unroll
+    for (int j = 0; j < VJ; ++j) { o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f; }
+    float m_run = -INFINITY, l_run = 0.f;                    // l_run: this lane's share of the row's sum
+
+    for (int seg = 0; seg < n_seg; ++seg) {
+        const int p_begin = seg * SEG, p_end = min(p_begin + SEG, p_last + 1);
+        auto load_k = [&](int nt, uint4 (&dst)[NW / 4]) {
+            const int p = p_begin + 8 * nt + g8;
+            const bf16_t *src = kbase + (size_t)p * HD + DL * t4;
+#pragma unroll
+            for (int q = 0; q < NW / 4; ++q)
+                dst[q] = p < p_end ? *reinterpret_cast<const uint4 *>(src + 8 * q) : make_uint4(0u, 0u, 0u, 0u);
+        };
+        float sc[NT][2];                                     // scores of (row g8, positions 8 nt + 2 t4 + {0, 1})
+        {
+            uint4 kb[2][NW / 4];
+            load_k(0, kb[0]);
+            load_k(1, kb[1]);
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                uint4(&kq)[NW / 4] = kb[nt & 1];
+                float ch[4] = {0.f, 0.f, 0.f, 0.f}, cl[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int q = 0; q < NW / 4; ++q) {
+                    mma_rows8(cl, ql[4 * q], ql[4 * q + 1], kq[q].x, kq[q].y);
+                    mma_rows8(ch, qh[4 * q], qh[4 * q + 1], kq[q].x, kq[q].y);
+                    mma_rows8(cl, ql[4 * q + 2], ql[4 * q + 3], kq[q].z, kq[q].w);
+                    mma_rows8(ch, qh[4 * q + 2], qh[4 * q + 3], kq[q].z, kq[q].w);
+                }
+                sc[nt][0] = cl[0] + ch[0];
+                sc[nt][1] = cl[1] + ch[1];
+                if (nt + 2 < NT) load_k(nt + 2, kq);
+            }
+        }
+        auto load_v = [&](int nt, uint4 (&dst)[2][(VW + 3) / 4]) {
+#pragma unroll
+            for (int rr = 0; rr < 2; ++rr) {
+                const int p = p_begin + 8 * nt + 2 * t4 + rr;
+                const bf16_t *src = vbase + (size_t)p * HD + 2 * VW * g8;
+                if (VW >= 4) {
+#pragma unroll
+                    for (int q = 0; q < VW / 4; ++q)
+                        dst[rr][q] = p < p_end ? *reinterpret_cast<const uint4 *>(src + 8 * q) : make_uint4(0u, 0u, 0u, 0u);
+                } else {
+                    const uint2 v = p < p_end ? *reinterpret_cast<const uint2 *>(src) : make_uint2(0u, 0u);
+                    dst[rr][0] = make_uint4(v.x, v.y, 0u, 0u);
+                }
+            }
+        };
+        uint4 vb[2][2][(VW + 3) / 4];
+        load_v(0, vb[0]);
+        load_v(1, vb[1]);
+
+        // ---- running softmax: new maximum, old sums and outputs rescaled ----
+        float mx = -INFINITY;
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int p = p_begin + 8 * nt + 2 * t4 + e;
+                sc[nt][e] = (live && p <= p_row) ? sc[nt][e] * scale : -INFINITY;
+                mx = fmaxf(mx, sc[nt][e]);
+            }
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+        const float m_new = fmaxf(m_run, mx);
+        const float f = m_run == -INFINITY ? 0.f : expf(m_run - m_new);
+        m_run = m_new;
+        l_run *= f;
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const float pj = sc[nt][e] == -INFINITY ? 0.f : expf(sc[nt][e] - m_new);
+                sc[nt][e] = pj;
+                l_run += pj;
+            }
+#pragma unroll
+        for (int j = 0; j < VJ; ++j) { o[j][0] *= f; o[j][1] *= f; }
+
+        // ---- o += p V ----
+#pragma unroll
+        for (int np = 0; np < NT; np += 2) {
+            uint32_t ah[2], al[2];
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                const uint32_t h0 = float_to_bf16_rne(sc[np + i][0]), h1 = float_to_bf16_rne(sc[np + i][1]);
+                const uint32_t l0 = float_to_bf16_rne(sc[np + i][0] - __uint_as_float(h0 << 16));
+                const uint32_t l1 = float_to_bf16_rne(sc[np + i][1] - __uint_as_float(h1 << 16));
+                ah[i] = pack_bf16(h0, h1);
+                al[i] = pack_bf16(l0, l1);
+            }
+#pragma unroll
+            for (int j = 0; j < VJ; ++j) {
+                const int wi = (j >> 1) & 3;
+                uint32_t b[2];
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+                    const uint4 &wa = vb[i][0][j / 8], &wb = vb[i][1][j / 8];
+                    const uint32_t xa = wi == 0 ? wa.x : wi == 1 ? wa.y : wi == 2 ? wa.z : wa.w;
+                    const uint32_t xb = wi == 0 ? wb.x : wi == 1 ? wb.y : wi == 2 ? wb.z : wb.w;
+                    b[i] = __byte_perm(xa, xb, (j & 1) ? 0x7632 : 0x5410);     // dimension j of the two positions' rows
+                }
+                mma_rows8(o[j], al[0], al[1], b[0], b[1]);
+                mma_rows8(o[j], ah[0], ah[1], b[0], b[1]);
+            }
+            if (np + 2 < NT) { load_v(np + 2, vb[0]); load_v(np + 3, vb[1]); }
+        }
+    }
+
+    // ---- row g8: dimensions DL t4 + j (o[j][0]) and DL t4 + VJ + j (o[j][1]), divided by the row's sum ----
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+    if (live) {
+        const size_t base = (size_t)t_row * ((size_t)H * HD) + (size_t)h * HD + DL * t4;
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            uint32_t hw[VJ / 2], lw[VJ / 2];
+#pragma unroll
+            for (int j = 0; j < VJ; j += 2) {
+                const float v0 = o[j][half] / l_run, v1 = o[j + 1][half] / l_run;
+                const uint32_t h0 = float_to_bf16_rne(v0), h1 = float_to_bf16_rne(v1);
+                hw[j >> 1] = pack_bf16(h0, h1);
+                lw[j >> 1] = pack_bf16(float_to_bf16_rne(v0 - __uint_as_float(h0 << 16)), float_to_bf16_rne(v1 - __uint_as_float(h1 << 16)));
+            }
+#pragma unroll
+            for (int w = 0; w < VJ / 2; w += 4) {
+                *reinterpret_cast<uint4 *>(out_hi + base + half * VJ + 2 * w) = make_uint4(hw[w], hw[w + 1], hw[w + 2], hw[w + 3]);
+                *reinterpret_cast<uint4 *>(out_lo + base + half * VJ + 2 * w) = make_uint4(lw[w], lw[w + 1], lw[w + 2], lw[w + 3]);
+            }
+        }
+    }
+}
+
+}  // namespace prefill
+}  // namespace knnssd

@@ -1,0 +1,76 @@
+// Host side of the tensor-core prompt pass: TMA tensor maps and the launches of prefill.cuh's kernels.
+#pragma once
+
+#include "prefill.cuh"
+
+#include <cuda_runtime.h>
+
+namespace knnssd {
+namespace prefill {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The driver's tensor-map encoder, looked up through the runtime (the library does not link against the driver).
+inline EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// Map of a row-major bf16 matrix [rows][cols] (cols a multiple of 64) read in boxes of 128 rows x 64 columns, 128-byte
+// swizzle; rows past the end read as zero.
+inline bool make_map(CUtensorMap *m, const void *base, size_t rows, size_t cols) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t gdim[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t gstride[1] = {(cuuint64_t)cols * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)BK, 128u};
+    const cuuint32_t estr[2] = {1u, 1u};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+inline bool gemm_attrs_once() {
+    static bool done = false, ok = false;
+    if (!done) {
+        done = true;
+        ok = cudaFuncSetAttribute(gemm_split_kernel<PF_STORE>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM) == cudaSuccess &&
+             cudaFuncSetAttribute(gemm_split_kernel<PF_ADD>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM) == cudaSuccess &&
+             cudaFuncSetAttribute(gemm_split_kernel<PF_SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM) == cudaSuccess;
+    }
+    return ok;
+}
+
+// One contraction over T rows.  `planes` = the activation map (hi rows [0, cap), lo rows [cap, 2 cap)); W0 (and W1 for
+// SwiGLU: W0 = gate, W1 = up) are [N][K] bf16.  Returns false if a tensor map could not be made.
+inline bool launch_gemm(const CUtensorMap &planes, int cap, const void *W0, const void *W1, int N, int K, int T, int epi, float *y,
+                        int ldy, int col0, bf16_t *out_hi, bf16_t *out_lo, int ldo, int *err, cudaStream_t s) {
+    if (!gemm_attrs_once()) return false;
+    CUtensorMap tb0, tb1;
+    if (!make_map(&tb0, W0, (size_t)N, (size_t)K)) return false;
+    if (epi == PF_SWIGLU) {
+        if (!make_map(&tb1, W1, (size_t)N, (size_t)K)) return false;
+    } else {
+        tb1 = tb0;
+    }
+    GemmArgs g{T, K, N, y, ldy, col0, out_hi, out_lo, ldo, err};
+    const int per = epi == PF_SWIGLU ? BN / 2 : BN;
+    const dim3 grid((T + BM - 1) / BM, (N + per - 1) / per);
+    if (epi == PF_STORE) gemm_split_kernel<PF_STORE><<<grid, GEMM_THREADS, GEMM_SMEM, s>>>(planes, tb0, tb1, g, cap);
+    else if (epi == PF_ADD) gemm_split_kernel<PF_ADD><<<grid, GEMM_THREADS, GEMM_SMEM, s>>>(planes, tb0, tb1, g, cap);
+    else gemm_split_kernel<PF_SWIGLU><<<grid, GEMM_THREADS, GEMM_SMEM, s>>>(planes, tb0, tb1, g, cap);
+    return true;
+}
+
+}  // namespace prefill
+}  // namespace knnssd
