@@ -76,6 +76,13 @@ struct knnssd_ctx {
     uint32_t *xs_x = nullptr, *xs_attn = nullptr, *xs_act = nullptr;   // pre-split activations (see LinPhase::xs)
     float *ssp = nullptr;                                              // [MAXM][n_sms] partial sums of squares of x rows
 
+    // tensor-core prompt pass (same eligibility as the pass kernel): activations of up to pf_cap rows
+    bool pf_ok = false;
+    int pf_cap = 0;                                          // rows per chunk, a multiple of 128
+    float *pf_x = nullptr, *pf_qkv = nullptr;                // residual stream [cap][d]; q, k, v [cap][nq + 2 nkv]
+    bf16_t *pf_ad = nullptr, *pf_aq = nullptr, *pf_af = nullptr;   // hi / lo planes [2][cap][d], [2][cap][nq], [2][cap][d_ff]
+    CUtensorMap pf_map_d{}, pf_map_q{}, pf_map_f{};
+
     // instrumentation
     long long launches = 0;
     bool time_linear = false;
@@ -427,7 +434,7 @@ void free_all(knnssd_ctx *c) {
                     c->anchor_inv_norm, c->cosines, c->amax_v, c->part_ml, c->rope_cs, c->pool_sum, c->inv_freq, c->chain,
                     c->target, c->prompt, c->out_tokens, c->accept_log, c->amax_i, c->flag, c->knn_out, c->state,
                     c->ops_full, c->ops_draft, c->bar, c->gabort, c->attn_cnt, c->amax_cnt, c->mpart_o, c->mamax_v, c->mpart_ml,
-                    c->mamax_i, c->trace, c->xs_x, c->xs_attn, c->xs_act, c->ssp};
+                    c->mamax_i, c->trace, c->xs_x, c->xs_attn, c->xs_act, c->ssp, c->pf_x, c->pf_qkv, c->pf_ad, c->pf_aq, c->pf_af};
     for (void *p : ptrs)
         if (p) cudaFree(p);
     if (c->pinned) cudaFreeHost(c->pinned);
@@ -449,6 +456,66 @@ float elapsed_ms(knnssd_ctx *c) {
     return ms;
 }
 
+// The prompt pass on the tensor cores: rows [t0, t0 + T) of the prompt at a time, every linear map one contraction
+// over all T rows.  Leaves K/V of all layers in the cache, the pooled numerator in pool_sum and the last row's greedy
+// token in chain[0].  Returns false if a tensor map could not be made.
+template <int HD>
+bool prefill_tensor(knnssd_ctx *c, int n) {
+    const knnssd_config &g = c->cfg;
+    const int d = g.d_model, H = g.n_heads, Hkv = g.n_kv_heads, F = g.d_ff, V = g.vocab;
+    const int nq = H * HD, nkv = Hkv * HD, ldq = nq + 2 * nkv, cap = c->pf_cap;
+    cudaStream_t s = c->stream;
+    int *err = stream_err_ptr();
+    const size_t layer_stride = (size_t)Hkv * g.max_seq * HD;
+    bool ok = true;
+    for (int t0 = 0; t0 < n && ok; t0 += cap) {
+        const int T = n - t0 < cap ? n - t0 : cap;
+        const bool last = t0 + T == n;
+        prefill::embed_rows_kernel<<<T, 256, 0, s>>>(reinterpret_cast<const bf16_t *>(c->tok_embed), c->prompt + t0, d, c->pf_x);
+        c->launches++;
+        for (int l = 0; l < g.n_layers && ok; ++l) {
+            const Layer &ly = c->layers[l];
+            bf16_t *kc = reinterpret_cast<bf16_t *>(c->kcache) + (size_t)l * layer_stride;
+            bf16_t *vc = reinterpret_cast<bf16_t *>(c->vcache) + (size_t)l * layer_stride;
+            prefill::norm_split_kernel<<<T, 256, 0, s>>>(c->pf_x, d, ly.attn_norm, g.rms_eps, c->pf_ad, c->pf_ad + (size_t)cap * d);
+            ok = ok && prefill::launch_gemm(c->pf_map_d, cap, ly.wq, nullptr, nq, d, T, prefill::PF_STORE, c->pf_qkv, ldq, 0, nullptr,
+                                            nullptr, 0, err, s);
+            ok = ok && prefill::launch_gemm(c->pf_map_d, cap, ly.wk, nullptr, nkv, d, T, prefill::PF_STORE, c->pf_qkv, ldq, nq, nullptr,
+                                            nullptr, 0, err, s);
+            ok = ok && prefill::launch_gemm(c->pf_map_d, cap, ly.wv, nullptr, nkv, d, T, prefill::PF_STORE, c->pf_qkv, ldq, nq + nkv,
+                                            nullptr, nullptr, 0, err, s);
+            prefill::rope_kv_rows_kernel<<<dim3(H + 2 * Hkv, T), HD / 2, 0, s>>>(c->pf_qkv, H, Hkv, HD, c->inv_freq, kc, vc, g.max_seq, t0);
+            prefill::attn_prompt_kernel<HD><<<dim3((T + 7) / 8, (H + 3) / 4), 128, 0, s>>>(c->pf_qkv, H, Hkv, kc, vc, g.max_seq, t0, T,
+                                                                                           c->pf_aq, c->pf_aq + (size_t)cap * nq);
+            ok = ok && prefill::launch_gemm(c->pf_map_q, cap, ly.wo, nullptr, d, nq, T, prefill::PF_ADD, c->pf_x, d, 0, nullptr, nullptr, 0,
+                                            err, s);
+            prefill::norm_split_kernel<<<T, 256, 0, s>>>(c->pf_x, d, ly.mlp_norm, g.rms_eps, c->pf_ad, c->pf_ad + (size_t)cap * d);
+            ok = ok && prefill::launch_gemm(c->pf_map_d, cap, ly.w_gate, ly.w_up, F, d, T, prefill::PF_SWIGLU, nullptr, 0, 0, c->pf_af,
+                                            c->pf_af + (size_t)cap * F, F, err, s);
+            ok = ok && prefill::launch_gemm(c->pf_map_f, cap, ly.w_down, nullptr, d, F, T, prefill::PF_ADD, c->pf_x, d, 0, nullptr, nullptr,
+                                            0, err, s);
+            c->launches += 11;
+        }
+        // pooled numerator: every row's final hidden state (mean pooling) or the last row's
+        if (g.pool_mode == 0) {
+            rmsnorm_rows_kernel<<<T, 256, 0, s>>>(c->pf_x, c->final_norm, d, g.rms_eps, c->pf_qkv);     // [T][d] scratch
+            pool_accumulate_kernel<<<(d + 255) / 256, 256, 0, s>>>(c->pf_qkv, T, d, c->pool_sum, t0 == 0);
+            c->launches += 2;
+        } else if (last) {
+            rmsnorm_rows_kernel<<<1, 256, 0, s>>>(c->pf_x + (size_t)(T - 1) * d, c->final_norm, d, g.rms_eps, c->hfinal);
+            pool_accumulate_kernel<<<(d + 255) / 256, 256, 0, s>>>(c->hfinal, 1, d, c->pool_sum, 1);
+            c->launches += 2;
+        }
+        if (last) {
+            ctx_linear(c, make_args(c->lm_head, V, d, c->pf_x + (size_t)(T - 1) * d, c->final_norm, g.rms_eps, c->logits, EPI_STORE, 1));
+            argmax_partial_kernel<<<dim3(kArgmaxBlocks, 1), 256, 0, s>>>(c->logits, V, kArgmaxBlocks, c->amax_v, c->amax_i);
+            argmax_final_kernel<<<1, 32, 0, s>>>(c->amax_v, c->amax_i, kArgmaxBlocks, c->chain);
+            c->launches += 2;
+        }
+    }
+    return ok;
+}
+
 knnssd_status do_prefill(knnssd_ctx *c, const int *tokens_host, int n, float *pooled_dev, int *first_token) {
     const knnssd_config &g = c->cfg;
     if (!tokens_host || n < 1) return fail(c, KNNSSD_ERR_INVALID_ARG, "prefill: need at least one prompt token");
@@ -463,7 +530,13 @@ knnssd_status do_prefill(knnssd_ctx *c, const int *tokens_host, int n, float *po
     cudaEventRecord(c->ev0, s);
     const int d = g.d_model;
     const int chunk = c->mega_ok ? pass::MAXM : kMaxRows;   // rows per pass: what the faster path takes
-    for (int t0 = 0; t0 < n; t0 += chunk) {
+    // prompts longer than one pass's rows go through the tensor-core prompt pass where the model is eligible for it
+    const bool tensor_path = c->pf_ok && n > pass::MAXM;
+    if (tensor_path) {
+        const bool made = g.head_dim == 128 ? prefill_tensor<128>(c, n) : prefill_tensor<64>(c, n);
+        if (!made) { cudaStreamSynchronize(s); return fail(c, KNNSSD_ERR_CUDA, "prefill: cannot encode a tensor map"); }
+    }
+    for (int t0 = 0; t0 < n && !tensor_path; t0 += chunk) {
         const int M = (n - t0 < chunk) ? n - t0 : chunk;
         const bool last = t0 + M == n;
         // mean pooling needs every row's final hidden state; last-token pooling only the last row's
@@ -656,6 +729,25 @@ knnssd_status knnssd_init(const knnssd_config *cfg, const knnssd_weights *w, con
         ok2 &= dev_alloc(&c->xs_act, (size_t)pass::MAXM * (g.d_ff / 128) * stream::SLOT_WORDS) == cudaSuccess;
         ok2 &= dev_alloc(&c->ssp, (size_t)pass::MAXM * c->n_sms) == cudaSuccess;
         if (!ok2) { cudaGetLastError(); return bail(KNNSSD_ERR_CUDA); }
+        // tensor-core prompt pass: needs the driver's tensor-map encoder; without it prompts go through the pass kernel
+        if (prefill::encode_tiled_fn() && prefill::gemm_attrs_once()) {
+            const int cap_seq = (g.max_seq + prefill::BM - 1) / prefill::BM * prefill::BM;
+            c->pf_cap = cap_seq < 1024 ? cap_seq : 1024;
+            const size_t cap = (size_t)c->pf_cap;
+            bool ok3 = true;
+            ok3 &= dev_alloc(&c->pf_x, cap * d) == cudaSuccess;
+            ok3 &= dev_alloc(&c->pf_qkv, cap * (nq + 2 * nkv)) == cudaSuccess;
+            ok3 &= dev_alloc(&c->pf_ad, 2 * cap * d) == cudaSuccess;
+            ok3 &= dev_alloc(&c->pf_aq, 2 * cap * nq) == cudaSuccess;
+            ok3 &= dev_alloc(&c->pf_af, 2 * cap * g.d_ff) == cudaSuccess;
+            if (!ok3) { cudaGetLastError(); return bail(KNNSSD_ERR_CUDA); }
+            cudaMemsetAsync(c->pf_ad, 0, 2 * cap * d * sizeof(bf16_t), c->stream);
+            cudaMemsetAsync(c->pf_aq, 0, 2 * cap * nq * sizeof(bf16_t), c->stream);
+            cudaMemsetAsync(c->pf_af, 0, 2 * cap * g.d_ff * sizeof(bf16_t), c->stream);
+            c->pf_ok = prefill::make_map(&c->pf_map_d, c->pf_ad, 2 * cap, (size_t)d) &&
+                       prefill::make_map(&c->pf_map_q, c->pf_aq, 2 * cap, (size_t)nq) &&
+                       prefill::make_map(&c->pf_map_f, c->pf_af, 2 * cap, (size_t)g.d_ff);
+        }
         pass::Model &md = c->model;
         md.tok_embed = reinterpret_cast<const bf16_t *>(c->tok_embed); md.final_norm = c->final_norm; md.rms_eps = g.rms_eps;
         md.d_model = d; md.H = g.n_heads; md.Hkv = g.n_kv_heads; md.hd = hd; md.vocab = g.vocab; md.max_seq = g.max_seq;

@@ -250,6 +250,8 @@ SHAPES: Dict[str, ModelShape] = {
     "gqa-bf16": ModelShape("gqa-bf16", 2, 512, 8, 2, 64, 1384, 2056, "bf16", 1e-6, 1000000.0),
     # every linear of this one has n_in % 128 == 0 (the streaming kernel's path), ragged row counts, two column tiles
     "stream-bf16": ModelShape("stream-bf16", 3, 768, 6, 2, 128, 1920, 3001, "bf16", 1e-5, 10000.0),
+    # the same with 64-wide heads and four query heads per K/V head
+    "stream64-bf16": ModelShape("stream64-bf16", 2, 512, 8, 2, 64, 1408, 2056, "bf16", 1e-6, 1000000.0),
     "gqa-fp32": ModelShape("gqa-fp32", 2, 256, 4, 2, 64, 688, 520, "fp32", 1e-6, 1000000.0),
 }
 

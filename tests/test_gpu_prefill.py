@@ -98,3 +98,102 @@ def test_gemm_rejects_bad_arguments(kb):
     with pytest.raises(kb.KnnssdError) as e:
         kb.knnssd_gemm_split(torch.zeros((16, 128), dtype=torch.bfloat16, device="cuda"), x, 2)   # SwiGLU without W1
     assert e.value.status == 1
+
+
+# ---- the whole prompt pass ---------------------------------------------------------------------------
+
+TOL = 2e-2          # bf16 weights and K/V: the tolerance of the decode-path tests
+
+
+def _to_dev(w):
+    return {k: ([t.cuda() for t in v] if isinstance(v, list) else v.cuda()) for k, v in w.items()}
+
+
+def _pair(kb, shape_name, max_seq, max_draft=8, pool_mode=0, damp=None):
+    shape = si.SHAPES[shape_name]
+    w = si.make_model_weights(shape, 0, gain_spread=0.1, damp=damp)
+    om = oracle.OracleModel(shape, w, max_seq)
+    sess = kb.Session.from_shape(shape, _to_dev(w), max_seq, max_draft=max_draft, pool_mode=pool_mode)
+    return shape, om, sess
+
+
+# prompt lengths: just past one pass's rows, one ragged tile, two tiles and a tail, three tiles exactly
+@pytest.mark.parametrize("prompt_len", [17, 100, 300, 384])
+@pytest.mark.parametrize("shape_name", ["stream-bf16", "stream64-bf16"])
+def test_prompt_pass_matches_oracle(kb, shape_name, prompt_len):
+    """First token and pooled state of the prompt pass, then - reading the K/V cache it left - the logits and final
+    hidden states of a verification pass over forced rows, and the tokens generated from there."""
+    shape, om, sess = _pair(kb, shape_name, prompt_len + 80)
+    prompt = si.uniform_tokens(5, 0, prompt_len, shape.vocab).numpy()
+    pooled_o, first_o, _ = om.prefill(prompt)
+    first_g, pooled_g = sess.prefill(prompt, want_pooled=True)
+    assert first_g == first_o
+    assert np.abs(pooled_g.cpu().numpy() - pooled_o).max() < TOL
+    rows = si.uniform_tokens(6, 1, 7, shape.vocab).numpy()
+    o = om.forward(np.concatenate([[first_o], rows]).astype(np.int32), prompt_len, want_hidden=True)
+    sess.set_skipmask(np.zeros(2 * shape.n_layers, dtype=np.uint8))
+    g = sess.verify(rows, want_logits=True, want_hidden=True)
+    assert np.abs(g["logits"].cpu().numpy() - o["logits"]).max() < TOL
+    assert np.abs(g["hidden"].cpu().numpy() - o["hidden"]).max() < TOL
+    a, nxt = oracle.accept(rows, o["argmax"])
+    assert (g["n_accepted"], g["next_token"]) == (a, nxt)
+
+
+@pytest.mark.parametrize("shape_name", ["stream-bf16", "stream64-bf16"])
+def test_generate_after_a_long_prompt_matches_oracle_exactly(kb, shape_name):
+    base = si.SHAPES[shape_name]
+    mask = si.skip_mask(0, 2 * base.n_layers, 2)
+    damp = {int(j): 0.05 for j in np.nonzero(mask)[0]}
+    shape, om, sess = _pair(kb, shape_name, 300, damp=damp)
+    prompt = si.uniform_tokens(2, 0, 200, shape.vocab).numpy()
+    _, first, _ = om.prefill(prompt)
+    want = om.generate(first, 40, 4, mask)
+    sess.set_skipmask(mask)
+    got = sess.generate(prompt, 40, 4)
+    assert np.array_equal(got["tokens"], want["tokens"]), f"oracle min margin {want['min_margin']}"
+    assert np.array_equal(got["accepts"], want["accepts"])
+
+
+def test_prompt_longer_than_one_chunk(kb):
+    """More than 1024 prompt rows: the second chunk's attention reads the first chunk's K/V from the cache."""
+    shape, om, sess = _pair(kb, "stream64-bf16", 1200)
+    prompt = si.uniform_tokens(3, 0, 1100, shape.vocab).numpy()
+    pooled_o, first_o, _ = om.prefill(prompt)
+    first_g, pooled_g = sess.prefill(prompt, want_pooled=True)
+    assert first_g == first_o
+    assert np.abs(pooled_g.cpu().numpy() - pooled_o).max() < TOL
+    o = om.forward(np.array([first_o], dtype=np.int32), 1100)
+    sess.set_skipmask(np.zeros(2 * shape.n_layers, dtype=np.uint8))
+    g = sess.verify(np.zeros(0, dtype=np.int32), want_logits=True)
+    assert np.abs(g["logits"].cpu().numpy() - o["logits"]).max() < TOL
+    assert g["next_token"] == int(o["argmax"][0])
+
+
+def test_last_token_pooling_after_the_prompt_pass(kb):
+    shape, om, sess = _pair(kb, "stream-bf16", 200, pool_mode=1)
+    prompt = si.uniform_tokens(4, 0, 90, shape.vocab).numpy()
+    _, first_o, _ = om.prefill(prompt)
+    first_g, pooled_g = sess.prefill(prompt, want_pooled=True)
+    assert first_g == first_o
+    h = om.forward(prompt[-1:], 89, want_hidden=True, want_logits=False)["hidden"][0]   # K/V of rows 0..88 are in place
+    assert np.abs(pooled_g.cpu().numpy() - h).max() < TOL
+
+
+def test_sixteen_row_pass_matches_oracle(kb):
+    """The widest pass the decode kernel takes (two blocks of 8 rows): 15 forced rows after the pending token."""
+    shape, om, sess = _pair(kb, "stream-bf16", 120, max_draft=15)
+    prompt = si.uniform_tokens(0, 0, 37, shape.vocab).numpy()
+    _, first_o, _ = om.prefill(prompt)
+    assert sess.prefill(prompt) == first_o
+    sess.set_skipmask(np.zeros(2 * shape.n_layers, dtype=np.uint8))
+    for n_rows in (15, 9):
+        rows = si.uniform_tokens(7, n_rows, n_rows, shape.vocab).numpy()
+        n = sess.length
+        om.length = n                                       # rows the last verification rejected are dead
+        o = om.forward(np.concatenate([[first_o], rows]).astype(np.int32), n, want_hidden=True)
+        g = sess.verify(rows, want_logits=True, want_hidden=True)
+        assert np.abs(g["logits"].cpu().numpy() - o["logits"]).max() < TOL
+        assert np.abs(g["hidden"].cpu().numpy() - o["hidden"]).max() < TOL
+        a, nxt = oracle.accept(rows, o["argmax"])
+        assert (g["n_accepted"], g["next_token"]) == (a, nxt)
+        first_o = nxt                                       # the pending token of the next round
