@@ -479,21 +479,21 @@ bool prefill_tensor(knnssd_ctx *c, int n) {
             bf16_t *vc = reinterpret_cast<bf16_t *>(c->vcache) + (size_t)l * layer_stride;
             prefill::norm_split_kernel<<<T, 256, 0, s>>>(c->pf_x, d, ly.attn_norm, g.rms_eps, c->pf_ad, c->pf_ad + (size_t)cap * d);
             ok = ok && prefill::launch_gemm(c->pf_map_d, cap, ly.wq, nullptr, nq, d, T, prefill::PF_STORE, c->pf_qkv, ldq, 0, nullptr,
-                                            nullptr, 0, err, s);
+                                            nullptr, 0, err, c->n_sms, s);
             ok = ok && prefill::launch_gemm(c->pf_map_d, cap, ly.wk, nullptr, nkv, d, T, prefill::PF_STORE, c->pf_qkv, ldq, nq, nullptr,
-                                            nullptr, 0, err, s);
+                                            nullptr, 0, err, c->n_sms, s);
             ok = ok && prefill::launch_gemm(c->pf_map_d, cap, ly.wv, nullptr, nkv, d, T, prefill::PF_STORE, c->pf_qkv, ldq, nq + nkv,
-                                            nullptr, nullptr, 0, err, s);
+                                            nullptr, nullptr, 0, err, c->n_sms, s);
             prefill::rope_kv_rows_kernel<<<dim3(H + 2 * Hkv, T), HD / 2, 0, s>>>(c->pf_qkv, H, Hkv, HD, c->inv_freq, kc, vc, g.max_seq, t0);
             prefill::attn_prompt_kernel<HD><<<dim3((T + 7) / 8, (H + 3) / 4), 128, 0, s>>>(c->pf_qkv, H, Hkv, kc, vc, g.max_seq, t0, T,
                                                                                            c->pf_aq, c->pf_aq + (size_t)cap * nq);
             ok = ok && prefill::launch_gemm(c->pf_map_q, cap, ly.wo, nullptr, d, nq, T, prefill::PF_ADD, c->pf_x, d, 0, nullptr, nullptr, 0,
-                                            err, s);
+                                            err, c->n_sms, s);
             prefill::norm_split_kernel<<<T, 256, 0, s>>>(c->pf_x, d, ly.mlp_norm, g.rms_eps, c->pf_ad, c->pf_ad + (size_t)cap * d);
             ok = ok && prefill::launch_gemm(c->pf_map_d, cap, ly.w_gate, ly.w_up, F, d, T, prefill::PF_SWIGLU, nullptr, 0, 0, c->pf_af,
-                                            c->pf_af + (size_t)cap * F, F, err, s);
+                                            c->pf_af + (size_t)cap * F, F, err, c->n_sms, s);
             ok = ok && prefill::launch_gemm(c->pf_map_f, cap, ly.w_down, nullptr, d, F, T, prefill::PF_ADD, c->pf_x, d, 0, nullptr, nullptr,
-                                            0, err, s);
+                                            0, err, c->n_sms, s);
             c->launches += 11;
         }
         // pooled numerator: every row's final hidden state (mean pooling) or the last row's
@@ -744,9 +744,9 @@ knnssd_status knnssd_init(const knnssd_config *cfg, const knnssd_weights *w, con
             cudaMemsetAsync(c->pf_ad, 0, 2 * cap * d * sizeof(bf16_t), c->stream);
             cudaMemsetAsync(c->pf_aq, 0, 2 * cap * nq * sizeof(bf16_t), c->stream);
             cudaMemsetAsync(c->pf_af, 0, 2 * cap * g.d_ff * sizeof(bf16_t), c->stream);
-            c->pf_ok = prefill::make_map(&c->pf_map_d, c->pf_ad, 2 * cap, (size_t)d) &&
-                       prefill::make_map(&c->pf_map_q, c->pf_aq, 2 * cap, (size_t)nq) &&
-                       prefill::make_map(&c->pf_map_f, c->pf_af, 2 * cap, (size_t)g.d_ff);
+            c->pf_ok = prefill::make_map(&c->pf_map_d, c->pf_ad, 2 * cap, (size_t)d, prefill::BM) &&
+                       prefill::make_map(&c->pf_map_q, c->pf_aq, 2 * cap, (size_t)nq, prefill::BM) &&
+                       prefill::make_map(&c->pf_map_f, c->pf_af, 2 * cap, (size_t)g.d_ff, prefill::BM);
         }
         pass::Model &md = c->model;
         md.tok_embed = reinterpret_cast<const bf16_t *>(c->tok_embed); md.final_norm = c->final_norm; md.rms_eps = g.rms_eps;
@@ -1109,6 +1109,9 @@ knnssd_status knnssd_gemm_split(const void *W0_dev, const void *W1_dev, int n_ou
         (reinterpret_cast<uintptr_t>(y_dev) & 15u))
         return KNNSSD_ERR_SHAPE;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+    int dev = 0, n_sms = 148;
+    if (cudaGetDevice(&dev) != cudaSuccess) return KNNSSD_ERR_CUDA;
+    cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev);
     const int cap = (T + prefill::BM - 1) / prefill::BM * prefill::BM;
     bf16_t *planes = nullptr, *outp = nullptr;
     const size_t plane = (size_t)cap * n_in, oplane = (size_t)T * n_out;
@@ -1118,9 +1121,9 @@ knnssd_status knnssd_gemm_split(const void *W0_dev, const void *W1_dev, int n_ou
     cudaMemsetAsync(planes, 0, 2 * plane * sizeof(bf16_t), s);
     prefill::split_rows_kernel<<<T, 256, 0, s>>>(x_dev, n_in, planes, planes + plane);
     CUtensorMap ta;
-    if (!prefill::make_map(&ta, planes, (size_t)2 * cap, (size_t)n_in) ||
+    if (!prefill::make_map(&ta, planes, (size_t)2 * cap, (size_t)n_in, prefill::BM) ||
         !prefill::launch_gemm(ta, cap, W0_dev, W1_dev, n_out, n_in, T, mode, y_dev, n_out, 0, outp, outp ? outp + oplane : nullptr,
-                              n_out, stream_err_ptr(), s))
+                              n_out, stream_err_ptr(), n_sms, s))
         st = KNNSSD_ERR_CUDA;
     if (st == KNNSSD_OK && mode == 2) prefill::join_planes_kernel<<<T, 256, 0, s>>>(outp, outp + oplane, n_out, y_dev);
     cudaError_t e = cudaStreamSynchronize(s);

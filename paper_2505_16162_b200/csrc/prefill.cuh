@@ -30,12 +30,14 @@ using stream::mbar_try_wait;
 using stream::smem_u32;
 
 constexpr int BM = 128;                               // tokens per tile: rows of the accumulator = lanes of tensor memory
-constexpr int BN = 256;                               // accumulator columns per tile: two boxes of 128 weight rows
+constexpr int BN_MAX = 320;                           // most accumulator columns per tile (a launch picks 128, 192, 256 or 320)
+constexpr int BOX_N = 64;                             // weight rows per TMA box
 constexpr int BK = 64;                                // input columns per stage: 128 bytes of bf16 = one swizzle row
 constexpr int STAGES = 3;
 constexpr int A_BYTES = BM * BK * 2;                  // one term of the activation tile
-constexpr int B_BYTES = BN * BK * 2;
+constexpr int B_BYTES = BN_MAX * BK * 2;
 constexpr int STAGE_BYTES = 2 * A_BYTES + B_BYTES;    // hi plane, lo plane, weights
+constexpr int TMEM_COLS = 512;                        // columns of tensor memory a CTA takes (a power of two >= BN_MAX)
 constexpr int GEMM_THREADS = 192;                     // warp 0: TMA; warp 1: MMA issue + tensor-memory owner; warps 2..5: epilogue
 constexpr int GEMM_SMEM = STAGES * STAGE_BYTES + 1024 + 128;   // + slack to align the tiles to 1024 bytes + barriers
 constexpr unsigned WAIT_LIMIT = 4000000u;           // polls of one wait (a whole tile takes well under a millisecond)
@@ -46,6 +48,7 @@ struct GemmArgs {
     int T;             // live rows
     int K;             // input width, a multiple of BK
     int N;             // output units (per matrix)
+    int bn;            // accumulator columns per tile: a multiple of 64 (SwiGLU: of 128), at most BN_MAX
     float *y;          // STORE: y[t * ldy + col0 + n] = sum;  ADD: y[t * ldy + n] += sum
     int ldy, col0;
     bf16_t *out_hi;    // SWIGLU: silu(gate) * up as two bf16 planes, [t * ldo + n]
@@ -71,16 +74,18 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t saddr) {
 }
 // Instruction descriptor, kind::f16: fp32 accumulator (bits 4..5 = 1), A and B bf16 (bits 7..9 and 10..12 = 1), both
 // K-major (bits 15, 16 = 0), N / 8 in bits 17..22, M / 16 in bits 24..28.
-constexpr uint32_t UMMA_IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+__device__ __forceinline__ uint32_t umma_idesc(int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+}
 
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t accumulate) {
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
     asm volatile(
         "{\n\t"
         ".reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t"
         "}\n" ::"r"(tmem_d),
-        "l"(da), "l"(db), "r"(UMMA_IDESC), "r"(accumulate)
+        "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
         : "memory");
 }
 // The barrier gets one arrival once every MMA this thread issued before has finished.
@@ -123,10 +128,10 @@ __device__ __forceinline__ bool pf_wait(uint64_t *b, uint32_t parity, volatile i
 
 __device__ __forceinline__ uint32_t pack_bf16(uint32_t lo16, uint32_t hi16) { return lo16 | (hi16 << 16); }
 
-// One CTA per tile of 128 tokens x 256 accumulator columns.  EPI = PF_SWIGLU: columns 0..127 are units n0..n0+127 of
-// the gate matrix (map tb0) and columns 128..255 the same units of the up matrix (map tb1); otherwise the columns are
-// units n0..n0+255 of one matrix (tb0 = tb1).  ta covers both activation planes: rows [0, Tpad) the hi terms, rows
-// [Tpad, 2 Tpad) the lo terms.
+// One CTA per tile of 128 tokens x bn accumulator columns.  EPI = PF_SWIGLU: columns [0, bn / 2) are units n0 .. of
+// the gate matrix (map tb0) and columns [bn / 2, bn) the same units of the up matrix (map tb1); otherwise the columns
+// are units n0 .. n0 + bn - 1 of one matrix (tb0 = tb1).  ta covers both activation planes: rows [0, Tpad) the hi
+// terms, rows [Tpad, 2 Tpad) the lo terms.  The weight maps are read in boxes of BOX_N rows.
 template <int EPI>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_split_kernel(const __grid_constant__ CUtensorMap ta, const __grid_constant__ CUtensorMap tb0,
@@ -140,7 +145,8 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap ta, const __grid_constant_
     volatile int *cta_abort = reinterpret_cast<volatile int *>(tmem_slot + 1);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int t0 = blockIdx.x * BM;
-    const int n0 = blockIdx.y * (EPI == PF_SWIGLU ? BN / 2 : BN);
+    const int bn = g.bn, per = EPI == PF_SWIGLU ? bn / 2 : bn;      // units of a matrix per tile
+    const int n0 = blockIdx.y * per;
     const int nkb = g.K / BK;
 
     if (threadIdx.x == 0) {
@@ -151,7 +157,7 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap ta, const __grid_constant_
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(BN) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
@@ -168,11 +174,14 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap ta, const __grid_constant_
                 const uint32_t ph = (uint32_t)(kb / STAGES) & 1u;
                 if (!pf_wait(&empty[s], ph ^ 1u, cta_abort, g.err, 21)) break;
                 unsigned char *st = smem + s * STAGE_BYTES;
-                stream::mbar_expect_tx(&full[s], STAGE_BYTES);
+                stream::mbar_expect_tx(&full[s], 2 * A_BYTES + bn * BK * 2);
                 tma_load_2d(st, &ta, kb * BK, t0, &full[s]);
                 tma_load_2d(st + A_BYTES, &ta, kb * BK, Tpad + t0, &full[s]);
-                tma_load_2d(st + 2 * A_BYTES, &tb0, kb * BK, n0, &full[s]);
-                tma_load_2d(st + 2 * A_BYTES + B_BYTES / 2, &tb1, kb * BK, EPI == PF_SWIGLU ? n0 : n0 + BN / 2, &full[s]);
+                for (int j = 0; j < bn / BOX_N; ++j) {
+                    const int r = j * BOX_N;                 // accumulator column the box starts at
+                    const bool second = EPI == PF_SWIGLU && r >= per;
+                    tma_load_2d(st + 2 * A_BYTES + r * BK * 2, second ? &tb1 : &tb0, kb * BK, n0 + (second ? r - per : r), &full[s]);
+                }
                 armed = kb + 1;
             }
             if (*cta_abort) {
@@ -194,11 +203,20 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap ta, const __grid_constant_
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t a_hi = smem_u32(smem + s * STAGE_BYTES), a_lo = a_hi + A_BYTES, b = a_hi + 2 * A_BYTES;
+                // at most 256 columns per instruction: a wider tile takes a second one for the rest
+                const int n1 = bn < 256 ? bn : 256, n2 = bn - n1;
+                const uint32_t id1 = umma_idesc(n1), id2 = umma_idesc(n2 ? n2 : 16);
 #pragma unroll
                 for (int k = 0; k < BK / 16; ++k) {
-                    const uint64_t db = umma_desc(b + 32 * k);
-                    umma_bf16(tmem, umma_desc(a_hi + 32 * k), db, (kb | k) != 0 ? 1u : 0u);
-                    umma_bf16(tmem, umma_desc(a_lo + 32 * k), db, 1u);
+                    const uint32_t acc = (kb | k) != 0 ? 1u : 0u;
+                    const uint64_t db = umma_desc(b + 32 * k), dh = umma_desc(a_hi + 32 * k), dl = umma_desc(a_lo + 32 * k);
+                    umma_bf16(tmem, dh, db, id1, acc);
+                    umma_bf16(tmem, dl, db, id1, 1u);
+                    if (n2) {
+                        const uint64_t db2 = umma_desc(b + 256 * BK * 2 + 32 * k);
+                        umma_bf16(tmem + 256, dh, db2, id2, acc);
+                        umma_bf16(tmem + 256, dl, db2, id2, 1u);
+                    }
                 }
                 umma_commit(&empty[s]);
             }
@@ -214,10 +232,10 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap ta, const __grid_constant_
         const uint32_t trow = tmem + ((uint32_t)(32 * q) << 16);
         if (ok) {
             if (EPI == PF_SWIGLU) {
-                for (int c0 = 0; c0 < BN / 2 && n0 + c0 < g.N; c0 += 32) {
+                for (int c0 = 0; c0 < per && n0 + c0 < g.N; c0 += 32) {
                     float gt[32], up[32];
                     tmem_ld32(trow + c0, gt);
-                    tmem_ld32(trow + BN / 2 + c0, up);
+                    tmem_ld32(trow + per + c0, up);
                     if (t < g.T) {
                         uint32_t hi[16], lo[16];
 #pragma unroll
@@ -248,7 +266,7 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap ta, const __grid_constant_
                     }
                 }
             } else {
-                for (int c0 = 0; c0 < BN && n0 + c0 < g.N; c0 += 32) {
+                for (int c0 = 0; c0 < bn && n0 + c0 < g.N; c0 += 32) {
                     float v[32];
                     tmem_ld32(trow + c0, v);
                     if (t < g.T) {
@@ -275,7 +293,7 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap ta, const __grid_constant_
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(BN) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
     }
 }
 

@@ -27,14 +27,14 @@ inline EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
-// Map of a row-major bf16 matrix [rows][cols] (cols a multiple of 64) read in boxes of 128 rows x 64 columns, 128-byte
-// swizzle; rows past the end read as zero.
-inline bool make_map(CUtensorMap *m, const void *base, size_t rows, size_t cols) {
+// Map of a row-major bf16 matrix [rows][cols] (cols a multiple of 64) read in boxes of box_rows rows x 64 columns,
+// 128-byte swizzle; rows past the end read as zero.
+inline bool make_map(CUtensorMap *m, const void *base, size_t rows, size_t cols, int box_rows) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
     const cuuint64_t gdim[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
     const cuuint64_t gstride[1] = {(cuuint64_t)cols * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)BK, 128u};
+    const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1u, 1u};
     return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
@@ -51,20 +51,38 @@ inline bool gemm_attrs_once() {
     return ok;
 }
 
+// Accumulator columns per tile: all CTAs of a launch run at once on n_sms SMs, round after round, and a round takes
+// time in proportion to the tile's columns; the width with the fewest column-rounds wins (ties: the wider tile, which
+// re-reads the activations less).
+inline int pick_bn(int T, int N, bool swiglu, int n_sms) {
+    const int row_tiles = (T + BM - 1) / BM;
+    int best = 0;
+    long best_cost = 0;
+    for (int bn = 128; bn <= BN_MAX; bn += 64) {
+        if (swiglu && bn % 128) continue;
+        const int per = swiglu ? bn / 2 : bn;
+        const long ctas = (long)row_tiles * ((N + per - 1) / per);
+        const long cost = ((ctas + n_sms - 1) / n_sms) * bn;
+        if (!best || cost <= best_cost) { best = bn; best_cost = cost; }
+    }
+    return best;
+}
+
 // One contraction over T rows.  `planes` = the activation map (hi rows [0, cap), lo rows [cap, 2 cap)); W0 (and W1 for
 // SwiGLU: W0 = gate, W1 = up) are [N][K] bf16.  Returns false if a tensor map could not be made.
 inline bool launch_gemm(const CUtensorMap &planes, int cap, const void *W0, const void *W1, int N, int K, int T, int epi, float *y,
-                        int ldy, int col0, bf16_t *out_hi, bf16_t *out_lo, int ldo, int *err, cudaStream_t s) {
+                        int ldy, int col0, bf16_t *out_hi, bf16_t *out_lo, int ldo, int *err, int n_sms, cudaStream_t s) {
     if (!gemm_attrs_once()) return false;
     CUtensorMap tb0, tb1;
-    if (!make_map(&tb0, W0, (size_t)N, (size_t)K)) return false;
+    if (!make_map(&tb0, W0, (size_t)N, (size_t)K, BOX_N)) return false;
     if (epi == PF_SWIGLU) {
-        if (!make_map(&tb1, W1, (size_t)N, (size_t)K)) return false;
+        if (!make_map(&tb1, W1, (size_t)N, (size_t)K, BOX_N)) return false;
     } else {
         tb1 = tb0;
     }
-    GemmArgs g{T, K, N, y, ldy, col0, out_hi, out_lo, ldo, err};
-    const int per = epi == PF_SWIGLU ? BN / 2 : BN;
+    const int bn = pick_bn(T, N, epi == PF_SWIGLU, n_sms);
+    GemmArgs g{T, K, N, bn, y, ldy, col0, out_hi, out_lo, ldo, err};
+    const int per = epi == PF_SWIGLU ? bn / 2 : bn;
     const dim3 grid((T + BM - 1) / BM, (N + per - 1) / per);
     if (epi == PF_STORE) gemm_split_kernel<PF_STORE><<<grid, GEMM_THREADS, GEMM_SMEM, s>>>(planes, tb0, tb1, g, cap);
     else if (epi == PF_ADD) gemm_split_kernel<PF_ADD><<<grid, GEMM_THREADS, GEMM_SMEM, s>>>(planes, tb0, tb1, g, cap);

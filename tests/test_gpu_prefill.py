@@ -44,7 +44,10 @@ def _inputs(n_out, n_in, T, seed=3):
 # one tile; ragged rows and units (second weight box partly / wholly past the end, a column chunk cut short);
 # several row tiles; the 13B-shaped widths; one row
 GEMM_CASES = [(512, 256, 128), (1000, 320, 77), (136, 64, 5), (640, 1024, 300), (5120, 5120, 260), (264, 13824, 130),
-              (15360, 5120, 1)]
+              (15360, 5120, 1),
+              # tile widths other than 128 columns (the launch picks the width with the fewest column-rounds on the
+              # GPU's SMs): 192, 320 (two MMAs per step) and 256 on a 148-SM part
+              (5120, 256, 520), (5120, 256, 900), (4608, 256, 1024)]
 
 
 @pytest.mark.parametrize("n_out,n_in,T", GEMM_CASES)
@@ -64,7 +67,7 @@ def test_gemm_add_matches_oracle(kb, n_out, n_in, T):
     assert np.abs(got - want).max() < _tol(n_in, want)
 
 
-@pytest.mark.parametrize("n_out,n_in,T", [(1000, 320, 77), (13824, 5120, 140), (200, 256, 128)])
+@pytest.mark.parametrize("n_out,n_in,T", [(1000, 320, 77), (13824, 5120, 140), (200, 256, 128), (2304, 128, 1024)])
 def test_gemm_swiglu_matches_oracle(kb, n_out, n_in, T):
     Wg, x = _inputs(n_out, n_in, T)
     Wu = si.normal_weight(11, 80, n_out, n_in, 0.02, "bf16")
