@@ -53,6 +53,22 @@ def peaks():
     return 6650.0, "fallback"
 
 
+def prompt_pass_report(shape, rows, ms_list):
+    ms = sorted(ms_list)[len(ms_list) // 2]
+    d, hd = shape.d_model, shape.head_dim
+    weights = shape.n_layers * (2 * d * shape.n_heads * hd + 2 * d * shape.n_kv_heads * hd + 3 * d * shape.d_ff)
+    flop = 4.0 * rows * weights
+    out = {"rows": rows, "ms": ms, "linear_tflops_executed": flop / ms / 1e9, "bound": "tensor"}
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            pk = json.load(f)
+        out["peak_bf16_tflops_sustained"] = pk.get("bf16_tflops_sustained")
+        if pk.get("bf16_tflops_sustained"):
+            out["frac_of_measured_sustained"] = out["linear_tflops_executed"] / pk["bf16_tflops_sustained"]
+    return out
+
+
 def pass_bytes(shape, mask, n_ctx, rows):
     """Algorithmic bytes of one pass: weights of the retained sublayers + LM head + K/V rows attended."""
     b = 2 if shape.dtype == "bf16" else 4
@@ -231,10 +247,12 @@ def run_ours(args):
     e2e_tokens = 0
     e2e_steps = max(1, min(args.steps, 2))
     rounds_e2e = 0
+    prefill_ms = []
     for _ in range(e2e_steps):
         rr = sess.generate(prompt, max_new, k, use_selection=True)
         e2e_tokens += len(rr["tokens"])
         rounds_e2e += rr["stats"]["rounds"]
+        prefill_ms.append(rr["stats"]["ms_prefill"])
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - te
 
@@ -294,6 +312,9 @@ def run_ours(args):
         },
         "acceptance": {"mean_generated_length": M_len, "alpha": alpha, "rounds": stats["rounds"],
                        "expected_speedup_c_plain": metrics.expected_speedup(M_len, alpha, metrics.cost_coefficient(n_skip / (2 * shape.n_layers))) if alpha > 0 else None},
+        # the prompt pass inside the end-to-end steps (CUDA events around it): every linear map is one tensor-core
+        # contraction over all prompt rows, activations as two bf16 terms, so 4 x rows x weights FLOP are executed
+        "prompt_pass": prompt_pass_report(shape, P, prefill_ms),
         "setup_s": {"weights": t_weights},
         "clocks": clocks,
     }

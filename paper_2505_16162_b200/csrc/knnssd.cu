@@ -80,6 +80,7 @@ struct knnssd_ctx {
     bool pf_ok = false;
     int pf_cap = 0;                                          // rows per chunk, a multiple of 128
     float *pf_x = nullptr, *pf_qkv = nullptr;                // residual stream [cap][d]; q, k, v [cap][nq + 2 nkv]
+    float2 *pf_cs = nullptr;                                 // rotary (cos, sin) of the chunk's rows [cap][hd / 2]
     bf16_t *pf_ad = nullptr, *pf_aq = nullptr, *pf_af = nullptr;   // hi / lo planes [2][cap][d], [2][cap][nq], [2][cap][d_ff]
     CUtensorMap pf_map_d{}, pf_map_q{}, pf_map_f{};
 
@@ -434,7 +435,7 @@ void free_all(knnssd_ctx *c) {
                     c->anchor_inv_norm, c->cosines, c->amax_v, c->part_ml, c->rope_cs, c->pool_sum, c->inv_freq, c->chain,
                     c->target, c->prompt, c->out_tokens, c->accept_log, c->amax_i, c->flag, c->knn_out, c->state,
                     c->ops_full, c->ops_draft, c->bar, c->gabort, c->attn_cnt, c->amax_cnt, c->mpart_o, c->mamax_v, c->mpart_ml,
-                    c->mamax_i, c->trace, c->xs_x, c->xs_attn, c->xs_act, c->ssp, c->pf_x, c->pf_qkv, c->pf_ad, c->pf_aq, c->pf_af};
+                    c->mamax_i, c->trace, c->xs_x, c->xs_attn, c->xs_act, c->ssp, c->pf_x, c->pf_qkv, c->pf_ad, c->pf_aq, c->pf_af, c->pf_cs};
     for (void *p : ptrs)
         if (p) cudaFree(p);
     if (c->pinned) cudaFreeHost(c->pinned);
@@ -472,7 +473,8 @@ bool prefill_tensor(knnssd_ctx *c, int n) {
         const int T = n - t0 < cap ? n - t0 : cap;
         const bool last = t0 + T == n;
         prefill::embed_rows_kernel<<<T, 256, 0, s>>>(reinterpret_cast<const bf16_t *>(c->tok_embed), c->prompt + t0, d, c->pf_x);
-        c->launches++;
+        prefill::rope_table_kernel<<<T, HD / 2, 0, s>>>(c->inv_freq, t0, c->pf_cs);
+        c->launches += 2;
         for (int l = 0; l < g.n_layers && ok; ++l) {
             const Layer &ly = c->layers[l];
             bf16_t *kc = reinterpret_cast<bf16_t *>(c->kcache) + (size_t)l * layer_stride;
@@ -484,7 +486,7 @@ bool prefill_tensor(knnssd_ctx *c, int n) {
                                             nullptr, 0, err, c->n_sms, s);
             ok = ok && prefill::launch_gemm(c->pf_map_d, cap, ly.wv, nullptr, nkv, d, T, prefill::PF_STORE, c->pf_qkv, ldq, nq + nkv,
                                             nullptr, nullptr, 0, err, c->n_sms, s);
-            prefill::rope_kv_rows_kernel<<<dim3(H + 2 * Hkv, T), HD / 2, 0, s>>>(c->pf_qkv, H, Hkv, HD, c->inv_freq, kc, vc, g.max_seq, t0);
+            prefill::rope_kv_rows_kernel<<<dim3(H + 2 * Hkv, T), HD / 2, 0, s>>>(c->pf_qkv, H, Hkv, HD, c->pf_cs, kc, vc, g.max_seq, t0);
             prefill::attn_prompt_kernel<HD><<<dim3((T + 7) / 8, (H + 3) / 4), 128, 0, s>>>(c->pf_qkv, H, Hkv, kc, vc, g.max_seq, t0, T,
                                                                                            c->pf_aq, c->pf_aq + (size_t)cap * nq);
             ok = ok && prefill::launch_gemm(c->pf_map_q, cap, ly.wo, nullptr, d, nq, T, prefill::PF_ADD, c->pf_x, d, 0, nullptr, nullptr, 0,
@@ -737,6 +739,7 @@ knnssd_status knnssd_init(const knnssd_config *cfg, const knnssd_weights *w, con
             bool ok3 = true;
             ok3 &= dev_alloc(&c->pf_x, cap * d) == cudaSuccess;
             ok3 &= dev_alloc(&c->pf_qkv, cap * (nq + 2 * nkv)) == cudaSuccess;
+            ok3 &= dev_alloc(&c->pf_cs, cap * (hd / 2)) == cudaSuccess;
             ok3 &= dev_alloc(&c->pf_ad, 2 * cap * d) == cudaSuccess;
             ok3 &= dev_alloc(&c->pf_aq, 2 * cap * nq) == cudaSuccess;
             ok3 &= dev_alloc(&c->pf_af, 2 * cap * g.d_ff) == cudaSuccess;

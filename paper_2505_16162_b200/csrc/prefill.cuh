@@ -341,17 +341,24 @@ __global__ void __launch_bounds__(256) norm_split_kernel(const float *__restrict
     }
 }
 
+// (cos, sin) of the rotary angles of rows t = 0 .. T-1 at positions pos0 + t, once per chunk: all layers and heads
+// use the same table.  grid = T, hd / 2 threads.
+__global__ void rope_table_kernel(const double *__restrict__ inv_freq, int pos0, float2 *__restrict__ table) {
+    double sn, cs;
+    sincos((double)(pos0 + (int)blockIdx.x) * inv_freq[threadIdx.x], &sn, &cs);
+    table[(size_t)blockIdx.x * blockDim.x + threadIdx.x] = make_float2((float)cs, (float)sn);
+}
+
 // Rotary embedding of the q and k heads of row t at position pos0 + t (q in place, fp32); K and V rows rounded to
 // bf16 into the cache.  grid = (H + 2 Hkv, T), hd / 2 threads: thread i owns the pair (i, i + hd / 2).
-__global__ void rope_kv_rows_kernel(float *__restrict__ qkv, int H, int Hkv, int hd, const double *__restrict__ inv_freq,
+__global__ void rope_kv_rows_kernel(float *__restrict__ qkv, int H, int Hkv, int hd, const float2 *__restrict__ table,
                                     bf16_t *__restrict__ kc, bf16_t *__restrict__ vc, int max_seq, int pos0) {
     const int slot = blockIdx.x, t = blockIdx.y, i = threadIdx.x, half = hd / 2;
     float *row = qkv + (size_t)t * (H + 2 * Hkv) * hd + (size_t)slot * hd;
     const int pos = pos0 + t;
     if (slot < H + Hkv) {
-        double sn, cs;
-        sincos((double)pos * inv_freq[i], &sn, &cs);
-        const float c = (float)cs, s = (float)sn;
+        const float2 cs2 = table[(size_t)t * half + i];
+        const float c = cs2.x, s = cs2.y;
         const float a = row[i], b = row[i + half];
         const float ra = a * c - b * s, rb = b * c + a * s;
         if (slot < H) {

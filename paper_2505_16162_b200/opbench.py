@@ -9,6 +9,11 @@ Several copies of the matrix are cycled through so that every launch reads from 
 
 times the persistent pass kernel (rows 1 = a draft step under a seeded 45 % skip mask, rows k+1 = a verification pass)
 on a model of the named widths cut to ``--layers`` layers, small enough for a multi-pass profiler capture.
+
+    python -m paper_2505_16162_b200.opbench prompt --shape llama13b --layers 4 --context 1024 --iters 5
+
+times the tensor-core prompt pass (``knnssd_prefill``) over ``--context`` rows and prints the tensor-core rate of its
+linear maps (both bf16 terms of the activations counted: 4 x rows x weights FLOP).
 """
 from __future__ import annotations
 
@@ -73,9 +78,30 @@ def bench_pass(shape_name: str, layers: int, context: int, rows: int, iters: int
             "attention_sublayers": n_attn, "mlp_sublayers": n_mlp}
 
 
+def bench_prompt(shape_name: str, layers: int, rows: int, iters: int, seed: int = 0):
+    build.build()
+    from . import binding as kb
+    torch.cuda.set_device(0)
+    shape = si.SHAPES[shape_name].with_layers(layers)
+    w = si.make_model_weights(shape, seed, device="cuda")
+    sess = kb.Session.from_shape(shape, w, rows + 64, max_draft=8)
+    prompt = si.uniform_tokens(seed, 0, rows, shape.vocab).numpy()
+    ms = []
+    for _ in range(iters + 2):
+        sess.prefill(prompt)
+        ms.append(sess.get_stats()["ms_prefill"])         # CUDA events around the pass, on its stream
+    ms = sorted(ms[2:])
+    d, hd = shape.d_model, shape.head_dim
+    weights = layers * (2 * d * shape.n_heads * hd + 2 * d * shape.n_kv_heads * hd + 3 * d * shape.d_ff)
+    flop = 4.0 * rows * weights                             # 2 per multiply-add, two bf16 terms per activation
+    med = ms[len(ms) // 2]
+    return {"op": "prompt", "shape": shape.name, "rows": rows, "ms_per_pass": med, "ms_min": ms[0],
+            "linear_flop": flop, "tflops": flop / med / 1e9}
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("op", choices=["linear", "pass"])
+    ap.add_argument("op", choices=["linear", "pass", "prompt"])
     ap.add_argument("--shape", default="llama13b")
     ap.add_argument("--layers", type=int, default=4)
     ap.add_argument("--context", type=int, default=1280)
@@ -86,7 +112,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp32"])
     a = ap.parse_args()
-    if a.op == "pass":
+    if a.op == "prompt":
+        print(json.dumps(bench_prompt(a.shape, a.layers, a.context, a.iters)))
+    elif a.op == "pass":
         print(json.dumps(bench_pass(a.shape, a.layers, a.context, a.rows, a.iters)))
     else:
         print(json.dumps(bench_linear(a.n_out, a.n_in, a.rows, a.iters, a.warmup, a.dtype)))
