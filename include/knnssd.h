@@ -223,6 +223,29 @@ knnssd_status knnssd_gemm_split(const void *W0_dev, const void *W1_dev, int n_ou
                                 int mode, float *y_dev, void *cuda_stream);
 
 /*
+ * Anchor construction of the pre-inference stage (Sec. 4.1): K-means (Lloyd's iteration) over the sampled last
+ * hidden vectors with as many clusters as domains, then, per cluster, the k members nearest to its centroid (Eq. (2)).
+ * The paper does not say how K-means is started or stopped: the starting centroids are an argument, and the iteration
+ * stops when a round changes no assignment or after max_rounds rounds.  A round = assign every point to its nearest
+ * centroid (squared Euclidean distance, lowest index among equal distances), then move each centroid to the mean of
+ * its members (a centroid without members stays).  Distances, sums and centroids are fp64.
+ *   x_dev               DEVICE fp32 [n_points][d], row-major, 16-byte aligned; borrowed
+ *   init_centroids_dev  DEVICE fp32 [n_clusters][d]
+ *   max_rounds >= 1, 1 <= k, 1 <= n_clusters <= 16 (more: KNNSSD_ERR_CAPACITY), n_points >= n_clusters
+ *   labels_host         HOST int32 [n_points]: the cluster of each point (NULL: not wanted)
+ *   centroids_out_dev   DEVICE fp64 [n_clusters][d] (NULL: not wanted)
+ *   anchors_host        HOST int32 [n_clusters][k]: point indices, nearest first, lowest index first among equal
+ *                       distances; -1 where a cluster has fewer than k members
+ *   rounds_host         HOST: assignment rounds done (NULL: not wanted)
+ *   ms_rounds_host      HOST: device time of all rounds' kernels, CUDA events on the stream (NULL: not wanted)
+ * Allocates and frees its scratch; synchronises the stream.
+ */
+knnssd_status knnssd_build_anchors(const float *x_dev, int n_points, int d, int n_clusters,
+                                   const float *init_centroids_dev, int max_rounds, int k, int *labels_host,
+                                   double *centroids_out_dev, int *anchors_host, int *rounds_host, float *ms_rounds_host,
+                                   void *cuda_stream);
+
+/*
  * Cosine top-1 (Sec. 4.2, Eq. (4)) of one query against n anchors of dimension d, all DEVICE fp32; HOST outputs.
  * KNNSSD_ERR_DEGENERATE for a zero / non-finite query or anchor.
  */

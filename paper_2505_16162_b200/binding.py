@@ -23,7 +23,7 @@ STATUS = {0: "OK", 1: "ERR_INVALID_ARG", 2: "ERR_SHAPE", 3: "ERR_CAPACITY", 4: "
 EXPORTS = ["knnssd_init", "knnssd_destroy", "knnssd_prefill", "knnssd_select_skipset", "knnssd_set_skipmask",
            "knnssd_draft", "knnssd_verify", "knnssd_generate", "knnssd_decode", "knnssd_get_launch_count", "knnssd_get_length", "knnssd_set_length",
            "knnssd_set_pending", "knnssd_get_stats", "knnssd_last_error", "knnssd_time_pass", "knnssd_trace_pass", "knnssd_linear",
-           "knnssd_gemm_split", "knnssd_cosine_top1", "knnssd_cosine_top1_static"]
+           "knnssd_gemm_split", "knnssd_build_anchors", "knnssd_cosine_top1", "knnssd_cosine_top1_static"]
 
 
 class KnnssdError(RuntimeError):
@@ -77,6 +77,7 @@ def _load():
         "knnssd_trace_pass": (I, [P, I, I, I, PI, PI, PF, PF, PI]),
         "knnssd_linear": (I, [P, I, I, I, P, I, P, P]),
         "knnssd_gemm_split": (I, [P, P, I, I, P, I, I, P, P]),
+        "knnssd_build_anchors": (I, [P, I, I, I, P, I, I, P, P, P, PI, PF, P]),
         "knnssd_cosine_top1": (I, [P, P, I, I, PI, PF, P]),
         "knnssd_cosine_top1_static": (I, [P, P, I, I, PI, PF, P]),
     }
@@ -137,6 +138,24 @@ def knnssd_gemm_split(W0: torch.Tensor, x: torch.Tensor, mode: int = 0, W1: Opti
     if rc:
         raise KnnssdError(rc, "knnssd_gemm_split")
     return y
+
+
+def knnssd_build_anchors(x: torch.Tensor, init_centroids: torch.Tensor, max_rounds: int, k: int):
+    """Sec. 4.1: K-means over the rows of x (fp32 [N][d], CUDA) from ``init_centroids`` (fp32 [n][d]), then Eq. (2).
+    Returns dict(labels int32 [N], centroids fp64 CUDA [n][d], anchors int32 [n][k], rounds, ms_rounds)."""
+    N, d = x.shape
+    n = init_centroids.shape[0]
+    labels = np.zeros(N, dtype=np.int32)
+    anchors = np.zeros((n, k), dtype=np.int32)
+    mu = torch.empty((n, d), dtype=torch.float64, device=x.device)
+    rounds, ms = C.c_int(), C.c_float()
+    with torch.cuda.device(x.device):
+        rc = _lib.knnssd_build_anchors(_dev_ptr(x, torch.float32), N, d, n, _dev_ptr(init_centroids, torch.float32), max_rounds, k,
+                                       labels.ctypes.data, _dev_ptr(mu), anchors.ctypes.data, C.byref(rounds), C.byref(ms),
+                                       torch.cuda.current_stream().cuda_stream)
+    if rc:
+        raise KnnssdError(rc, "knnssd_build_anchors")
+    return {"labels": labels, "centroids": mu, "anchors": anchors, "rounds": rounds.value, "ms_rounds": ms.value}
 
 
 def knnssd_cosine_top1(query: torch.Tensor, anchors: torch.Tensor):

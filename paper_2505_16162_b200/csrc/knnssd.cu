@@ -6,6 +6,7 @@
 #include "linear_stream.cuh"
 #include "pass_kernel.cuh"
 #include "prefill_host.cuh"
+#include "anchors.cuh"
 
 #include <cmath>
 #include <cstdio>
@@ -1140,6 +1141,95 @@ knnssd_status knnssd_gemm_split(const void *W0_dev, const void *W1_dev, int n_ou
     cudaFree(planes);
     if (outp) cudaFree(outp);
     return st;
+}
+
+namespace {
+__global__ void widen_kernel(const float *__restrict__ a, size_t n, double *__restrict__ b) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) b[i] = (double)a[i];
+}
+}  // namespace
+
+knnssd_status knnssd_build_anchors(const float *x_dev, int n_points, int d, int n_clusters,
+                                   const float *init_centroids_dev, int max_rounds, int k, int *labels_host,
+                                   double *centroids_out_dev, int *anchors_host, int *rounds_host, float *ms_rounds_host,
+                                   void *cuda_stream) {
+    if (!x_dev || !init_centroids_dev || !anchors_host || n_points < 1 || d < 1 || n_clusters < 1 || max_rounds < 1 || k < 1 ||
+        n_points < n_clusters)
+        return KNNSSD_ERR_INVALID_ARG;
+    if (n_clusters > anchors::MAXC) return KNNSSD_ERR_CAPACITY;
+    if (reinterpret_cast<uintptr_t>(x_dev) & 15u) return KNNSSD_ERR_SHAPE;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+    const int N = n_points, n = n_clusters;
+    int S = (N + 63) / 64;                        // slices of the centroid sums: at least 64 points each, at most 64 slices
+    if (S > 64) S = 64;
+    const int per = (N + S - 1) / S;
+    double *mu = nullptr, *dist = nullptr, *part = nullptr;
+    int *labels = nullptr, *small = nullptr, *out = nullptr;     // small: [0] changed, [1 .. n] counts
+    unsigned char *taken = nullptr;
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    bool ok = dev_alloc(&mu, (size_t)n * d) == cudaSuccess && dev_alloc(&dist, (size_t)N) == cudaSuccess &&
+              dev_alloc(&part, (size_t)S * n * d) == cudaSuccess && dev_alloc(&labels, (size_t)N) == cudaSuccess &&
+              dev_alloc(&small, (size_t)n + 1) == cudaSuccess && dev_alloc(&out, (size_t)n * k) == cudaSuccess &&
+              dev_alloc(&taken, (size_t)N) == cudaSuccess && cudaEventCreate(&e0) == cudaSuccess &&
+              cudaEventCreate(&e1) == cudaSuccess;
+    auto cleanup = [&]() {
+        void *ptrs[] = {mu, dist, part, labels, small, out, taken};
+        for (void *p : ptrs)
+            if (p) cudaFree(p);
+        if (e0) cudaEventDestroy(e0);
+        if (e1) cudaEventDestroy(e1);
+    };
+    if (!ok) { cudaGetLastError(); cleanup(); return KNNSSD_ERR_CUDA; }
+    widen_kernel<<<(unsigned)(((size_t)n * d + 255) / 256), 256, 0, s>>>(init_centroids_dev, (size_t)n * d, mu);
+    cudaMemsetAsync(labels, 0xFF, sizeof(int) * N, s);           // -1: the first round changes every assignment
+    const dim3 cols((d + 255) / 256);
+    int rounds = 0, changed = 1;
+    float ms_total = 0.f;
+    cudaError_t e = cudaSuccess;
+    while (rounds < max_rounds && e == cudaSuccess) {
+        cudaMemsetAsync(small, 0, sizeof(int) * (n + 1), s);
+        cudaEventRecord(e0, s);
+        anchors::assign_kernel<<<(N + anchors::PTS - 1) / anchors::PTS, anchors::PTS * 32, 0, s>>>(x_dev, N, d, mu, n, 1, labels, dist,
+                                                                                                  small + 1, small);
+        cudaEventRecord(e1, s);
+        e = cudaMemcpyAsync(&changed, small, sizeof(int), cudaMemcpyDeviceToHost, s);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+        if (e != cudaSuccess) break;
+        float ms = 0.f;
+        cudaEventElapsedTime(&ms, e0, e1);
+        ms_total += ms;
+        ++rounds;
+        if (!changed) break;
+        cudaEventRecord(e0, s);
+        anchors::partial_sums_kernel<<<dim3(cols.x, S), 256, 0, s>>>(x_dev, N, d, labels, n, per, part);
+        anchors::fold_centroids_kernel<<<dim3(cols.x, n), 256, 0, s>>>(part, small + 1, n, d, S, mu);
+        cudaEventRecord(e1, s);
+        e = cudaStreamSynchronize(s);
+        if (e != cudaSuccess) break;
+        cudaEventElapsedTime(&ms, e0, e1);
+        ms_total += ms;
+    }
+    if (e == cudaSuccess) {
+        // the anchors are measured against the final centroids (they moved after the last assignment if the round
+        // limit ended the iteration)
+        if (changed)
+            anchors::assign_kernel<<<(N + anchors::PTS - 1) / anchors::PTS, anchors::PTS * 32, 0, s>>>(x_dev, N, d, mu, n, 0, labels, dist,
+                                                                                                      small + 1, small);
+        cudaMemsetAsync(taken, 0, (size_t)N, s);
+        anchors::select_anchors_kernel<<<n, 256, 0, s>>>(dist, labels, N, k, taken, out);
+        e = cudaMemcpyAsync(anchors_host, out, sizeof(int) * n * k, cudaMemcpyDeviceToHost, s);
+        if (e == cudaSuccess && labels_host) e = cudaMemcpyAsync(labels_host, labels, sizeof(int) * N, cudaMemcpyDeviceToHost, s);
+        if (e == cudaSuccess && centroids_out_dev)
+            e = cudaMemcpyAsync(centroids_out_dev, mu, sizeof(double) * n * d, cudaMemcpyDeviceToDevice, s);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+        if (e == cudaSuccess) e = cudaGetLastError();
+    }
+    cleanup();
+    if (e != cudaSuccess) { cudaGetLastError(); return KNNSSD_ERR_CUDA; }
+    if (rounds_host) *rounds_host = rounds;
+    if (ms_rounds_host) *ms_rounds_host = ms_total;
+    return KNNSSD_OK;
 }
 
 knnssd_status knnssd_cosine_top1(const float *query_dev, const float *anchors_dev, int n, int d, int *best, float *cosine,
