@@ -318,9 +318,35 @@ def run_ours(args):
         "setup_s": {"weights": t_weights},
         "clocks": clocks,
     }
+    if world == 1:
+        out["anchor_construction"] = anchor_construction_report(shape, args.seed, dev, peak, not args.no_cpu_baseline)
     if not args.no_cpu_baseline and world == 1:
         out["cpu_baseline"] = cpu_baseline(args, shape, w, masks[dom], steps=1, warmup=0, sess=sess)
     print(json.dumps(out))
+
+
+def anchor_construction_report(shape, seed, dev, hbm_peak, with_oracle):
+    """The pre-inference step that makes the anchors (not part of the timed decode step): K-means over N_DOMAINS x 1000
+    synthetic pooled vectors of the model's width from a start inside one domain, 10 anchors per cluster; device time
+    of the rounds' kernels, and the oracle's wall time on the same input with the results compared."""
+    per, k_anchor = 1000, 10
+    X = si.anchors(seed + 3, N_DOMAINS, per, shape.d_model, 0.5, normalise=False).to(dev)
+    init = X[:N_DOMAINS].contiguous()
+    res = [kb.knnssd_build_anchors(X, init, 50, k_anchor) for _ in range(5)]
+    ms = sorted(r["ms_rounds"] for r in res[2:])[1]
+    rounds = res[-1]["rounds"]
+    nbytes = X.numel() * 4 * (2 * (rounds - 1) + 1)          # a round reads the points twice; the last only assigns
+    out = {"points": int(X.shape[0]), "d": shape.d_model, "clusters": N_DOMAINS, "anchors_per_cluster": k_anchor, "rounds": rounds,
+           "ms_rounds": ms, "gbs": nbytes / ms / 1e6, "frac_of_hbm_peak": nbytes / ms / 1e6 / hbm_peak,
+           "note": "the points (102 MB at d = 5120) mostly stay in L2 between the two reads of a round"}
+    if with_oracle:
+        from oracle import anchors as oa
+        t0 = time.perf_counter()
+        want = oa.build_anchors(X.cpu().numpy(), init.cpu().numpy().astype(np.float64), 50, k_anchor)
+        out["oracle_s"] = time.perf_counter() - t0
+        out["gpu_matches_oracle"] = bool(np.array_equal(want["labels"], res[-1]["labels"]) and
+                                         np.array_equal(want["anchors"], res[-1]["anchors"]) and want["rounds"] == rounds)
+    return out
 
 
 def cpu_baseline(args, shape, w_dev, mask, steps, warmup, per_step=None, sess=None):

@@ -1184,14 +1184,21 @@ knnssd_status knnssd_build_anchors(const float *x_dev, int n_points, int d, int 
     widen_kernel<<<(unsigned)(((size_t)n * d + 255) / 256), 256, 0, s>>>(init_centroids_dev, (size_t)n * d, mu);
     cudaMemsetAsync(labels, 0xFF, sizeof(int) * N, s);           // -1: the first round changes every assignment
     const dim3 cols((d + 255) / 256);
+    const int agrid = (N + anchors::PTS - 1) / anchors::PTS;
+    const bool vec = d % 4 == 0;                                 // rows stay 16-byte aligned
+    auto launch_assign = [&](int relabel) {
+#define KNNSSD_ASSIGN(V, NC) anchors::assign_kernel<V, NC><<<agrid, 256, 0, s>>>(x_dev, N, d, mu, n, relabel, labels, dist, small + 1, small)
+        if (vec) { if (n <= 4) KNNSSD_ASSIGN(true, 4); else if (n <= 8) KNNSSD_ASSIGN(true, 8); else KNNSSD_ASSIGN(true, 16); }
+        else { if (n <= 4) KNNSSD_ASSIGN(false, 4); else if (n <= 8) KNNSSD_ASSIGN(false, 8); else KNNSSD_ASSIGN(false, 16); }
+#undef KNNSSD_ASSIGN
+    };
     int rounds = 0, changed = 1;
     float ms_total = 0.f;
     cudaError_t e = cudaSuccess;
     while (rounds < max_rounds && e == cudaSuccess) {
         cudaMemsetAsync(small, 0, sizeof(int) * (n + 1), s);
         cudaEventRecord(e0, s);
-        anchors::assign_kernel<<<(N + anchors::PTS - 1) / anchors::PTS, anchors::PTS * 32, 0, s>>>(x_dev, N, d, mu, n, 1, labels, dist,
-                                                                                                  small + 1, small);
+        launch_assign(1);
         cudaEventRecord(e1, s);
         e = cudaMemcpyAsync(&changed, small, sizeof(int), cudaMemcpyDeviceToHost, s);
         if (e == cudaSuccess) e = cudaStreamSynchronize(s);
@@ -1213,9 +1220,7 @@ knnssd_status knnssd_build_anchors(const float *x_dev, int n_points, int d, int 
     if (e == cudaSuccess) {
         // the anchors are measured against the final centroids (they moved after the last assignment if the round
         // limit ended the iteration)
-        if (changed)
-            anchors::assign_kernel<<<(N + anchors::PTS - 1) / anchors::PTS, anchors::PTS * 32, 0, s>>>(x_dev, N, d, mu, n, 0, labels, dist,
-                                                                                                      small + 1, small);
+        if (changed) launch_assign(0);
         cudaMemsetAsync(taken, 0, (size_t)N, s);
         anchors::select_anchors_kernel<<<n, 256, 0, s>>>(dist, labels, N, k, taken, out);
         e = cudaMemcpyAsync(anchors_host, out, sizeof(int) * n * k, cudaMemcpyDeviceToHost, s);

@@ -14,6 +14,12 @@ on a model of the named widths cut to ``--layers`` layers, small enough for a mu
 
 times the tensor-core prompt pass (``knnssd_prefill``) over ``--context`` rows and prints the tensor-core rate of its
 linear maps (both bf16 terms of the activations counted: 4 x rows x weights FLOP).
+
+    python -m paper_2505_16162_b200.opbench anchors --n-out 5 --rows 1000 --n-in 5120 --iters 10
+
+times anchor construction (``knnssd_build_anchors``: ``--n-out`` domains x ``--rows`` sampled vectors of width
+``--n-in``, 10 anchors each) from a start inside one domain, and prints the device time per K-means round and the
+rate at which a round reads the points (twice per round: assignment and centroid sums).
 """
 from __future__ import annotations
 
@@ -99,9 +105,28 @@ def bench_prompt(shape_name: str, layers: int, rows: int, iters: int, seed: int 
             "linear_flop": flop, "tflops": flop / med / 1e9}
 
 
+def bench_anchors(n_domains: int, per: int, d: int, iters: int, k: int = 10, seed: int = 3):
+    build.build()
+    from . import binding as kb
+    torch.cuda.set_device(0)
+    X = si.anchors(seed, n_domains, per, d, 0.5, normalise=False).cuda()
+    init = X[:n_domains].contiguous()                        # all from the first domain: several rounds
+    ms, rounds = [], 0
+    for _ in range(iters + 2):
+        r = kb.knnssd_build_anchors(X, init, 50, k)
+        ms.append(r["ms_rounds"])
+        rounds = r["rounds"]
+    ms = sorted(ms[2:])
+    med = ms[len(ms) // 2]
+    nbytes = 2.0 * X.numel() * 4 * (rounds - 1) + X.numel() * 4       # the last round only assigns
+    return {"op": "anchors", "points": X.shape[0], "d": d, "clusters": n_domains, "k": k, "rounds": rounds,
+            "ms_rounds": med, "ms_per_round": med / rounds, "algorithmic_bytes": nbytes, "gbs": nbytes / med / 1e6,
+            "points_bytes": X.numel() * 4}
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("op", choices=["linear", "pass", "prompt"])
+    ap.add_argument("op", choices=["linear", "pass", "prompt", "anchors"])
     ap.add_argument("--shape", default="llama13b")
     ap.add_argument("--layers", type=int, default=4)
     ap.add_argument("--context", type=int, default=1280)
@@ -112,7 +137,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp32"])
     a = ap.parse_args()
-    if a.op == "prompt":
+    if a.op == "anchors":
+        print(json.dumps(bench_anchors(a.n_out, a.rows, a.n_in, a.iters)))
+    elif a.op == "prompt":
         print(json.dumps(bench_prompt(a.shape, a.layers, a.context, a.iters)))
     elif a.op == "pass":
         print(json.dumps(bench_pass(a.shape, a.layers, a.context, a.rows, a.iters)))
