@@ -329,6 +329,7 @@ def anchor_construction_report(shape, seed, dev, hbm_peak, with_oracle):
     """The pre-inference step that makes the anchors (not part of the timed decode step): K-means over N_DOMAINS x 1000
     synthetic pooled vectors of the model's width from a start inside one domain, 10 anchors per cluster; device time
     of the rounds' kernels, and the oracle's wall time on the same input with the results compared."""
+    from paper_2505_16162_b200 import binding as kb
     per, k_anchor = 1000, 10
     X = si.anchors(seed + 3, N_DOMAINS, per, shape.d_model, 0.5, normalise=False).to(dev)
     init = X[:N_DOMAINS].contiguous()
