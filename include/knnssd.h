@@ -167,11 +167,29 @@ long long knnssd_get_launch_count(const knnssd_ctx *ctx);
  * (new_len <= current length; the pending token is unchanged, so this is meant for tests and benchmarks). */
 int knnssd_get_length(const knnssd_ctx *ctx);
 knnssd_status knnssd_set_length(knnssd_ctx *ctx, int new_len);
+
 /* Replace the pending token (HOST value); lets a caller teacher-force a token stream. */
 knnssd_status knnssd_set_pending(knnssd_ctx *ctx, int token);
 
 knnssd_status knnssd_get_stats(const knnssd_ctx *ctx, knnssd_stats *out);
 const char *knnssd_last_error(const knnssd_ctx *ctx);
+
+/*
+ * The objective of the mask search (Sec. 4.1, Eq. (3)): f(z) = the average inference time per verified token of
+ * self-speculative decoding with the skip mask z on a domain's anchor samples.  The optimiser that proposes masks
+ * (Bayesian optimisation in the paper) is the caller's; this call evaluates a batch of candidate masks.  For each
+ * sample the prompt pass runs once (it does not depend on the mask); then every mask decodes max_new tokens (greedy,
+ * k drafts per round) from the state the prompt pass left, and its draft + verification device time is added up.
+ *   masks_host          HOST [n_masks][2 * n_layers], entries 0 / 1
+ *   tokens_host         HOST int32: the samples' prompts one after the other; lens_host HOST int32 [n_samples]
+ *   ms_per_token_host   HOST [n_masks]: sum over samples of (draft + verify ms, CUDA events) / tokens generated by
+ *                       draft-and-verify rounds (max_new - 1 per sample: the first token comes from the prompt pass)
+ *   accepted_host, drafted_host   HOST [n_masks] totals, or NULL
+ * Leaves the session prefilled with the last sample and the last mask active.  Errors as knnssd_prefill / knnssd_decode.
+ */
+knnssd_status knnssd_mask_objective(knnssd_ctx *ctx, const unsigned char *masks_host, int n_masks,
+                                    const int *tokens_host, const int *lens_host, int n_samples, int max_new, int k,
+                                    float *ms_per_token_host, int *accepted_host, int *drafted_host);
 
 /*
  * Device-time measurement of the two passes at the current length, for benchmarks: runs `iters` draft passes of one

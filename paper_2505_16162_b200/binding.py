@@ -22,7 +22,7 @@ STATUS = {0: "OK", 1: "ERR_INVALID_ARG", 2: "ERR_SHAPE", 3: "ERR_CAPACITY", 4: "
 
 EXPORTS = ["knnssd_init", "knnssd_destroy", "knnssd_prefill", "knnssd_select_skipset", "knnssd_set_skipmask",
            "knnssd_draft", "knnssd_verify", "knnssd_generate", "knnssd_decode", "knnssd_get_launch_count", "knnssd_get_length", "knnssd_set_length",
-           "knnssd_set_pending", "knnssd_get_stats", "knnssd_last_error", "knnssd_time_pass", "knnssd_trace_pass", "knnssd_linear",
+           "knnssd_set_pending", "knnssd_mask_objective", "knnssd_get_stats", "knnssd_last_error", "knnssd_time_pass", "knnssd_trace_pass", "knnssd_linear",
            "knnssd_gemm_split", "knnssd_build_anchors", "knnssd_cosine_top1", "knnssd_cosine_top1_static"]
 
 
@@ -71,6 +71,7 @@ def _load():
         "knnssd_get_length": (I, [P]),
         "knnssd_set_length": (I, [P, I]),
         "knnssd_set_pending": (I, [P, I]),
+        "knnssd_mask_objective": (I, [P, P, I, P, P, I, I, I, P, P, P]),
         "knnssd_get_stats": (I, [P, C.POINTER(Stats)]),
         "knnssd_last_error": (C.c_char_p, [P]),
         "knnssd_time_pass": (I, [P, I, I, I, PF, PI, PF, PI]),
@@ -315,6 +316,19 @@ class Session:
 
     def set_pending(self, token: int):
         self._check(_lib.knnssd_set_pending(self.h, int(token)))
+
+    def mask_objective(self, masks, prompts, max_new: int, k: int):
+        """Eq. (3)'s objective for each candidate mask over the given sample prompts: (ms per verified token [n_masks],
+        accepted [n_masks], drafted [n_masks])."""
+        m = np.ascontiguousarray(np.asarray(masks, dtype=np.uint8))
+        lens = _host_i32([len(p) for p in prompts])
+        toks = _host_i32(np.concatenate([np.asarray(p, dtype=np.int32) for p in prompts]))
+        n = m.shape[0]
+        ms = np.zeros(n, dtype=np.float32)
+        acc, drf = np.zeros(n, dtype=np.int32), np.zeros(n, dtype=np.int32)
+        self._check(_lib.knnssd_mask_objective(self.h, m.ctypes.data, n, toks.ctypes.data, lens.ctypes.data, len(prompts), max_new, k,
+                                               ms.ctypes.data, acc.ctypes.data, drf.ctypes.data))
+        return ms, acc, drf
 
     def get_stats(self):
         st = Stats()

@@ -979,6 +979,53 @@ knnssd_status knnssd_set_pending(knnssd_ctx *c, int token) {
     return KNNSSD_OK;
 }
 
+knnssd_status knnssd_mask_objective(knnssd_ctx *c, const unsigned char *masks_host, int n_masks, const int *tokens_host,
+                                    const int *lens_host, int n_samples, int max_new, int k, float *ms_per_token_host,
+                                    int *accepted_host, int *drafted_host) {
+    if (!c) return KNNSSD_ERR_INVALID_ARG;
+    DeviceGuard dg(c->device);
+    if (!masks_host || !tokens_host || !lens_host || !ms_per_token_host || n_masks < 1 || n_samples < 1 || max_new < 1)
+        return fail(c, KNNSSD_ERR_INVALID_ARG, "mask_objective: bad arguments");
+    const int L2 = 2 * c->cfg.n_layers;
+    for (size_t j = 0; j < (size_t)n_masks * L2; ++j)
+        if (masks_host[j] > 1) return fail(c, KNNSSD_ERR_INVALID_ARG, "mask_objective: mask entries must be 0 or 1");
+    std::vector<double> ms(n_masks, 0.0);
+    std::vector<long long> tok(n_masks, 0), acc(n_masks, 0), drf(n_masks, 0);
+    std::vector<int> out(max_new);
+    size_t off = 0;
+    for (int sidx = 0; sidx < n_samples; ++sidx) {
+        const int P = lens_host[sidx];
+        int first = 0;
+        // the prompt pass does not depend on the mask: once per sample, then every mask decodes from the state it left
+        knnssd_status st = do_prefill(c, tokens_host + off, P, nullptr, &first);
+        if (st != KNNSSD_OK) return st;
+        off += (size_t)P;
+        for (int m = 0; m < n_masks; ++m) {
+            if (m > 0) {
+                st = knnssd_set_length(c, P);
+                if (st == KNNSSD_OK) st = knnssd_set_pending(c, first);
+                if (st != KNNSSD_OK) return st;
+            }
+            c->active_mask.assign(masks_host + (size_t)m * L2, masks_host + (size_t)(m + 1) * L2);
+            c->has_mask = true;
+            int n_out = 0;
+            knnssd_stats stt{};
+            st = do_decode(c, max_new, k, 0, out.data(), &n_out, nullptr, nullptr, &stt);
+            if (st != KNNSSD_OK) return st;
+            ms[m] += (double)stt.ms_draft + (double)stt.ms_verify;
+            tok[m] += n_out - 1;                              // the first token of the output came from the prompt pass
+            acc[m] += stt.accepted;
+            drf[m] += stt.drafted;
+        }
+    }
+    for (int m = 0; m < n_masks; ++m) {
+        ms_per_token_host[m] = tok[m] > 0 ? (float)(ms[m] / (double)tok[m]) : 0.f;
+        if (accepted_host) accepted_host[m] = (int)acc[m];
+        if (drafted_host) drafted_host[m] = (int)drf[m];
+    }
+    return KNNSSD_OK;
+}
+
 knnssd_status knnssd_get_stats(const knnssd_ctx *c, knnssd_stats *out) {
     if (!c || !out) return KNNSSD_ERR_INVALID_ARG;
     *out = c->stats;

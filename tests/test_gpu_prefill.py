@@ -200,3 +200,29 @@ def test_sixteen_row_pass_matches_oracle(kb):
         a, nxt = oracle.accept(rows, o["argmax"])
         assert (g["n_accepted"], g["next_token"]) == (a, nxt)
         first_o = nxt                                       # the pending token of the next round
+
+
+# ---- the mask-search objective (Sec. 4.1, Eq. (3)) -------------------------------------------------------
+
+def test_mask_objective_counts_match_oracle(kb):
+    """f(z) is a time, so the oracle cannot give its value; what it fixes is what was timed: for every candidate
+    mask and sample the accepted / drafted totals of the decode loop must be the oracle's, and the value must be the
+    per-token time of exactly those rounds."""
+    shape, om, sess = _pair(kb, "stream-bf16", 200)
+    L2 = 2 * shape.n_layers
+    masks = np.stack([np.zeros(L2, dtype=np.uint8), si.skip_mask(0, L2, 2), si.skip_mask(1, L2, 3)])
+    prompts = [si.uniform_tokens(20 + i, 0, n, shape.vocab).numpy() for i, n in enumerate((21, 60))]
+    max_new, k = 20, 4
+    ms, acc, drf = sess.mask_objective(masks, prompts, max_new, k)
+    want_acc, want_drf = np.zeros(3, dtype=np.int64), np.zeros(3, dtype=np.int64)
+    for p in prompts:
+        for m in range(3):
+            _, first, _ = om.prefill(p)
+            r = om.generate(first, max_new, k, masks[m])
+            want_acc[m] += r["accepted"]
+            want_drf[m] += r["drafted"]
+    assert np.array_equal(acc, want_acc) and np.array_equal(drf, want_drf)
+    assert acc[0] == drf[0]                                   # nothing skipped: the draft model is the full model
+    assert (ms > 0).all()
+    # the session is left usable, with the last mask active
+    assert len(sess.decode(5, 2)["tokens"]) == 5
