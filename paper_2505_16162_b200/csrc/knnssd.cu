@@ -487,8 +487,8 @@ bool prefill_tensor(knnssd_ctx *c, int n) {
                                             nullptr, 0, err, c->n_sms, s);
             ok = ok && prefill::launch_gemm(c->pf_map_d, cap, ly.wv, nullptr, nkv, d, T, prefill::PF_STORE, c->pf_qkv, ldq, nq + nkv,
                                             nullptr, nullptr, 0, err, c->n_sms, s);
-            prefill::rope_kv_rows_kernel<<<dim3(H + 2 * Hkv, T), HD / 2, 0, s>>>(c->pf_qkv, H, Hkv, HD, c->pf_cs, kc, vc, g.max_seq, t0);
-            prefill::attn_prompt_kernel<HD><<<dim3((T + 7) / 8, (H + 3) / 4), 128, 0, s>>>(c->pf_qkv, H, Hkv, kc, vc, g.max_seq, t0, T,
+            prefill::rope_kv_rows_kernel<<<T, 256, 0, s>>>(c->pf_qkv, H, Hkv, HD, c->pf_cs, kc, vc, g.max_seq, t0);
+            prefill::attn_prompt_kernel<HD><<<dim3((T + 15) / 16, (H + 3) / 4), 128, 0, s>>>(c->pf_qkv, H, Hkv, kc, vc, g.max_seq, t0, T,
                                                                                            c->pf_aq, c->pf_aq + (size_t)cap * nq);
             ok = ok && prefill::launch_gemm(c->pf_map_q, cap, ly.wo, nullptr, d, nq, T, prefill::PF_ADD, c->pf_x, d, 0, nullptr, nullptr, 0,
                                             err, c->n_sms, s);

@@ -11,7 +11,7 @@
 //                       SwiGLU of a gate tile and an up tile.
 //   norm_split_kernel   RMSNorm of each row, written as the two bf16 planes the next map reads.
 //   rope_kv_kernel      rotary embedding of q and k, K/V rows rounded to bf16 into the cache.
-//   attn_prompt_kernel  causal attention of 8 query rows per warp over the cached K/V, on mma.sync (the sizes are
+//   attn_prompt_kernel  causal attention of 16 query rows per warp over the cached K/V, on mma.sync (the sizes are
 //                       small next to the linear maps), output written as bf16 planes for the O projection.
 //
 // Every wait in these kernels is bounded; a wait that gives up sets the error word and the kernel returns after
@@ -350,29 +350,33 @@ __global__ void rope_table_kernel(const double *__restrict__ inv_freq, int pos0,
 }
 
 // Rotary embedding of the q and k heads of row t at position pos0 + t (q in place, fp32); K and V rows rounded to
-// bf16 into the cache.  grid = (H + 2 Hkv, T), hd / 2 threads: thread i owns the pair (i, i + hd / 2).
-__global__ void rope_kv_rows_kernel(float *__restrict__ qkv, int H, int Hkv, int hd, const float2 *__restrict__ table,
-                                    bf16_t *__restrict__ kc, bf16_t *__restrict__ vc, int max_seq, int pos0) {
-    const int slot = blockIdx.x, t = blockIdx.y, i = threadIdx.x, half = hd / 2;
-    float *row = qkv + (size_t)t * (H + 2 * Hkv) * hd + (size_t)slot * hd;
-    const int pos = pos0 + t;
-    if (slot < H + Hkv) {
-        const float2 cs2 = table[(size_t)t * half + i];
-        const float c = cs2.x, s = cs2.y;
+// bf16 into the cache.  grid = T, 256 threads: a thread walks pairs (i, i + hd / 2) of the row's H + 2 Hkv head slots.
+__global__ void __launch_bounds__(256) rope_kv_rows_kernel(float *__restrict__ qkv, int H, int Hkv, int hd,
+                                                           const float2 *__restrict__ table, bf16_t *__restrict__ kc,
+                                                           bf16_t *__restrict__ vc, int max_seq, int pos0) {
+    const int t = blockIdx.x, half = hd / 2, pos = pos0 + t;
+    float *trow = qkv + (size_t)t * (H + 2 * Hkv) * hd;
+    for (int idx = threadIdx.x; idx < (H + 2 * Hkv) * half; idx += 256) {
+        const int slot = idx / half, i = idx % half;
+        float *row = trow + (size_t)slot * hd;
         const float a = row[i], b = row[i + half];
-        const float ra = a * c - b * s, rb = b * c + a * s;
-        if (slot < H) {
-            row[i] = ra;
-            row[i + half] = rb;
+        if (slot < H + Hkv) {
+            const float2 cs2 = table[(size_t)t * half + i];
+            const float c = cs2.x, s = cs2.y;
+            const float ra = a * c - b * s, rb = b * c + a * s;
+            if (slot < H) {
+                row[i] = ra;
+                row[i + half] = rb;
+            } else {
+                bf16_t *dst = kc + ((size_t)(slot - H) * max_seq + pos) * hd;
+                dst[i] = float_to_bf16_rne(ra);
+                dst[i + half] = float_to_bf16_rne(rb);
+            }
         } else {
-            bf16_t *dst = kc + ((size_t)(slot - H) * max_seq + pos) * hd;
-            dst[i] = float_to_bf16_rne(ra);
-            dst[i + half] = float_to_bf16_rne(rb);
+            bf16_t *dst = vc + ((size_t)(slot - H - Hkv) * max_seq + pos) * hd;
+            dst[i] = float_to_bf16_rne(a);
+            dst[i + half] = float_to_bf16_rne(b);
         }
-    } else {
-        bf16_t *dst = vc + ((size_t)(slot - H - Hkv) * max_seq + pos) * hd;
-        dst[i] = float_to_bf16_rne(row[i]);
-        dst[i + half] = float_to_bf16_rne(row[i + half]);
     }
 }
 
@@ -396,64 +400,58 @@ __global__ void split_rows_kernel(const float *__restrict__ x, int n, bf16_t *__
 // Causal attention over the prompt
 // ---------------------------------------------------------------------------------------------
 
-// m16n8k16 with only rows 0..7 of the 16-row operand in use (registers of rows 8..15 are zero).
-__device__ __forceinline__ void mma_rows8(float (&c)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-                 : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
-}
-
-// One warp per (head, block of 8 consecutive prompt rows); it walks the positions 0 .. (its last row's position) in
-// segments of 64 with a running maximum and sum (the softmax of a row is taken over all its positions at once in
-// exact arithmetic; the running form differs from it by rounding only).  K and V, this chunk's rows included, are
-// already in the cache in bf16; q is rotated fp32 and is split into hi + lo here, as are the probabilities.
-// Lane (g8, t4) = (lane / 4, lane % 4): row g8 of the block.  Index conventions of the two products:
+// One warp per (head, block of 16 consecutive prompt rows); it walks the positions 0 .. (its last row's position) in
+// segments of 64 with a running maximum and sum per row (the softmax of a row is taken over all its positions at once
+// in exact arithmetic; the running form differs from it by rounding only).  K and V, this chunk's rows included, are
+// already in the cache in bf16; q is rotated fp32 and is split into hi + lo bf16 here (kept in shared memory, one
+// 16-row tile per warp), as are the probabilities.  m16n8k16 bf16 products, fp32 accumulation.
+// Lane (g8, t4) = (lane / 4, lane % 4) holds rows g8 and g8 + 8 of the block.  Index conventions of the two products:
 //   scores  column n = g8 of a tile is position 8 nt + g8; k-step s of the lane covers dimensions DL t4 + 4 s .. + 3
 //           for q and K alike (a dot product may take its terms in any order), so a lane reads one contiguous run of
 //           DL = HD / 4 dimensions of a K row;
 //   output  over pairs of tiles, k-indices (2 t4, 2 t4 + 1) = the lane's two positions of the first tile and
 //           (2 t4 + 8, 2 t4 + 9) those of the second; column n = g8 of V-tile j is dimension (HD / 8) g8 + j.
-// grid = (ceil(T / 8), ceil(H / 4)), 128 threads; the last row blocks (longest walks) are scheduled first.
+// grid = (ceil(T / 16), ceil(H / 4)), 128 threads; the last row blocks (longest walks) are scheduled first.
 template <int HD>
 __global__ void __launch_bounds__(128) attn_prompt_kernel(const float *__restrict__ qkv, int H, int Hkv, const bf16_t *__restrict__ kc,
                                                           const bf16_t *__restrict__ vc, int max_seq, int pos0, int T,
                                                           bf16_t *__restrict__ out_hi, bf16_t *__restrict__ out_lo) {
-    constexpr int DL = HD / 4, NW = HD / 8, VW = HD / 16, VJ = HD / 8, SEG = 64, NT = SEG / 8;
+    constexpr int DL = HD / 4, NW = HD / 8, VW = HD / 16, VJ = HD / 8, SEG = 64, NT = SEG / 8, RB = 16;
+    constexpr int QP = HD / 2 + 4;                           // words per q row in shared memory (padded)
+    __shared__ uint32_t qs[4][2][RB][QP];                    // [warp][term][row][word = dimensions (2w, 2w + 1)]
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g8 = lane >> 2, t4 = lane & 3;
     const int h = blockIdx.y * 4 + warp;
-    if (h >= H) return;
+    if (h >= H) return;                                      // whole warps only: nothing below is block-wide
     const int rb = gridDim.x - 1 - blockIdx.x;
-    const int t_row = rb * 8 + g8;
-    const bool live = t_row < T;
-    const int p_row = pos0 + t_row;
-    const int p_last = pos0 + min(rb * 8 + 7, T - 1);
+    const int t_first = rb * RB;
+    const int p_last = pos0 + min(t_first + RB - 1, T - 1);
     const int n_seg = p_last / SEG + 1;
     const int kvh = h / (H / Hkv);
     const int qstride = (H + 2 * Hkv) * HD;
     const bf16_t *kbase = kc + (size_t)kvh * max_seq * HD, *vbase = vc + (size_t)kvh * max_seq * HD;
     const float scale = 1.0f / sqrtf((float)HD);
+    int t_row[2], p_row[2];
+    bool live[2];
+#pragma unroll
+    for (int r = 0; r < 2; ++r) { t_row[r] = t_first + g8 + 8 * r; live[r] = t_row[r] < T; p_row[r] = pos0 + t_row[r]; }
 
-    uint32_t qh[NW], ql[NW];                                 // word w = dimensions (2w, 2w + 1) of the lane's run
-    {
-        const float *qr = qkv + (size_t)min(t_row, T - 1) * qstride + (size_t)h * HD + DL * t4;
-#pragma unroll
-        for (int e = 0; e < DL; e += 4) {
-            const float4 a = live ? *reinterpret_cast<const float4 *>(qr + e) : make_float4(0.f, 0.f, 0.f, 0.f);
-            const float v[4] = {a.x, a.y, a.z, a.w};
-#pragma unroll
-            for (int i = 0; i < 4; i += 2) {
-                const uint32_t h0 = float_to_bf16_rne(v[i]), h1 = float_to_bf16_rne(v[i + 1]);
-                const uint32_t l0 = float_to_bf16_rne(v[i] - __uint_as_float(h0 << 16));
-                const uint32_t l1 = float_to_bf16_rne(v[i + 1] - __uint_as_float(h1 << 16));
-                qh[(e + i) >> 1] = pack_bf16(h0, h1);
-                ql[(e + i) >> 1] = pack_bf16(l0, l1);
-            }
-        }
+    // ---- the block's q rows, split into hi + lo, into this warp's tile ----
+    for (int idx = lane; idx < RB * (HD / 2); idx += 32) {
+        const int r = idx / (HD / 2), w = idx % (HD / 2);
+        float2 v = make_float2(0.f, 0.f);
+        if (t_first + r < T) v = *reinterpret_cast<const float2 *>(qkv + (size_t)(t_first + r) * qstride + (size_t)h * HD + 2 * w);
+        const uint32_t h0 = float_to_bf16_rne(v.x), h1 = float_to_bf16_rne(v.y);
+        qs[warp][0][r][w] = pack_bf16(h0, h1);
+        qs[warp][1][r][w] = pack_bf16(float_to_bf16_rne(v.x - __uint_as_float(h0 << 16)), float_to_bf16_rne(v.y - __uint_as_float(h1 << 16)));
     }
+    __syncwarp();
+    const uint32_t *qh0 = &qs[warp][0][g8][(DL / 2) * t4], *qh1 = &qs[warp][0][g8 + 8][(DL / 2) * t4];
+    const uint32_t *ql0 = &qs[warp][1][g8][(DL / 2) * t4], *ql1 = &qs[warp][1][g8 + 8][(DL / 2) * t4];
+
     float o[VJ][4];
 #pragma unroll
     for (int j = 0; j < VJ; ++j) { o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f; }
-    float m_run = -INFINITY, l_run = 0.f;                    // l_run: this lane's share of the row's sum
+    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};   // l_run: this lane's share of the row's sum
 
     for (int seg = 0; seg < n_seg; ++seg) {
         const int p_begin = seg * SEG, p_end = min(p_begin + SEG, p_last + 1);
@@ -464,7 +462,7 @@ __global__ void __launch_bounds__(128) attn_prompt_kernel(const float *__restric
             for (int q = 0; q < NW / 4; ++q)
                 dst[q] = p < p_end ? *reinterpret_cast<const uint4 *>(src + 8 * q) : make_uint4(0u, 0u, 0u, 0u);
         };
-        float sc[NT][2];                                     // scores of (row g8, positions 8 nt + 2 t4 + {0, 1})
+        float sc[NT][4];               // scores of rows (g8: [0], [1]; g8 + 8: [2], [3]) x positions 8 nt + 2 t4 + {0, 1}
         {
             uint4 kb[2][NW / 4];
             load_k(0, kb[0]);
@@ -472,16 +470,16 @@ __global__ void __launch_bounds__(128) attn_prompt_kernel(const float *__restric
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
                 uint4(&kq)[NW / 4] = kb[nt & 1];
-                float ch[4] = {0.f, 0.f, 0.f, 0.f}, cl[4] = {0.f, 0.f, 0.f, 0.f};
+                float c[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
                 for (int q = 0; q < NW / 4; ++q) {
-                    mma_rows8(cl, ql[4 * q], ql[4 * q + 1], kq[q].x, kq[q].y);
-                    mma_rows8(ch, qh[4 * q], qh[4 * q + 1], kq[q].x, kq[q].y);
-                    mma_rows8(cl, ql[4 * q + 2], ql[4 * q + 3], kq[q].z, kq[q].w);
-                    mma_rows8(ch, qh[4 * q + 2], qh[4 * q + 3], kq[q].z, kq[q].w);
+                    // words 4q .. 4q+3 of the lane's run: k-steps 2q (x, y) and 2q + 1 (z, w); the lo term first
+                    stream::mma_bf16(c, ql0[4 * q], ql1[4 * q], ql0[4 * q + 1], ql1[4 * q + 1], kq[q].x, kq[q].y);
+                    stream::mma_bf16(c, qh0[4 * q], qh1[4 * q], qh0[4 * q + 1], qh1[4 * q + 1], kq[q].x, kq[q].y);
+                    stream::mma_bf16(c, ql0[4 * q + 2], ql1[4 * q + 2], ql0[4 * q + 3], ql1[4 * q + 3], kq[q].z, kq[q].w);
+                    stream::mma_bf16(c, qh0[4 * q + 2], qh1[4 * q + 2], qh0[4 * q + 3], qh1[4 * q + 3], kq[q].z, kq[q].w);
                 }
-                sc[nt][0] = cl[0] + ch[0];
-                sc[nt][1] = cl[1] + ch[1];
+                sc[nt][0] = c[0]; sc[nt][1] = c[1]; sc[nt][2] = c[2]; sc[nt][3] = c[3];
                 if (nt + 2 < NT) load_k(nt + 2, kq);
             }
         }
@@ -504,45 +502,50 @@ __global__ void __launch_bounds__(128) attn_prompt_kernel(const float *__restric
         load_v(0, vb[0]);
         load_v(1, vb[1]);
 
-        // ---- running softmax: new maximum, old sums and outputs rescaled ----
-        float mx = -INFINITY;
+        // ---- running softmax per row: new maximum, old sums and outputs rescaled ----
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt)
+        for (int r = 0; r < 2; ++r) {
+            float mx = -INFINITY;
 #pragma unroll
-            for (int e = 0; e < 2; ++e) {
-                const int p = p_begin + 8 * nt + 2 * t4 + e;
-                sc[nt][e] = (live && p <= p_row) ? sc[nt][e] * scale : -INFINITY;
-                mx = fmaxf(mx, sc[nt][e]);
-            }
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-        const float m_new = fmaxf(m_run, mx);
-        const float f = m_run == -INFINITY ? 0.f : expf(m_run - m_new);
-        m_run = m_new;
-        l_run *= f;
+            for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt)
+                for (int e = 0; e < 2; ++e) {
+                    const int p = p_begin + 8 * nt + 2 * t4 + e;
+                    float &v = sc[nt][2 * r + e];
+                    v = (live[r] && p <= p_row[r]) ? v * scale : -INFINITY;
+                    mx = fmaxf(mx, v);
+                }
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+            const float m_new = fmaxf(m_run[r], mx);
+            const float f = m_run[r] == -INFINITY ? 0.f : expf(m_run[r] - m_new);
+            m_run[r] = m_new;
+            l_run[r] *= f;
 #pragma unroll
-            for (int e = 0; e < 2; ++e) {
-                const float pj = sc[nt][e] == -INFINITY ? 0.f : expf(sc[nt][e] - m_new);
-                sc[nt][e] = pj;
-                l_run += pj;
-            }
+            for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-        for (int j = 0; j < VJ; ++j) { o[j][0] *= f; o[j][1] *= f; }
+                for (int e = 0; e < 2; ++e) {
+                    float &v = sc[nt][2 * r + e];
+                    v = v == -INFINITY ? 0.f : expf(v - m_new);
+                    l_run[r] += v;
+                }
+#pragma unroll
+            for (int j = 0; j < VJ; ++j) { o[j][2 * r] *= f; o[j][2 * r + 1] *= f; }
+        }
 
         // ---- o += p V ----
 #pragma unroll
         for (int np = 0; np < NT; np += 2) {
-            uint32_t ah[2], al[2];
+            uint32_t ah[4], al[4];     // [0], [1]: rows g8, g8 + 8 of tile np; [2], [3]: of tile np + 1
 #pragma unroll
-            for (int i = 0; i < 2; ++i) {
-                const uint32_t h0 = float_to_bf16_rne(sc[np + i][0]), h1 = float_to_bf16_rne(sc[np + i][1]);
-                const uint32_t l0 = float_to_bf16_rne(sc[np + i][0] - __uint_as_float(h0 << 16));
-                const uint32_t l1 = float_to_bf16_rne(sc[np + i][1] - __uint_as_float(h1 << 16));
-                ah[i] = pack_bf16(h0, h1);
-                al[i] = pack_bf16(l0, l1);
-            }
+            for (int i = 0; i < 2; ++i)
+#pragma unroll
+                for (int r = 0; r < 2; ++r) {
+                    const float v0 = sc[np + i][2 * r], v1 = sc[np + i][2 * r + 1];
+                    const uint32_t h0 = float_to_bf16_rne(v0), h1 = float_to_bf16_rne(v1);
+                    ah[2 * i + r] = pack_bf16(h0, h1);
+                    al[2 * i + r] = pack_bf16(float_to_bf16_rne(v0 - __uint_as_float(h0 << 16)), float_to_bf16_rne(v1 - __uint_as_float(h1 << 16)));
+                }
 #pragma unroll
             for (int j = 0; j < VJ; ++j) {
                 const int wi = (j >> 1) & 3;
@@ -554,24 +557,27 @@ __global__ void __launch_bounds__(128) attn_prompt_kernel(const float *__restric
                     const uint32_t xb = wi == 0 ? wb.x : wi == 1 ? wb.y : wi == 2 ? wb.z : wb.w;
                     b[i] = __byte_perm(xa, xb, (j & 1) ? 0x7632 : 0x5410);     // dimension j of the two positions' rows
                 }
-                mma_rows8(o[j], al[0], al[1], b[0], b[1]);
-                mma_rows8(o[j], ah[0], ah[1], b[0], b[1]);
+                stream::mma_bf16(o[j], al[0], al[1], al[2], al[3], b[0], b[1]);
+                stream::mma_bf16(o[j], ah[0], ah[1], ah[2], ah[3], b[0], b[1]);
             }
             if (np + 2 < NT) { load_v(np + 2, vb[0]); load_v(np + 3, vb[1]); }
         }
     }
 
-    // ---- row g8: dimensions DL t4 + j (o[j][0]) and DL t4 + VJ + j (o[j][1]), divided by the row's sum ----
-    l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
-    l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
-    if (live) {
-        const size_t base = (size_t)t_row * ((size_t)H * HD) + (size_t)h * HD + DL * t4;
+    // ---- rows g8 ([0], [1]) and g8 + 8 ([2], [3]): dimensions DL t4 + j and DL t4 + VJ + j, divided by the row's sum ----
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        float l = l_run[r];
+        l += __shfl_xor_sync(0xffffffffu, l, 1);
+        l += __shfl_xor_sync(0xffffffffu, l, 2);
+        if (!live[r]) continue;
+        const size_t base = (size_t)t_row[r] * ((size_t)H * HD) + (size_t)h * HD + DL * t4;
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
             uint32_t hw[VJ / 2], lw[VJ / 2];
 #pragma unroll
             for (int j = 0; j < VJ; j += 2) {
-                const float v0 = o[j][half] / l_run, v1 = o[j + 1][half] / l_run;
+                const float v0 = o[j][2 * r + half] / l, v1 = o[j + 1][2 * r + half] / l;
                 const uint32_t h0 = float_to_bf16_rne(v0), h1 = float_to_bf16_rne(v1);
                 hw[j >> 1] = pack_bf16(h0, h1);
                 lw[j >> 1] = pack_bf16(float_to_bf16_rne(v0 - __uint_as_float(h0 << 16)), float_to_bf16_rne(v1 - __uint_as_float(h1 << 16)));
