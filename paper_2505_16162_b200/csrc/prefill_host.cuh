@@ -40,14 +40,18 @@ inline bool make_map(CUtensorMap *m, const void *base, size_t rows, size_t cols,
               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// The contraction kernels need more dynamic shared memory than the default limit; the attribute belongs to the
+// current device, so it is set once per device (one process may drive several GPUs).
 inline bool gemm_attrs_once() {
-    static bool done = false, ok = false;
-    if (!done) {
-        done = true;
-        ok = cudaFuncSetAttribute(gemm_split_kernel<PF_STORE>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM) == cudaSuccess &&
-             cudaFuncSetAttribute(gemm_split_kernel<PF_ADD>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM) == cudaSuccess &&
-             cudaFuncSetAttribute(gemm_split_kernel<PF_SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM) == cudaSuccess;
-    }
+    static bool done[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+    if (done[dev]) return true;
+    const bool ok =
+        cudaFuncSetAttribute(gemm_split_kernel<PF_STORE>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM) == cudaSuccess &&
+        cudaFuncSetAttribute(gemm_split_kernel<PF_ADD>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM) == cudaSuccess &&
+        cudaFuncSetAttribute(gemm_split_kernel<PF_SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM) == cudaSuccess;
+    done[dev] = ok;
     return ok;
 }
 

@@ -157,15 +157,16 @@ def test_generate_after_a_long_prompt_matches_oracle_exactly(kb, shape_name):
     assert np.array_equal(got["accepts"], want["accepts"])
 
 
-def test_prompt_longer_than_one_chunk(kb):
-    """More than 1024 prompt rows: the second chunk's attention reads the first chunk's K/V from the cache."""
+@pytest.mark.parametrize("n_prompt", [1025, 1100])
+def test_prompt_longer_than_one_chunk(kb, n_prompt):
+    """More than 1024 prompt rows: the second chunk (a single row, or 76) reads the first chunk's K/V from the cache."""
     shape, om, sess = _pair(kb, "stream64-bf16", 1200)
-    prompt = si.uniform_tokens(3, 0, 1100, shape.vocab).numpy()
+    prompt = si.uniform_tokens(3, 0, n_prompt, shape.vocab).numpy()
     pooled_o, first_o, _ = om.prefill(prompt)
     first_g, pooled_g = sess.prefill(prompt, want_pooled=True)
     assert first_g == first_o
     assert np.abs(pooled_g.cpu().numpy() - pooled_o).max() < TOL
-    o = om.forward(np.array([first_o], dtype=np.int32), 1100)
+    o = om.forward(np.array([first_o], dtype=np.int32), n_prompt)
     sess.set_skipmask(np.zeros(2 * shape.n_layers, dtype=np.uint8))
     g = sess.verify(np.zeros(0, dtype=np.int32), want_logits=True)
     assert np.abs(g["logits"].cpu().numpy() - o["logits"]).max() < TOL
