@@ -30,7 +30,7 @@ using stream::mbar_try_wait;
 using stream::smem_u32;
 
 constexpr int BM = 128;                               // tokens per tile: rows of the accumulator = lanes of tensor memory
-constexpr int BN_MAX = 320;                           // most accumulator columns per tile (a launch picks 128, 192, 256 or 320)
+constexpr int BN_MAX = 320;                           // most accumulator columns per tile (a launch picks 64, 128, .. 320)
 constexpr int BOX_N = 64;                             // weight rows per TMA box
 constexpr int BK = 64;                                // input columns per stage: 128 bytes of bf16 = one swizzle row
 constexpr int STAGES = 3;

@@ -62,7 +62,7 @@ inline int pick_bn(int T, int N, bool swiglu, int n_sms) {
     const int row_tiles = (T + BM - 1) / BM;
     int best = 0;
     long best_cost = 0;
-    for (int bn = 128; bn <= BN_MAX; bn += 64) {
+    for (int bn = BOX_N; bn <= BN_MAX; bn += BOX_N) {
         if (swiglu && bn % 128) continue;
         const int per = swiglu ? bn / 2 : bn;
         const long ctas = (long)row_tiles * ((N + per - 1) / per);
