@@ -322,7 +322,8 @@ void run_pass_mega(knnssd_ctx *c, int M, const int *tok_dev, int pos_off, const 
     pr.out_row0 = out_row0;
     pr.bar_base = c->bar_total;
     if (head_row0 < M) bars += 1;
-    if (M >= pass::MERGE_ROWS) bars += n_attn;
+    pr.merge_op = pass::merge_rows_separately(M, c->cfg.n_heads / c->cfg.n_kv_heads) ? 1 : 0;
+    if (pr.merge_op) bars += n_attn;
     if (M > pass::BLKM) bars += n_attn;
     cudaError_t e;
     if (M > pass::BLKM) e = c->cfg.head_dim == 128 ? launch_pass_t<128, 2>(c, pr) : launch_pass_t<64, 2>(c, pr);

@@ -29,7 +29,7 @@ constexpr int SEGP = 64;           // attention: positions per segment (fixed ab
 constexpr unsigned BAR_SPIN_LIMIT = 4000000u;
 
 enum { OP_EMBED = 0, OP_LINEAR = 1, OP_ATTN = 2, OP_HIDDEN = 3, OP_ARGMAX = 4, OP_ATTN_MERGE = 5, OP_KV_APPEND = 6 };
-constexpr int MERGE_ROWS = 3;      // passes with at least this many rows merge attention partials in a separate operation
+constexpr int MERGE_ROWS = 3;      // tasks with at least this many (row, head) pairs leave the merge to a separate operation
 
 struct Op {
     int type;
@@ -72,7 +72,14 @@ struct Params {
     int want_hidden;
     int out_row0;              // row of the logits / hidden-state buffers that this pass's row 0 goes to
     unsigned long long bar_base;   // value of *bar when this launch starts
+    int merge_op;              // the attention partials are merged by the separate merge operation (merge_rows_separately)
 };
+
+// Whether a pass of M rows merges its attention partials in the separate operation: when an attention task carries
+// at least MERGE_ROWS (row, head) pairs - all G query heads of a K/V head for passes of up to BLKM rows.
+__host__ __device__ inline bool merge_rows_separately(int M, int G);
+
+__host__ __device__ inline bool merge_rows_separately(int M, int G) { return M > BLKM || M * G >= MERGE_ROWS; }
 
 __device__ __forceinline__ unsigned long long globaltimer_ns() {
     unsigned long long t;
@@ -327,8 +334,15 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
     const int M = pr.M, H = md.H, Hkv = md.Hkv, G = H / Hkv;
     const int P0 = md.state->len + pr.pos_off, Ttot = P0 + M;
     const int Pc = all_cached ? Ttot : P0;                   // positions below Pc are read from the cache
-    const int rm = row0 + g8;                                // the pass row this lane's MMA row stands for
-    const int n_seg = (Ttot + SEGP - 1) / SEGP, n_tasks = H * n_seg;
+    // A task = (segment, head group, block of 8 rows).  Passes of up to BLKM rows (all_cached false) take the G query
+    // heads that share a K/V head together: the rows of a group are the (head-in-group, pass row) pairs rr = hg M + m,
+    // eight per block, so that a K/V segment is read once per block instead of once per head and a GQA model has
+    // G times fewer tasks.  With all_cached a task is one head and the block is given by row0.
+    const int Gt = all_cached ? 1 : G;                       // query heads per group
+    const int n_grp = H / Gt;
+    const int R = all_cached ? M : M * Gt;                   // rows of a group
+    const int nblk = all_cached ? 1 : (R + BLKM - 1) / BLKM;
+    const int n_seg = (Ttot + SEGP - 1) / SEGP, n_tasks = n_grp * n_seg * nblk;
     const int qstride = (H + 2 * Hkv) * HD;
     const float scale = 1.0f / sqrtf((float)HD);
     const bool upper = t4 >= 2;                              // this lane's run lies in the second half of the head
@@ -338,23 +352,28 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
     const float2 *my_cs = md.rope_cs + (size_t)cta * MAXM * HALF;                           // this CTA's copy
 
     for (int t = warp * n_cta + cta; t < n_tasks; t += NCW * n_cta) {
-        const int seg = t / H, h = t % H, kvh = h / G;
+        const int blk = t % nblk, tt = t / nblk, seg = tt / n_grp, grp = tt % n_grp;
+        const int kvh = all_cached ? grp / G : grp;
+        const int rr = blk * BLKM + g8;                      // this lane's row of the group (grouped tasks)
+        const int rm = all_cached ? row0 + g8 : rr % M;      // the pass row this lane's MMA row stands for
+        const int h = all_cached ? grp : kvh * G + min(rr / M, G - 1);   // and its query head
+        const bool row_in = all_cached ? rm < M : rr < R;
         const int p_begin = seg * SEGP, p_end = min(p_begin + SEGP, Ttot);
         const int m_first = max(0, p_begin - P0);           // first row that sees this segment
-        const bool writer = (h % G) == 0;
+        const bool writer = !all_cached && blk == 0;         // one task per (segment, K/V head) puts the new rows into the cache
         bf16_t *kbase = op.kc + (size_t)kvh * md.max_seq * HD;
         bf16_t *vbase = op.vc + (size_t)kvh * md.max_seq * HD;
-        if (row0 + BLKM <= m_first) continue;               // none of this block's rows sees the segment
-        // row rm's own position lies in this segment and is not in the cache yet
-        const bool row_new = !all_cached && rm < M && P0 + rm >= p_begin && P0 + rm < p_end;
-        const bool row_live = rm < M && rm >= m_first;
+        if (all_cached && row0 + BLKM <= m_first) continue;  // none of this block's rows sees the segment
+        // pass row g8's own position lies in this segment and is not in the cache yet: this lane rotates / rounds its K, V
+        const bool row_new = !all_cached && g8 < M && P0 + g8 >= p_begin && P0 + g8 < p_end;
+        const bool row_live = row_in && rm >= m_first;
 
         KNNSSD_ATT_STAMP(0);
         // ---- this lane's run of q (row g8), of the new K row and of the new V row: load, rotate, round / split ----
         float qf[DL], kf[DL];
         {
             const float *qraw = md.qkv + (size_t)min(rm, M - 1) * qstride + (size_t)h * HD + DL * t4;
-            const float *kraw = md.qkv + (size_t)min(rm, M - 1) * qstride + (size_t)(H + kvh) * HD + DL * t4;
+            const float *kraw = md.qkv + (size_t)min(g8, M - 1) * qstride + (size_t)(H + kvh) * HD + DL * t4;
 #pragma unroll
             for (int e = 0; e < DL; e += 4) {
                 const float4 a = row_live ? __ldcg(reinterpret_cast<const float4 *>(qraw + e)) : make_float4(0.f, 0.f, 0.f, 0.f);
@@ -365,14 +384,15 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
 #pragma unroll
             for (int e = 0; e < DL; ++e) {
                 const float qp = __shfl_xor_sync(0xffffffffu, qf[e], 2), kp = __shfl_xor_sync(0xffffffffu, kf[e], 2);
-                const float2 cs = (row_live || row_new) ? my_cs[rm * HALF + ci + e] : make_float2(1.f, 0.f);
-                qf[e] = upper ? (qf[e] * cs.x + qp * cs.y) : (qf[e] * cs.x - qp * cs.y);
-                kf[e] = upper ? (kf[e] * cs.x + kp * cs.y) : (kf[e] * cs.x - kp * cs.y);
+                const float2 cq = row_live ? my_cs[rm * HALF + ci + e] : make_float2(1.f, 0.f);
+                const float2 ck = row_new ? my_cs[g8 * HALF + ci + e] : make_float2(1.f, 0.f);
+                qf[e] = upper ? (qf[e] * cq.x + qp * cq.y) : (qf[e] * cq.x - qp * cq.y);
+                kf[e] = upper ? (kf[e] * ck.x + kp * ck.y) : (kf[e] * ck.x - kp * ck.y);
             }
         }
         __syncwarp();
         if (row_new) {
-            const float *vraw = md.qkv + (size_t)rm * qstride + (size_t)(H + Hkv + kvh) * HD + DL * t4;
+            const float *vraw = md.qkv + (size_t)g8 * qstride + (size_t)(H + Hkv + kvh) * HD + DL * t4;
 #pragma unroll
             for (int e = 0; e < DL; e += 8) {
                 const float4 a = __ldcg(reinterpret_cast<const float4 *>(vraw + e)), b = __ldcg(reinterpret_cast<const float4 *>(vraw + e + 4));
@@ -539,13 +559,15 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
             last = atomicAdd(md.attn_cnt + rm * H + h, 1) == n_seg_m - 1;
         }
         KNNSSD_ATT_STAMP(7);
-        const unsigned last_mask = __ballot_sync(0xffffffffu, last);     // bit 4*m set: this warp finishes (row m, head h)
+        const unsigned last_mask = __ballot_sync(0xffffffffu, last);     // bit 4*g set: this warp finishes the (row, head) of lane row g
         if (last_mask) {
             __threadfence();
-            for (int m = m_first; m < M; ++m) {
-                if (!((last_mask >> (4 * m)) & 1u)) continue;
-                attn_merge_row<HD>(md, op, P0, m, h, lane);
-                if (lane == 0) md.attn_cnt[m * H + h] = 0;
+            for (int g = 0; g < BLKM; ++g) {
+                if (!((last_mask >> (4 * g)) & 1u)) continue;
+                const int rg = blk * BLKM + g;
+                const int mg = all_cached ? row0 + g : rg % M, hg = all_cached ? grp : kvh * G + rg / M;
+                attn_merge_row<HD>(md, op, P0, mg, hg, lane);
+                if (lane == 0) md.attn_cnt[mg * H + hg] = 0;
             }
         }
         KNNSSD_ATT_STAMP(8);
@@ -642,12 +664,12 @@ __global__ void __launch_bounds__(stream::NTHREADS, 1) pass_kernel(const Model m
             else if (op.type == OP_KV_APPEND) { if (NB > 1) kv_append_phase<HD>(md, op, pr, cta, n_cta, warp, lane); else ran = false; }
             else if (op.type == OP_ATTN) {
                 if (NB == 1) {
-                    attn_phase<HD>(md, op, pr, r, cta, n_cta, warp, lane, pr.M >= MERGE_ROWS, 0, false);
+                    attn_phase<HD>(md, op, pr, r, cta, n_cta, warp, lane, pr.merge_op != 0, 0, false);
                 } else {
                     for (int blk = 0; blk < NB; ++blk) attn_phase<HD>(md, op, pr, r, cta, n_cta, warp, lane, true, blk * BLKM, true);
                 }
             }
-            else if (op.type == OP_ATTN_MERGE) { if (pr.M >= MERGE_ROWS) attn_merge_phase<HD>(md, op, pr, cta, n_cta, warp, lane); else ran = false; }
+            else if (op.type == OP_ATTN_MERGE) { if (pr.merge_op) attn_merge_phase<HD>(md, op, pr, cta, n_cta, warp, lane); else ran = false; }
             else if (op.type == OP_HIDDEN) { if (pr.want_hidden) hidden_phase(md, pr, r, cta, tid); else ran = false; }
             else if (op.type == OP_ARGMAX) { if (pr.head_row0 < pr.M) argmax_phase(md, pr, r, cta, n_cta, tid); else ran = false; }
         }
