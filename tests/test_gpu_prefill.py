@@ -227,3 +227,26 @@ def test_mask_objective_counts_match_oracle(kb):
     assert (ms > 0).all()
     # the session is left usable, with the last mask active
     assert len(sess.decode(5, 2)["tokens"]) == 5
+
+
+@pytest.mark.parametrize("shape_name", ["stream-bf16", "stream64-bf16"])
+def test_every_row_count_of_the_common_kernel_with_grouped_heads(kb, shape_name):
+    """Verification passes of 1..8 rows on GQA shapes (3 and 4 query heads per K/V head): an attention task then
+    carries up to 8 of the (head, row) pairs of a K/V head and a group spans several tasks."""
+    shape, om, sess = _pair(kb, shape_name, 200)
+    prompt = si.uniform_tokens(1, 0, 70, shape.vocab).numpy()       # the last segment starts inside the prompt
+    _, first_o, _ = om.prefill(prompt)
+    assert sess.prefill(prompt) == first_o
+    sess.set_skipmask(np.zeros(2 * shape.n_layers, dtype=np.uint8))
+    pending = first_o
+    for n_rows in (7, 6, 5, 0, 3):
+        rows = si.uniform_tokens(30 + n_rows, 2, n_rows, shape.vocab).numpy() if n_rows else np.zeros(0, dtype=np.int32)
+        n = sess.length
+        om.length = n
+        o = om.forward(np.concatenate([[pending], rows]).astype(np.int32), n, want_hidden=True)
+        g = sess.verify(rows, want_logits=True, want_hidden=True)
+        assert np.abs(g["logits"].cpu().numpy() - o["logits"]).max() < TOL
+        assert np.abs(g["hidden"].cpu().numpy() - o["hidden"]).max() < TOL
+        a, nxt = oracle.accept(rows, o["argmax"])
+        assert (g["n_accepted"], g["next_token"]) == (a, nxt)
+        pending = nxt
