@@ -287,10 +287,17 @@ __device__ __forceinline__ void attn_merge_row(const Model &md, const Op &op, in
     for (int s0 = 0; s0 < n_seg_m; s0 += 16) {
         float pv[16][DPL];
 #pragma unroll
-        for (int i = 0; i < 16; ++i)
-#pragma unroll
-            for (int e = 0; e < DPL; ++e)
-                pv[i][e] = s0 + i < n_seg_m ? __ldcg(md.part_o + (base + s0 + i) * HD + d0 + e) : 0.f;
+        for (int i = 0; i < 16; ++i) {
+            // one vector load per segment (DPL = 4: 16 bytes, DPL = 2: 8 bytes)
+            const float *src = md.part_o + (base + s0 + i) * HD + d0;
+            if (DPL == 4) {
+                const float4 v = s0 + i < n_seg_m ? __ldcg(reinterpret_cast<const float4 *>(src)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                pv[i][0] = v.x; pv[i][1] = v.y; pv[i][DPL - 2] = v.z; pv[i][DPL - 1] = v.w;
+            } else {
+                const float2 v = s0 + i < n_seg_m ? __ldcg(reinterpret_cast<const float2 *>(src)) : make_float2(0.f, 0.f);
+                pv[i][0] = v.x; pv[i][DPL - 1] = v.y;
+            }
+        }
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
             const int sg = s0 + i;
