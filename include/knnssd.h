@@ -241,6 +241,19 @@ knnssd_status knnssd_gemm_split(const void *W0_dev, const void *W1_dev, int n_ou
                                 int mode, float *y_dev, void *cuda_stream);
 
 /*
+ * The same linear map as knnssd_linear for M <= 16 rows, on the 5th-generation tensor cores: the weights are the
+ * 128-row operand, the rows of x (two bf16 terms, hi + lo) the 16 columns, fp32 accumulation in tensor memory; the
+ * input columns are split into chunks across CTAs and the chunks' partial sums added in chunk order.  Stand-alone:
+ * the decode passes (Sec. 4.2) do not use it yet; it exists to measure what their linear phases would cost at 9..16
+ * rows.
+ *   W DEVICE bf16 [n_out][n_in], 16-byte aligned; x DEVICE fp32 [M][n_in]; y DEVICE fp32 [M][n_out]; n_in % 64 == 0;
+ *   M > 16: KNNSSD_ERR_CAPACITY.  ms_kernels_host: HOST, device time of the contraction + the chunk sum (CUDA
+ *   events), or NULL.  Allocates and frees its scratch; synchronises the stream.
+ */
+knnssd_status knnssd_linear_tc(const void *W_dev, int n_out, int n_in, const float *x_dev, int M, float *y_dev,
+                               float *ms_kernels_host, void *cuda_stream);
+
+/*
  * Anchor construction of the pre-inference stage (Sec. 4.1): K-means (Lloyd's iteration) over the sampled last
  * hidden vectors with as many clusters as domains, then, per cluster, the k members nearest to its centroid (Eq. (2)).
  * The paper does not say how K-means is started or stopped: the starting centroids are an argument, and the iteration

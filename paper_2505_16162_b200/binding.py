@@ -23,7 +23,7 @@ STATUS = {0: "OK", 1: "ERR_INVALID_ARG", 2: "ERR_SHAPE", 3: "ERR_CAPACITY", 4: "
 EXPORTS = ["knnssd_init", "knnssd_destroy", "knnssd_prefill", "knnssd_select_skipset", "knnssd_set_skipmask",
            "knnssd_draft", "knnssd_verify", "knnssd_generate", "knnssd_decode", "knnssd_get_launch_count", "knnssd_get_length", "knnssd_set_length",
            "knnssd_set_pending", "knnssd_mask_objective", "knnssd_get_stats", "knnssd_last_error", "knnssd_time_pass", "knnssd_trace_pass", "knnssd_linear",
-           "knnssd_gemm_split", "knnssd_build_anchors", "knnssd_cosine_top1", "knnssd_cosine_top1_static"]
+           "knnssd_gemm_split", "knnssd_linear_tc", "knnssd_build_anchors", "knnssd_cosine_top1", "knnssd_cosine_top1_static"]
 
 
 class KnnssdError(RuntimeError):
@@ -79,6 +79,7 @@ def _load():
         "knnssd_linear": (I, [P, I, I, I, P, I, P, P]),
         "knnssd_gemm_split": (I, [P, P, I, I, P, I, I, P, P]),
         "knnssd_build_anchors": (I, [P, I, I, I, P, I, I, P, P, P, PI, PF, P]),
+        "knnssd_linear_tc": (I, [P, I, I, P, I, P, PF, P]),
         "knnssd_cosine_top1": (I, [P, P, I, I, PI, PF, P]),
         "knnssd_cosine_top1_static": (I, [P, P, I, I, PI, PF, P]),
     }
@@ -139,6 +140,20 @@ def knnssd_gemm_split(W0: torch.Tensor, x: torch.Tensor, mode: int = 0, W1: Opti
     if rc:
         raise KnnssdError(rc, "knnssd_gemm_split")
     return y
+
+
+def knnssd_linear_tc(W: torch.Tensor, x: torch.Tensor):
+    """y = x @ W^T for up to 16 rows through the tensor-core weight-streaming kernel; returns (y, ms of its kernels)."""
+    M, n_in = x.shape
+    n_out = W.shape[0]
+    y = torch.empty((M, n_out), dtype=torch.float32, device=x.device)
+    ms = C.c_float()
+    with torch.cuda.device(x.device):
+        rc = _lib.knnssd_linear_tc(_dev_ptr(W, torch.bfloat16), n_out, n_in, _dev_ptr(x, torch.float32), M, _dev_ptr(y), C.byref(ms),
+                                   torch.cuda.current_stream().cuda_stream)
+    if rc:
+        raise KnnssdError(rc, "knnssd_linear_tc")
+    return y, ms.value
 
 
 def knnssd_build_anchors(x: torch.Tensor, init_centroids: torch.Tensor, max_rounds: int, k: int):

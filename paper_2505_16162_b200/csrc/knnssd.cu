@@ -7,6 +7,7 @@
 #include "pass_kernel.cuh"
 #include "prefill_host.cuh"
 #include "anchors.cuh"
+#include "linear_tc.cuh"
 
 #include <cmath>
 #include <cstdio>
@@ -1188,6 +1189,65 @@ knnssd_status knnssd_gemm_split(const void *W0_dev, const void *W1_dev, int n_ou
     }
     cudaFree(planes);
     if (outp) cudaFree(outp);
+    return st;
+}
+
+knnssd_status knnssd_linear_tc(const void *W_dev, int n_out, int n_in, const float *x_dev, int M, float *y_dev,
+                               float *ms_kernels_host, void *cuda_stream) {
+    if (!W_dev || !x_dev || !y_dev || n_out < 1 || n_in < 1 || M < 1) return KNNSSD_ERR_INVALID_ARG;
+    if (M > lintc::TN) return KNNSSD_ERR_CAPACITY;
+    if (n_in % lintc::BK != 0 || (reinterpret_cast<uintptr_t>(W_dev) & 15u)) return KNNSSD_ERR_SHAPE;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+    int dev = 0, n_sms = 148;
+    if (cudaGetDevice(&dev) != cudaSuccess) return KNNSSD_ERR_CUDA;
+    cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev);
+    const int tiles = (n_out + lintc::TM - 1) / lintc::TM, nkb = n_in / lintc::BK;
+    // chunks of the input columns: enough work items for every SM when the matrix has few 128-unit tiles, at least
+    // 8 k-blocks per item
+    int kc = tiles >= n_sms ? 1 : (n_sms + tiles - 1) / tiles;
+    if (kc > nkb / 8) kc = nkb / 8 > 0 ? nkb / 8 : 1;
+    const int kb_per = (nkb + kc - 1) / kc;
+    kc = (nkb + kb_per - 1) / kb_per;
+    bf16_t *planes = nullptr;
+    float *part = nullptr;
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    const size_t plane_elems = (size_t)2 * lintc::TN * n_in, part_elems = (size_t)kc * M * n_out;
+    bool ok = dev_alloc(&planes, plane_elems) == cudaSuccess && dev_alloc(&part, part_elems) == cudaSuccess &&
+              cudaEventCreate(&e0) == cudaSuccess && cudaEventCreate(&e1) == cudaSuccess;
+    auto cleanup = [&]() {
+        if (planes) cudaFree(planes);
+        if (part) cudaFree(part);
+        if (e0) cudaEventDestroy(e0);
+        if (e1) cudaEventDestroy(e1);
+    };
+    if (!ok) { cudaGetLastError(); cleanup(); return KNNSSD_ERR_CUDA; }
+    knnssd_status st = KNNSSD_OK;
+    CUtensorMap tw, tx;
+    if (cudaFuncSetAttribute(lintc::linear_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, lintc::SMEM) != cudaSuccess ||
+        !prefill::make_map(&tw, W_dev, (size_t)n_out, (size_t)n_in, lintc::TM) ||
+        !prefill::make_map(&tx, planes, (size_t)2 * lintc::TN, (size_t)n_in, lintc::TN)) {
+        cudaGetLastError();
+        cleanup();
+        return KNNSSD_ERR_CUDA;
+    }
+    cudaMemsetAsync(planes, 0, plane_elems * sizeof(bf16_t), s);
+    lintc::split_x_kernel<<<M, 256, 0, s>>>(x_dev, n_in, planes);
+    lintc::Args a{M, n_in, n_out, kc, kb_per, part, stream_err_ptr()};
+    cudaEventRecord(e0, s);
+    lintc::linear_tc_kernel<<<dim3(tiles, kc), lintc::THREADS, lintc::SMEM, s>>>(tw, tx, a);
+    const size_t n = (size_t)M * n_out;
+    lintc::reduce_chunks_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(part, kc, n, y_dev);
+    cudaEventRecord(e1, s);
+    cudaError_t e = cudaStreamSynchronize(s);
+    if (e == cudaSuccess) e = cudaGetLastError();
+    if (e != cudaSuccess) st = KNNSSD_ERR_CUDA;
+    if (st == KNNSSD_OK) {
+        int code = 0;
+        if (cudaMemcpy(&code, stream_err_ptr(), sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) st = KNNSSD_ERR_CUDA;
+        else if (code) { cudaMemset(stream_err_ptr(), 0, sizeof(int)); st = KNNSSD_ERR_TIMEOUT; }
+    }
+    if (st == KNNSSD_OK && ms_kernels_host) cudaEventElapsedTime(ms_kernels_host, e0, e1);
+    cleanup();
     return st;
 }
 

@@ -3,7 +3,8 @@
     python -m paper_2505_16162_b200.opbench linear --n-out 131072 --n-in 5120 --rows 5 --iters 20
 
 times ``knnssd_linear`` on seeded bf16 weights with CUDA events and prints GB/s (weight bytes / time).
-Several copies of the matrix are cycled through so that every launch reads from HBM, not from L2.
+Several copies of the matrix are cycled through so that every launch reads from HBM, not from L2.  ``linear_tc`` with
+the same options times the stand-alone tensor-core form (``knnssd_linear_tc``, up to 16 rows).
 
     python -m paper_2505_16162_b200.opbench pass --shape llama13b --layers 4 --context 1280 --rows 5 --iters 10
 
@@ -53,6 +54,26 @@ def bench_linear(n_out: int, n_in: int, rows: int, iters: int, warmup: int, dtyp
     us = e0.elapsed_time(e1) * 1e3 / iters
     return {"op": "linear", "n_out": n_out, "n_in": n_in, "rows": rows, "dtype": dtype, "us_per_launch": us,
             "weight_bytes": nbytes, "gbs": nbytes / us / 1e3, "copies_cycled": copies}
+
+
+def bench_linear_tc(n_out: int, n_in: int, rows: int, iters: int, warmup: int, pool_gb: float = 2.0):
+    """The stand-alone tensor-core linear map (``knnssd_linear_tc``), timed by its own CUDA events."""
+    build.build()
+    from . import binding as kb
+    torch.cuda.set_device(0)
+    nbytes = n_out * n_in * 2
+    copies = max(1, min(16, int(pool_gb * (1 << 30)) // nbytes))
+    Ws = [si.normal_weight(7, 100 + i, n_out, n_in, 0.02, "bf16", device="cuda") for i in range(copies)]
+    x = si.normal_f32(8, 99, torch.arange(rows * n_in, device="cuda"), 1.0).view(rows, n_in).contiguous()
+    ms = []
+    for i in range(warmup + iters):
+        _, t = kb.knnssd_linear_tc(Ws[i % copies], x)
+        if i >= warmup:
+            ms.append(t)
+    ms.sort()
+    med = ms[len(ms) // 2]
+    return {"op": "linear_tc", "n_out": n_out, "n_in": n_in, "rows": rows, "us_per_call": med * 1e3,
+            "weight_bytes": nbytes, "gbs": nbytes / med / 1e6, "copies_cycled": copies}
 
 
 def bench_pass(shape_name: str, layers: int, context: int, rows: int, iters: int, seed: int = 0):
@@ -126,7 +147,7 @@ def bench_anchors(n_domains: int, per: int, d: int, iters: int, k: int = 10, see
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("op", choices=["linear", "pass", "prompt", "anchors"])
+    ap.add_argument("op", choices=["linear", "linear_tc", "pass", "prompt", "anchors"])
     ap.add_argument("--shape", default="llama13b")
     ap.add_argument("--layers", type=int, default=4)
     ap.add_argument("--context", type=int, default=1280)
@@ -137,7 +158,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp32"])
     a = ap.parse_args()
-    if a.op == "anchors":
+    if a.op == "linear_tc":
+        print(json.dumps(bench_linear_tc(a.n_out, a.n_in, a.rows, a.iters, a.warmup)))
+    elif a.op == "anchors":
         print(json.dumps(bench_anchors(a.n_out, a.rows, a.n_in, a.iters)))
     elif a.op == "prompt":
         print(json.dumps(bench_prompt(a.shape, a.layers, a.context, a.iters)))

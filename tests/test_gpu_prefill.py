@@ -250,3 +250,29 @@ def test_every_row_count_of_the_common_kernel_with_grouped_heads(kb, shape_name)
         a, nxt = oracle.accept(rows, o["argmax"])
         assert (g["n_accepted"], g["next_token"]) == (a, nxt)
         pending = nxt
+
+
+# ---- weight-streaming linear map for up to 16 rows on the tensor cores (stand-alone) ------------------------
+
+@pytest.mark.parametrize("n_out,n_in,M", [(5120, 5120, 1), (5120, 5120, 16), (1003, 320, 9), (15360, 5120, 5), (130, 13824, 16),
+                                          (40000, 384, 7), (96, 64, 3)])
+def test_linear_tc_matches_oracle(kb, n_out, n_in, M):
+    W, x = _inputs(n_out, n_in, M)
+    want = _oracle_linear(W, x.numpy())
+    got, ms = kb.knnssd_linear_tc(W.cuda(), x.cuda())
+    assert np.abs(got.cpu().numpy() - want).max() < _tol(n_in, want)
+    assert ms > 0
+
+
+def test_linear_tc_rows_do_not_depend_on_the_batch_and_limits(kb):
+    W, x = _inputs(1003, 384, 16)
+    full, _ = kb.knnssd_linear_tc(W.cuda(), x.cuda())
+    for M in (1, 5, 9):
+        part, _ = kb.knnssd_linear_tc(W.cuda(), x[:M].contiguous().cuda())
+        assert torch.equal(part, full[:M])
+    with pytest.raises(kb.KnnssdError) as e:
+        kb.knnssd_linear_tc(W.cuda(), torch.zeros((17, 384), device="cuda"))
+    assert e.value.status == 3
+    with pytest.raises(kb.KnnssdError) as e:
+        kb.knnssd_linear_tc(torch.zeros((8, 96), dtype=torch.bfloat16, device="cuda"), torch.zeros((1, 96), device="cuda"))
+    assert e.value.status == 2
