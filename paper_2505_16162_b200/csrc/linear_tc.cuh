@@ -7,7 +7,8 @@
 // K = 16 per instruction, accumulator 128 lanes x 16 columns of tensor memory, so any row count up to 16 costs the
 // same.  A CTA takes one work item = (tile of 128 units, chunk of the input columns); the chunks' partial sums are
 // written out and added in chunk order by a second kernel (fixed order: the result does not depend on timing).
-// Operands come through TMA (128-byte swizzle) into a ring of 8 stages of 20 KB (16 KB of weights, 2 x 2 KB of x).
+// Operands come through TMA (128-byte swizzle) into a ring of 5 stages of 20 KB (16 KB of weights, 2 x 2 KB of x);
+// two CTAs share an SM.
 // All waits are bounded.
 #pragma once
 
@@ -28,7 +29,7 @@ using stream::smem_u32;
 constexpr int TM = 128;                     // units per tile (accumulator lanes)
 constexpr int TN = 16;                      // rows of x (accumulator columns)
 constexpr int BK = 64;                      // input columns per stage
-constexpr int STAGES = 8;
+constexpr int STAGES = 5;                     // 5 x 20 KB: two CTAs per SM, one streams while the other starts or drains
 constexpr int W_BYTES = TM * BK * 2;        // 16 KB
 constexpr int X_BYTES = TN * BK * 2;        // 2 KB per term
 constexpr int STAGE_BYTES = W_BYTES + 2 * X_BYTES;
@@ -48,7 +49,7 @@ struct Args {
 
 // tw: weights [n_out][K], boxes of 128 rows x 64 columns; tx: x planes [32][K] (rows 0..15 hi, 16..31 lo), boxes of
 // 16 rows x 64 columns.  grid = (ceil(n_out / 128), kc).
-__global__ void __launch_bounds__(THREADS, 1)
+__global__ void __launch_bounds__(THREADS, 2)
 linear_tc_kernel(const __grid_constant__ CUtensorMap tw, const __grid_constant__ CUtensorMap tx, Args g) {
     extern __shared__ unsigned char lt_smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(lt_smem_raw) + 1023) & ~(uintptr_t)1023);
