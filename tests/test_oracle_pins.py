@@ -291,3 +291,93 @@ def test_bf16_gqa_loop_is_lossless():
     mask = si.skip_mask(1, 4, 2)
     _, spec, plain, _, _ = _run("gqa-bf16", mask, 3, 14, prompt_len=20)
     assert np.array_equal(spec["tokens"], plain)
+
+
+# ---- the greedy choice and the cache's rounding points ----------------------------------------------
+
+def test_greedy_choice_is_the_arg_max_of_the_logits():
+    """Drafting equation of Sec. 4.2: the token is arg max of the logits.  The oracle's choice and its margin are
+    compared with numpy's on the logits it returns (full model and a masked draft model)."""
+    shape, w, om = _model("tiny")
+    toks = si.uniform_tokens(6, 0, 24, shape.vocab).numpy()
+    for mask in (None, si.skip_mask(0, 2 * shape.n_layers, 3)):
+        o = oracle.OracleModel(shape, w, 32).forward(toks, 0, skip_mask=mask)
+        lg = o["logits"]
+        assert np.array_equal(o["argmax"], np.argmax(lg, axis=1))
+        assert len(set(o["argmax"].tolist())) > 4              # not a constant
+        top2 = np.sort(lg, axis=1)[:, -2:]
+        assert np.array_equal(o["margin"], top2[:, 1] - top2[:, 0])
+        assert (o["margin"] > 0).all()
+    # only the last head_rows rows get a choice
+    o = oracle.OracleModel(shape, w, 32).forward(toks[:5], 0, head_rows=2)
+    assert (o["argmax"][:3] == -1).all() and np.array_equal(o["argmax"][3:], np.argmax(o["logits"][3:], axis=1))
+
+
+def test_equal_logits_go_to_the_lowest_token_id():
+    """Head rows v and v + V/2 are made identical, so every logit value occurs twice: the lower id must win and the
+    margin is zero."""
+    shape = si.SHAPES["tiny"]
+    w = si.make_model_weights(shape, 0, gain_spread=0.1)
+    half = shape.vocab // 2
+    w["lm_head"][half:] = w["lm_head"][:half]
+    om = oracle.OracleModel(shape, w, 32)
+    toks = si.uniform_tokens(8, 0, 12, shape.vocab).numpy()
+    o = om.forward(toks, 0)
+    lg = o["logits"]
+    assert np.array_equal(lg[:, :half], lg[:, half:])
+    assert (o["argmax"] < half).all()
+    assert np.array_equal(o["argmax"], np.argmax(lg[:, :half], axis=1))
+    assert (o["margin"] == 0).all()
+    # ... and the generation loop follows the same rule
+    _, first, _ = om.prefill(toks)
+    assert first < half
+    out = om.generate(first, 9, 2, si.skip_mask(0, 2 * shape.n_layers, 3))
+    assert (out["tokens"] < half).all() and out["min_margin"] == 0
+
+
+def test_two_position_attention_sees_k_and_v_rounded_to_bf16():
+    """One layer, two positions: the second row's softmax weighs both cached positions, so the result depends on the
+    cached K.  It must equal the fp64 recomputation with the rotated K and V both rounded to bf16 on entering the
+    cache, and differ from the one in which only V is rounded."""
+    shape = si.SHAPES["gqa-bf16"].with_layers(1)
+    w = si.make_model_weights(shape, 5, gain_spread=0.1)
+    w["wq"][0] = w["wq"][0] * 4                                # exact in bf16; spreads the two scores apart
+    w["wk"][0] = w["wk"][0] * 4
+    om = oracle.OracleModel(shape, w, 8)
+    toks = np.array([7, 11], dtype=np.int32)
+    got = om.forward(toks, 0)["logits"][1].astype(np.float64)
+    d, hd, H, Hkv = shape.d_model, shape.head_dim, shape.n_heads, shape.n_kv_heads
+
+    def norm(v, g):
+        return v / torch.sqrt((v * v).mean(dim=-1, keepdim=True) + shape.rms_eps) * _as_f64(g)
+
+    def turn(v, pos):          # v [heads][hd]; dimension i pairs with i + hd/2
+        i = torch.arange(hd // 2, dtype=torch.float64)
+        ang = pos * shape.rope_theta ** (-2.0 * i / hd)
+        a, b = v[:, :hd // 2], v[:, hd // 2:]
+        return torch.cat([a * torch.cos(ang) - b * torch.sin(ang), b * torch.cos(ang) + a * torch.sin(ang)], dim=1)
+
+    def through_cache(t, on):
+        return t.to(torch.float32).to(torch.bfloat16).to(torch.float64) if on else t
+
+    def full(round_k, round_v=True):
+        x = _as_f64(w["tok_embed"])[toks.astype(np.int64)]
+        h = norm(x, w["attn_norm"][0])
+        q = turn((_as_f64(w["wq"][0]) @ h[1]).view(H, hd), 1)
+        ks = torch.stack([through_cache(turn((_as_f64(w["wk"][0]) @ h[p]).view(Hkv, hd), p), round_k) for p in (0, 1)])
+        vs = torch.stack([through_cache((_as_f64(w["wv"][0]) @ h[p]).view(Hkv, hd), round_v) for p in (0, 1)])
+        g = H // Hkv
+        o = torch.zeros(H, hd, dtype=torch.float64)
+        for j in range(H):
+            s = (ks[:, j // g] @ q[j]) / math.sqrt(hd)
+            p = torch.softmax(s, dim=0)
+            o[j] = p @ vs[:, j // g]
+        y = x[1] + _as_f64(w["wo"][0]) @ o.reshape(H * hd)
+        hm = norm(y, w["mlp_norm"][0])
+        y = y + _as_f64(w["w_down"][0]) @ (torch.nn.functional.silu(_as_f64(w["w_gate"][0]) @ hm)
+                                          * (_as_f64(w["w_up"][0]) @ hm))
+        return (_as_f64(w["lm_head"]) @ norm(y, w["final_norm"])).numpy()
+
+    assert np.abs(got - full(True)).max() < 2e-6
+    assert np.abs(got - full(False)).max() > 1e-5
+    assert np.abs(got - full(True, round_v=False)).max() > 1e-5
