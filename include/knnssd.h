@@ -2,10 +2,15 @@
  * knnssd - decode hot path of KNN-SSD self-speculative decoding on one NVIDIA B200.
  *
  * C ABI of libknnssd.so.  Plain pointers and sizes only; every pointer is marked
- * HOST or DEVICE below.  All functions return a knnssd_status (0 = OK); on any
- * non-OK status the session (context length, KV cache validity, active skip mask)
- * is left as it was before the call, nothing aborts or throws across the boundary,
- * and knnssd_last_error() gives a one-line reason.  A context is bound to the CUDA
+ * HOST or DEVICE below.  All functions return a knnssd_status (0 = OK); on a
+ * non-OK status found before anything is enqueued (bad arguments, protocol order,
+ * capacity) the session (context length, KV cache validity, active skip mask) is
+ * left as it was before the call.  A failure found on the device while a pass ran
+ * (KNNSSD_ERR_TIMEOUT, KNNSSD_ERR_CUDA, non-finite logits reported as
+ * KNNSSD_ERR_DEGENERATE) leaves the cache in an unknown state: the context stays
+ * usable but must be prefilled again (calls before that return KNNSSD_ERR_STATE).
+ * Nothing aborts or throws across the boundary, and knnssd_last_error() gives a
+ * one-line reason.  A context is bound to the CUDA
  * device that was current at knnssd_init and to the stream passed there; calls on
  * one context must not overlap (not thread-safe per context).
  *
@@ -35,7 +40,7 @@ typedef enum {
     KNNSSD_ERR_STATE = 4,       /* call out of protocol order (e.g. draft before prefill / before a mask is set) */
     KNNSSD_ERR_DEGENERATE = 5,  /* zero or non-finite vector in the cosine search */
     KNNSSD_ERR_CUDA = 6,        /* a CUDA runtime call failed; text in knnssd_last_error */
-    KNNSSD_ERR_TIMEOUT = 7      /* reserved: a bounded device-side wait gave up */
+    KNNSSD_ERR_TIMEOUT = 7      /* a bounded device-side wait gave up (every wait in the kernels has a poll limit) */
 } knnssd_status;
 
 typedef struct {
@@ -113,7 +118,8 @@ knnssd_status knnssd_prefill(knnssd_ctx *ctx, const int *tokens_host, int n_toke
 knnssd_status knnssd_select_skipset(knnssd_ctx *ctx, const float *query_dev_or_null, int *domain, int *anchor,
                                     float *cosine);
 
-/* Make an explicit mask active.  mask_host: HOST bytes [2*n_layers], 1 = skipped while drafting. */
+/* Make an explicit mask z active (Sec. 3.1: z^(j) = 1 skips sublayer j while drafting; Sec. 4.1: a domain's stored
+ * z*_i is such a mask).  mask_host: HOST bytes [2*n_layers], 1 = skipped while drafting. */
 knnssd_status knnssd_set_skipmask(knnssd_ctx *ctx, const unsigned char *mask_host);
 
 /*
@@ -153,7 +159,8 @@ knnssd_status knnssd_generate(knnssd_ctx *ctx, const int *prompt_host, int n_pro
                               int *domain_or_null, knnssd_stats *stats_or_null);
 
 /*
- * The decode part of knnssd_generate on an already prefilled session: optional select_skipset on the pooled vector
+ * The draft-and-verify loop of Sec. 4.2 (k tokens drafted with M(z), one verification pass of the full model, the
+ * agreeing prefix kept, repeated), i.e. the decode part of knnssd_generate on an already prefilled session: optional select_skipset on the pooled vector
  * of the last prefill, then rounds of draft + verify until max_new tokens are out, the first of them being the
  * pending token.  Arguments as in knnssd_generate.  Statistics of rounds are restarted by this call.
  */
@@ -171,6 +178,8 @@ knnssd_status knnssd_set_length(knnssd_ctx *ctx, int new_len);
 /* Replace the pending token (HOST value); lets a caller teacher-force a token stream. */
 knnssd_status knnssd_set_pending(knnssd_ctx *ctx, int token);
 
+/* Counters behind the paper's reported quantities (App. C.2): mean generated length M = tokens per verification
+ * pass = (accepted + rounds) / rounds, acceptance rate alpha = accepted / drafted; plus device times per phase. */
 knnssd_status knnssd_get_stats(const knnssd_ctx *ctx, knnssd_stats *out);
 const char *knnssd_last_error(const knnssd_ctx *ctx);
 
@@ -216,6 +225,16 @@ knnssd_status knnssd_time_pass(knnssd_ctx *ctx, int which, int k, int iters, flo
 knnssd_status knnssd_trace_pass(knnssd_ctx *ctx, int which, int k, int cap, int *op_types, int *op_layers, float *us_work,
                                 float *us_barrier, int *n_ops);
 
+/*
+ * Test hook for the one device-side failure path (status enum above: KNNSSD_ERR_TIMEOUT).  Launches the persistent
+ * pass kernel on an operation list that holds only the embedding, with a grid barrier that waits for more arrivals
+ * than the launch has CTAs and a poll limit of spin_limit (1..1000000) instead of the kernel's own.  Every CTA's wait
+ * runs out after spin_limit polls (well under a millisecond for a few thousand), the kernel returns normally, and the
+ * call reports KNNSSD_ERR_TIMEOUT after bringing the barrier state back to idle.  Nothing faults or hangs.  The session
+ * then needs a new prefill.  KNNSSD_ERR_SHAPE for models the persistent kernel does not serve.
+ */
+knnssd_status knnssd_debug_barrier_timeout(knnssd_ctx *ctx, unsigned spin_limit);
+
 /* ---- stand-alone operators (same kernels the passes use; for per-kernel tests and measurements) ---- */
 
 /*
@@ -259,7 +278,9 @@ knnssd_status knnssd_linear_tc(const void *W_dev, int n_out, int n_in, const flo
  * The paper does not say how K-means is started or stopped: the starting centroids are an argument, and the iteration
  * stops when a round changes no assignment or after max_rounds rounds.  A round = assign every point to its nearest
  * centroid (squared Euclidean distance, lowest index among equal distances), then move each centroid to the mean of
- * its members (a centroid without members stays).  Distances, sums and centroids are fp64.
+ * its members (a centroid without members stays).  Member sums and centroids are fp64; the assignment compares
+ * distances formed from fp32 differences to the fp32-rounded centroid and accumulated to ~48 bits; Eq. (2) ranks the
+ * members by distances computed entirely in fp64 against the fp64 centroid.
  *   x_dev               DEVICE fp32 [n_points][d], row-major, 16-byte aligned; borrowed
  *   init_centroids_dev  DEVICE fp32 [n_clusters][d]
  *   max_rounds >= 1, 1 <= k, 1 <= n_clusters <= 16 (more: KNNSSD_ERR_CAPACITY), n_points >= n_clusters
@@ -297,7 +318,8 @@ knnssd_status knnssd_cosine_top1(const float *query_dev, const float *anchors_de
  *   limit       n <= KNNSSD_STATIC_MAX_ANCHORS; a larger n returns KNNSSD_ERR_CAPACITY and touches nothing
  *   cost        every GPU that loads the library holds the array (about 16 KB) until the process exits
  *   first call  the first call on each device looks up the array's device address (once per device, with that device
- *               current); make that first call before starting any stream capture
+ *               current).  Every call synchronises the stream and copies its two result words to the host, so it
+ *               cannot run inside a stream capture at all
  *   sharing     all calls on a device use the same array, and it keeps what the previous call left there; the call
  *               clears the words that must start at zero itself.  Two calls that overlap on one GPU (different
  *               streams or host threads) race on it: serialise them

@@ -23,7 +23,8 @@ STATUS = {0: "OK", 1: "ERR_INVALID_ARG", 2: "ERR_SHAPE", 3: "ERR_CAPACITY", 4: "
 EXPORTS = ["knnssd_init", "knnssd_destroy", "knnssd_prefill", "knnssd_select_skipset", "knnssd_set_skipmask",
            "knnssd_draft", "knnssd_verify", "knnssd_generate", "knnssd_decode", "knnssd_get_launch_count", "knnssd_get_length", "knnssd_set_length",
            "knnssd_set_pending", "knnssd_mask_objective", "knnssd_get_stats", "knnssd_last_error", "knnssd_time_pass", "knnssd_trace_pass", "knnssd_linear",
-           "knnssd_gemm_split", "knnssd_linear_tc", "knnssd_build_anchors", "knnssd_cosine_top1", "knnssd_cosine_top1_static"]
+           "knnssd_gemm_split", "knnssd_linear_tc", "knnssd_build_anchors", "knnssd_cosine_top1", "knnssd_cosine_top1_static",
+           "knnssd_debug_barrier_timeout"]
 
 
 class KnnssdError(RuntimeError):
@@ -82,6 +83,7 @@ def _load():
         "knnssd_linear_tc": (I, [P, I, I, P, I, P, PF, P]),
         "knnssd_cosine_top1": (I, [P, P, I, I, PI, PF, P]),
         "knnssd_cosine_top1_static": (I, [P, P, I, I, PI, PF, P]),
+        "knnssd_debug_barrier_timeout": (I, [P, C.c_uint]),
     }
     for name, (res, args) in sigs.items():
         fn = getattr(lib, name)
@@ -174,8 +176,15 @@ def knnssd_build_anchors(x: torch.Tensor, init_centroids: torch.Tensor, max_roun
     return {"labels": labels, "centroids": mu, "anchors": anchors, "rounds": rounds.value, "ms_rounds": ms.value}
 
 
+def _check_query(query: torch.Tensor, anchors: torch.Tensor):
+    # the C entry points get raw pointers and cannot see a query shorter than the anchors' rows
+    if anchors.dim() != 2 or query.numel() != anchors.shape[1]:
+        raise ValueError("anchors must be [n][d] and the query must hold d values")
+
+
 def knnssd_cosine_top1(query: torch.Tensor, anchors: torch.Tensor):
     """(best flat index, cosine) of Eq. (4); raises KnnssdError(ERR_DEGENERATE) on zero / non-finite norms."""
+    _check_query(query, anchors)
     n, d = anchors.shape
     best, cs = C.c_int(), C.c_float()
     with torch.cuda.device(query.device):
@@ -195,6 +204,7 @@ def knnssd_cosine_top1_static(query: torch.Tensor, anchors: torch.Tensor):
     the per-anchor cosines in a fixed array of its own, so nothing is allocated or freed here either - the inputs
     are used in place and the two results come back as Python numbers.  At most ``STATIC_MAX_ANCHORS`` anchors
     (ERR_CAPACITY beyond that).  All calls on a GPU share that array: do not overlap them."""
+    _check_query(query, anchors)
     n, d = anchors.shape
     best, cs = C.c_int(), C.c_float()
     with torch.cuda.device(query.device):
@@ -344,6 +354,10 @@ class Session:
         self._check(_lib.knnssd_mask_objective(self.h, m.ctypes.data, n, toks.ctypes.data, lens.ctypes.data, len(prompts), max_new, k,
                                                ms.ctypes.data, acc.ctypes.data, drf.ctypes.data))
         return ms, acc, drf
+
+    def debug_barrier_timeout(self, spin_limit: int = 4000):
+        """Makes one bounded grid-barrier wait run out (test hook); raises KnnssdError(ERR_TIMEOUT)."""
+        self._check(_lib.knnssd_debug_barrier_timeout(self.h, int(spin_limit)))
 
     def get_stats(self):
         st = Stats()

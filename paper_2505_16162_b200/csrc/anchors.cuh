@@ -181,6 +181,26 @@ __global__ void fold_centroids_kernel(const double *__restrict__ part, const int
     mu[(size_t)c * d + j] = s / (double)counts[c];
 }
 
+// dist[p] = ||x_p - mu_{labels[p]}|| with every difference, square and sum in fp64 against the fp64 centroid: the
+// distances Eq. (2) ranks the members by.  Points at equal distance in exact arithmetic (duplicates, or points mirrored
+// about their centroid) then get equal values, so the lowest index decides among them.  One warp per point, lanes
+// stride over the columns, fixed-order reduction.  Runs once per call.  grid = ceil(N / 8), 256 threads.
+__global__ void __launch_bounds__(256) member_dist_kernel(const float *__restrict__ x, int N, int d, const double *__restrict__ mu,
+                                                          const int *__restrict__ labels, double *__restrict__ dist) {
+    const int lane = threadIdx.x & 31, p = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (p >= N) return;
+    const float *xr = x + (size_t)p * d;
+    const double *m = mu + (size_t)labels[p] * d;
+    double s = 0.0;
+    for (int j = lane; j < d; j += 32) {
+        const double df = (double)__ldg(xr + j) - m[j];
+        s = fma(df, df, s);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) dist[p] = sqrt(s);
+}
+
 // Eq. (2) for cluster c = blockIdx.x: k times, the not yet taken member with the smallest (distance, index);
 // out[c][r] = its index, -1 once the cluster has run out of members.  taken[N] starts at zero.  256 threads.
 __global__ void __launch_bounds__(256) select_anchors_kernel(const double *__restrict__ dist, const int *__restrict__ labels, int N, int k,

@@ -14,6 +14,9 @@ namespace knnssd {
 
 typedef unsigned short bf16_t;  // raw bf16 bit pattern
 
+// Codes a kernel may leave in the device error word (besides the codes of bounded waits that gave up, all < 100).
+enum { ERR_BAD_TOKEN = 101, ERR_BAD_LOGITS = 102 };
+
 // Session scalars that live on the device so that a whole round can be enqueued
 // without the host knowing the accepted count of the previous one.
 struct DeviceState {
@@ -25,10 +28,12 @@ struct DeviceState {
 
 __device__ __forceinline__ float bf16_bits_to_float(unsigned int b) { return __uint_as_float(b << 16); }
 
+// Round to nearest even on the bit pattern.  A NaN stays a NaN (the integer rounding alone would carry the all-ones
+// NaN over into -0, and a non-finite activation would silently turn into zeros downstream).
 __device__ __forceinline__ bf16_t float_to_bf16_rne(float f) {
-    unsigned int u = __float_as_uint(f);
-    u = u + 0x7FFFu + ((u >> 16) & 1u);
-    return (bf16_t)(u >> 16);
+    const unsigned int u = __float_as_uint(f);
+    const unsigned int r = (u + 0x7FFFu + ((u >> 16) & 1u)) >> 16;
+    return (bf16_t)((u & 0x7FFFFFFFu) > 0x7F800000u ? 0x7FC0u : r);
 }
 
 // 16-byte streaming load of weights: read-only path, do not keep in L1.
@@ -82,9 +87,14 @@ __device__ __forceinline__ float warp_max(float v) {
 template <typename WT>
 __global__ void embed_rope_kernel(const WT *__restrict__ E, const int *__restrict__ tok, int d, float *__restrict__ x,
                                   const DeviceState *__restrict__ st, int pos_off, const double *__restrict__ inv_freq,
-                                  int half, float2 *__restrict__ cs) {
+                                  int half, float2 *__restrict__ cs, int vocab, int *__restrict__ err) {
     const int m = blockIdx.x;
-    const WT *row = E + (size_t)tok[m] * d;
+    int t = tok[m];
+    if (t < 0 || t >= vocab) {                 // never gather outside the table: report and read row 0 instead
+        if (threadIdx.x == 0) atomicExch(err, ERR_BAD_TOKEN);
+        t = 0;
+    }
+    const WT *row = E + (size_t)t * d;
     for (int i = threadIdx.x; i < d; i += blockDim.x) x[(size_t)m * d + i] = WeightLoad<WT>::load1(row + i);
     const int pos = st->len + pos_off + m;
     for (int i = threadIdx.x; i < half; i += blockDim.x) {
@@ -394,8 +404,14 @@ __global__ void pool_finish_kernel(const double *__restrict__ sum, int d, double
 // Greedy arg-max per row, lowest index on ties.  Stage 1: grid = (NB, M) blocks scan slices;
 // stage 2: grid = M blocks of 32 threads fold the NB partials.
 // ---------------------------------------------------------------------------------------------
+// A NaN never wins a comparison, so it is passed over like -inf.  A row without any value above -inf (all NaN or
+// -inf) leaves the index at its start value; argmax_checked turns that into token 0 and an error code.
 __device__ __forceinline__ void argmax_fold(float &bv, int &bi, float v, int i) {
     if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
+}
+__device__ __forceinline__ int argmax_checked(int bi, int V, int *err) {
+    if (bi < 0 || bi >= V) { atomicExch(err, ERR_BAD_LOGITS); return 0; }
+    return bi;
 }
 
 __global__ void __launch_bounds__(256) argmax_partial_kernel(const float *__restrict__ logits, int V, int NB,
@@ -423,7 +439,8 @@ __global__ void __launch_bounds__(256) argmax_partial_kernel(const float *__rest
     }
 }
 
-__global__ void argmax_final_kernel(const float *__restrict__ pv, const int *__restrict__ pi, int NB, int *__restrict__ out) {
+__global__ void argmax_final_kernel(const float *__restrict__ pv, const int *__restrict__ pi, int NB, int *__restrict__ out,
+                                    int V, int *__restrict__ err) {
     const int m = blockIdx.x, lane = threadIdx.x;
     float bv = -INFINITY;
     int bi = 0x7fffffff;
@@ -434,7 +451,7 @@ __global__ void argmax_final_kernel(const float *__restrict__ pv, const int *__r
         const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
         argmax_fold(bv, bi, ov, oi);
     }
-    if (lane == 0) out[m] = bi;
+    if (lane == 0) out[m] = argmax_checked(bi, V, err);
 }
 
 // ---------------------------------------------------------------------------------------------

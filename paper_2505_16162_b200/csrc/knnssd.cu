@@ -53,6 +53,9 @@ struct knnssd_ctx {
     int *chain = nullptr, *target = nullptr, *prompt = nullptr, *out_tokens = nullptr, *accept_log = nullptr;
     int *amax_i = nullptr, *flag = nullptr, *knn_out = nullptr;
     DeviceState *state = nullptr;
+    int *err_word = nullptr;   // this device's error word (bounded waits that gave up, bad token ids, non-finite logits)
+    bool enqueue_failed = false;   // a pass could not be enqueued (its operation list did not reach the device)
+    unsigned bar_spin_limit = 0;   // grid-barrier poll limit handed to the pass kernel (0 = its default)
     int *pinned = nullptr;  // host, pinned: small read-backs
     int n_splits = 1;
 
@@ -136,10 +139,23 @@ template <typename WT> void launch_linear_t(const LinearArgs &a, int grid, cudaS
 // Set by the streaming kernel if one of its bounded waits ever gives up (never in normal operation).
 __device__ int g_stream_err;
 
+constexpr int kMaxDevices = 64;
+
+// Index of the current device in the per-device tables below (0 if it cannot be read or is out of range).
+int current_device_slot() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) dev = 0;
+    return dev;
+}
+
+// Address of the error word on the CURRENT device (every device that loads the library has its own copy).
 int *stream_err_ptr() {
-    static int *p = nullptr;
-    if (!p) cudaGetSymbolAddress(reinterpret_cast<void **>(&p), g_stream_err);
-    return p;
+    static int *addr[kMaxDevices] = {};
+    static std::mutex mu;
+    const int dev = current_device_slot();
+    std::lock_guard<std::mutex> lock(mu);
+    if (!addr[dev]) cudaGetSymbolAddress(reinterpret_cast<void **>(&addr[dev]), g_stream_err);
+    return addr[dev];
 }
 
 bool stream_eligible(int dtype, const LinearArgs &a) {
@@ -154,10 +170,11 @@ stream::LinPhase to_phase(const LinearArgs &a) {
 }
 
 void launch_stream(const LinearArgs &a, int n_sms, cudaStream_t s) {
-    static bool configured = false;
-    if (!configured) {
+    static bool configured[kMaxDevices] = {};          // function attributes are per device
+    const int dev = current_device_slot();
+    if (!configured[dev]) {
         cudaFuncSetAttribute(stream::linear_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, stream::SMEM_BYTES);
-        configured = true;
+        configured[dev] = true;
     }
     stream::linear_stream_kernel<<<n_sms, stream::NTHREADS, stream::SMEM_BYTES, s>>>(to_phase(a), stream_err_ptr());
 }
@@ -291,10 +308,11 @@ knnssd_status upload_ops(knnssd_ctx *c, const std::vector<pass::Op> &ops, pass::
 }
 
 template <int HD, int NB> cudaError_t launch_pass_t(knnssd_ctx *c, const pass::Params &pr) {
-    static bool configured = false;
-    if (!configured) {
+    static bool configured[kMaxDevices] = {};          // function attributes are per device
+    const int dev = current_device_slot();
+    if (!configured[dev]) {
         cudaFuncSetAttribute(pass::pass_kernel<HD, NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, stream::SMEM_BYTES);
-        configured = true;
+        configured[dev] = true;
     }
     void *args[] = {const_cast<pass::Model *>(&c->model), const_cast<pass::Params *>(&pr)};
     return cudaLaunchCooperativeKernel(reinterpret_cast<void *>(pass::pass_kernel<HD, NB>), dim3(c->n_sms),
@@ -313,7 +331,7 @@ void run_pass_mega(knnssd_ctx *c, int M, const int *tok_dev, int pos_off, const 
         if (c->ops_draft_mask.size() != n || std::memcmp(c->ops_draft_mask.data(), mask, n) != 0) {
             const std::vector<pass::Op> ops = build_ops(c, mask, &c->bar_draft, &c->attn_draft);
             c->n_ops_draft = (int)ops.size();
-            if (upload_ops(c, ops, c->ops_draft) != KNNSSD_OK) return;
+            if (upload_ops(c, ops, c->ops_draft) != KNNSSD_OK) { c->enqueue_failed = true; return; }
             c->ops_draft_mask.assign(mask, mask + n);
         }
         pr.ops = c->ops_draft; pr.n_ops = c->n_ops_draft; bars = c->bar_draft; n_attn = c->attn_draft;
@@ -321,6 +339,7 @@ void run_pass_mega(knnssd_ctx *c, int M, const int *tok_dev, int pos_off, const 
     pr.M = M; pr.tok = tok_dev; pr.pos_off = pos_off; pr.head_row0 = head_row0; pr.argmax_out = argmax_out;
     pr.want_hidden = want_hidden ? 1 : 0;
     pr.out_row0 = out_row0;
+    pr.bar_spin_limit = c->bar_spin_limit;
     pr.bar_base = c->bar_total;
     if (head_row0 < M) bars += 1;
     pr.merge_op = pass::merge_rows_separately(M, c->cfg.n_heads / c->cfg.n_kv_heads) ? 1 : 0;
@@ -356,7 +375,7 @@ void run_pass_t(knnssd_ctx *c, int M, const int *tok_dev, int pos_off, const uns
     const int nq = H * hd, nkv = Hkv * hd;
     cudaStream_t s = c->stream;
     embed_rope_kernel<WT><<<M, 256, 0, s>>>(reinterpret_cast<const WT *>(c->tok_embed), tok_dev, d, c->x, c->state, pos_off,
-                                            c->inv_freq, hd / 2, c->rope_cs);
+                                            c->inv_freq, hd / 2, c->rope_cs, g.vocab, c->err_word);
     c->launches++;
     const size_t layer_stride = (size_t)Hkv * g.max_seq * hd;
     for (int l = 0; l < g.n_layers; ++l) {
@@ -401,7 +420,7 @@ void run_pass_t(knnssd_ctx *c, int M, const int *tok_dev, int pos_off, const uns
                                 c->logits + (size_t)head_row0 * V, EPI_STORE, hm));
         argmax_partial_kernel<<<dim3(kArgmaxBlocks, hm), 256, 0, s>>>(c->logits + (size_t)head_row0 * V, V, kArgmaxBlocks,
                                                                       c->amax_v, c->amax_i);
-        argmax_final_kernel<<<hm, 32, 0, s>>>(c->amax_v, c->amax_i, kArgmaxBlocks, argmax_out);
+        argmax_final_kernel<<<hm, 32, 0, s>>>(c->amax_v, c->amax_i, kArgmaxBlocks, argmax_out, V, c->err_word);
         c->launches += 2;
     }
 }
@@ -417,19 +436,34 @@ knnssd_status sync_check(knnssd_ctx *c, const char *what) {
     cudaError_t e = cudaStreamSynchronize(c->stream);
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) return fail(c, KNNSSD_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
+    if (c->enqueue_failed) {
+        c->enqueue_failed = false;
+        c->prefilled = false;
+        return fail(c, KNNSSD_ERR_CUDA, std::string(what) + ": a pass could not be enqueued (prefill again): " + c->err);
+    }
     return KNNSSD_OK;
 }
 
-// A bounded wait inside the streaming kernel gave up: report it once and clear the word.
+// What a non-zero device error word means.  Whatever it was, the pass that raised it did not finish: the session's
+// cache and pending token are no longer trustworthy, so the caller has to prefill again.
+knnssd_status fail_device_code(knnssd_ctx *c, const char *what, int code) {
+    cudaMemset(c->err_word, 0, sizeof(int));
+    reset_mega_state(c);
+    c->prefilled = false;
+    if (code == ERR_BAD_LOGITS)
+        return fail(c, KNNSSD_ERR_DEGENERATE, std::string(what) + ": a row of logits holds no finite value (prefill again)");
+    if (code == ERR_BAD_TOKEN)
+        return fail(c, KNNSSD_ERR_INVALID_ARG, std::string(what) + ": a token id on the device was out of range (prefill again)");
+    return fail(c, KNNSSD_ERR_TIMEOUT, std::string(what) + ": a device-side wait gave up (code " + std::to_string(code) +
+                                       "); prefill again");
+}
+
+// Read the device error word (synchronises); reports it once and clears it.
 knnssd_status check_stream_err(knnssd_ctx *c, const char *what) {
     int code = 0;
-    if (cudaMemcpy(&code, stream_err_ptr(), sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess)
+    if (cudaMemcpy(&code, c->err_word, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess)
         return fail(c, KNNSSD_ERR_CUDA, std::string(what) + ": cannot read the device error word");
-    if (code) {
-        cudaMemset(stream_err_ptr(), 0, sizeof(int));
-        reset_mega_state(c);
-        return fail(c, KNNSSD_ERR_TIMEOUT, std::string(what) + ": a device-side wait gave up (code " + std::to_string(code) + ")");
-    }
+    if (code) return fail_device_code(c, what, code);
     return KNNSSD_OK;
 }
 
@@ -469,7 +503,7 @@ bool prefill_tensor(knnssd_ctx *c, int n) {
     const int d = g.d_model, H = g.n_heads, Hkv = g.n_kv_heads, F = g.d_ff, V = g.vocab;
     const int nq = H * HD, nkv = Hkv * HD, ldq = nq + 2 * nkv, cap = c->pf_cap;
     cudaStream_t s = c->stream;
-    int *err = stream_err_ptr();
+    int *err = c->err_word;
     const size_t layer_stride = (size_t)Hkv * g.max_seq * HD;
     bool ok = true;
     for (int t0 = 0; t0 < n && ok; t0 += cap) {
@@ -514,7 +548,7 @@ bool prefill_tensor(knnssd_ctx *c, int n) {
         if (last) {
             ctx_linear(c, make_args(c->lm_head, V, d, c->pf_x + (size_t)(T - 1) * d, c->final_norm, g.rms_eps, c->logits, EPI_STORE, 1));
             argmax_partial_kernel<<<dim3(kArgmaxBlocks, 1), 256, 0, s>>>(c->logits, V, kArgmaxBlocks, c->amax_v, c->amax_i);
-            argmax_final_kernel<<<1, 32, 0, s>>>(c->amax_v, c->amax_i, kArgmaxBlocks, c->chain);
+            argmax_final_kernel<<<1, 32, 0, s>>>(c->amax_v, c->amax_i, kArgmaxBlocks, c->chain, V, c->err_word);
             c->launches += 2;
         }
     }
@@ -663,6 +697,8 @@ knnssd_status knnssd_init(const knnssd_config *cfg, const knnssd_weights *w, con
     auto bail = [&](knnssd_status s) { free_all(c); delete c; return s; };
     if (cudaGetDevice(&c->device) != cudaSuccess) return bail(KNNSSD_ERR_CUDA);
     cudaDeviceGetAttribute(&c->n_sms, cudaDevAttrMultiProcessorCount, c->device);
+    c->err_word = stream_err_ptr();
+    if (!c->err_word) return bail(KNNSSD_ERR_CUDA);
     const int d = g.d_model, hd = g.head_dim, nq = g.n_heads * hd, nkv = g.n_kv_heads * hd;
     const size_t cache_elems = (size_t)g.n_layers * g.n_kv_heads * g.max_seq * hd;
     c->n_splits = (g.max_seq + ATT_CHUNK - 1) / ATT_CHUNK;
@@ -706,6 +742,9 @@ knnssd_status knnssd_init(const knnssd_config *cfg, const knnssd_weights *w, con
     cudaMemcpyAsync(c->inv_freq, inv_freq.data(), sizeof(double) * inv_freq.size(), cudaMemcpyHostToDevice, c->stream);
     set_state_kernel<<<1, 1, 0, c->stream>>>(c->state, 0, 0);
     cudaMemsetAsync(c->flag, 0, sizeof(int), c->stream);
+    // token buffers start at a valid id, so that a pass that ends early never leaves garbage ids behind
+    cudaMemsetAsync(c->chain, 0, sizeof(int) * (kMaxRows + 1), c->stream);
+    cudaMemsetAsync(c->target, 0, sizeof(int) * kMaxRows, c->stream);
     if (na > 0) anchor_inv_norm_kernel<<<(na + 7) / 8, 256, 0, c->stream>>>(c->anchors, na, d, c->anchor_inv_norm, c->flag);
     cudaMemcpyAsync(c->pinned, c->flag, sizeof(int), cudaMemcpyDeviceToHost, c->stream);
     if (sync_check(c, "init") != KNNSSD_OK) return bail(KNNSSD_ERR_CUDA);
@@ -760,7 +799,7 @@ knnssd_status knnssd_init(const knnssd_config *cfg, const knnssd_weights *w, con
         md.n_seg_max = n_seg_max; md.inv_freq = c->inv_freq;
         md.x = c->x; md.qkv = c->qkv; md.attn = c->attn; md.logits = c->logits; md.hfinal = c->hfinal; md.rope_cs = c->rope_cs;
         md.part_o = c->mpart_o; md.part_ml = c->mpart_ml; md.attn_cnt = c->attn_cnt; md.amax_v = c->mamax_v; md.amax_i = c->mamax_i;
-        md.amax_cnt = c->amax_cnt; md.state = c->state; md.bar = c->bar; md.gabort = c->gabort; md.err = stream_err_ptr();
+        md.amax_cnt = c->amax_cnt; md.state = c->state; md.bar = c->bar; md.gabort = c->gabort; md.err = c->err_word;
         c->mega_ok = true;
         reset_mega_state(c);
         const std::vector<pass::Op> ops = build_ops(c, nullptr, &c->bar_full, &c->attn_full);
@@ -899,8 +938,11 @@ static knnssd_status do_decode(knnssd_ctx *c, int max_new, int k, int use_select
         enqueue_verify(c, keff, false, round);
         cudaEventRecord(c->ev2, s);
         CUDA_TRY(c, cudaMemcpyAsync(c->pinned, c->state, sizeof(DeviceState), cudaMemcpyDeviceToHost, s));
+        CUDA_TRY(c, cudaMemcpyAsync(c->pinned + 8, c->err_word, sizeof(int), cudaMemcpyDeviceToHost, s));
         st = sync_check(c, "decode");
         if (st != KNNSSD_OK) return st;
+        // a pass that gave up (or met a bad id / non-finite logits) must not be committed to the session
+        if (c->pinned[8]) return fail_device_code(c, "decode", c->pinned[8]);
         const DeviceState *hs = reinterpret_cast<const DeviceState *>(c->pinned);
         float ms = 0.f;
         cudaEventElapsedTime(&ms, c->ev0, c->ev1);
@@ -1139,6 +1181,36 @@ knnssd_status knnssd_trace_pass(knnssd_ctx *c, int which, int k, int cap, int *o
     return st;
 }
 
+knnssd_status knnssd_debug_barrier_timeout(knnssd_ctx *c, unsigned spin_limit) {
+    if (!c) return KNNSSD_ERR_INVALID_ARG;
+    DeviceGuard dg(c->device);
+    if (spin_limit < 1 || spin_limit > 1000000u) return fail(c, KNNSSD_ERR_INVALID_ARG, "debug_barrier_timeout: spin_limit must be 1..1000000");
+    if (!c->mega_ok) return fail(c, KNNSSD_ERR_SHAPE, "debug_barrier_timeout: this model does not run in the persistent kernel");
+    // an operation list holding just the embedding (no linear map: the producer warp issues no copy) whose barrier
+    // waits for one more round of arrivals than there are CTAs; every CTA runs out of polls, raises the abort word and
+    // falls through to the end of the kernel
+    pass::Op e{};
+    e.type = pass::OP_EMBED; e.barrier_after = 1;
+    e.lin.K = c->cfg.d_model; e.lin.ys = c->xs_x; e.lin.ss_out = c->ssp;
+    std::vector<pass::Op> ops(1, e);
+    c->ops_draft_mask.clear();                       // the draft list's slot is reused: it is rebuilt on the next draft
+    knnssd_status st = upload_ops(c, ops, c->ops_draft);
+    if (st != KNNSSD_OK) return st;
+    pass::Params pr{};
+    pr.ops = c->ops_draft; pr.n_ops = 1; pr.M = 1; pr.tok = c->chain; pr.pos_off = 0; pr.head_row0 = 1;
+    pr.argmax_out = c->target; pr.bar_spin_limit = spin_limit;
+    pr.bar_base = c->bar_total + (unsigned long long)c->n_sms;   // one CTA-count beyond what this launch can reach
+    const cudaError_t le = c->cfg.head_dim == 128 ? launch_pass_t<128, 1>(c, pr) : launch_pass_t<64, 1>(c, pr);
+    c->launches++;
+    if (le != cudaSuccess) return fail(c, KNNSSD_ERR_CUDA, std::string("debug_barrier_timeout: ") + cudaGetErrorString(le));
+    st = sync_check(c, "debug_barrier_timeout");
+    if (st != KNNSSD_OK) return st;
+    // the launch left n_sms arrivals on the counter: without an error the next pass would be off by them
+    st = check_stream_err(c, "debug_barrier_timeout");
+    if (st == KNNSSD_OK) { reset_mega_state(c); c->prefilled = false; }
+    return st;
+}
+
 knnssd_status knnssd_linear(const void *W_dev, int dtype, int n_out, int n_in, const float *x_dev, int M, float *y_dev,
                             void *cuda_stream) {
     if (!W_dev || !x_dev || !y_dev || n_out < 1 || n_in < 8 || M < 1 || M > kMaxRows || (dtype != 0 && dtype != 1))
@@ -1326,9 +1398,9 @@ knnssd_status knnssd_build_anchors(const float *x_dev, int n_points, int d, int 
         ms_total += ms;
     }
     if (e == cudaSuccess) {
-        // the anchors are measured against the final centroids (they moved after the last assignment if the round
-        // limit ended the iteration)
-        if (changed) launch_assign(0);
+        // the anchors are ranked by fp64 distances to the final fp64 centroids (which moved after the last assignment
+        // if the round limit ended the iteration)
+        anchors::member_dist_kernel<<<(N + 7) / 8, 256, 0, s>>>(x_dev, N, d, mu, labels, dist);
         cudaMemsetAsync(taken, 0, (size_t)N, s);
         anchors::select_anchors_kernel<<<n, 256, 0, s>>>(dist, labels, N, k, taken, out);
         e = cudaMemcpyAsync(anchors_host, out, sizeof(int) * n * k, cudaMemcpyDeviceToHost, s);
@@ -1376,7 +1448,6 @@ knnssd_status knnssd_cosine_top1(const float *query_dev, const float *anchors_de
 // In host code the name below is only a handle for cudaGetSymbolAddress; kernels get the address that call returns.
 namespace {
 constexpr int kStaticWords = KNNSSD_STATIC_MAX_ANCHORS + 4;
-constexpr int kMaxDevices = 64;
 }  // namespace
 static __device__ __align__(256) float g_top1_static_scratch[kStaticWords];
 

@@ -73,6 +73,7 @@ struct Params {
     int out_row0;              // row of the logits / hidden-state buffers that this pass's row 0 goes to
     unsigned long long bar_base;   // value of *bar when this launch starts
     int merge_op;              // the attention partials are merged by the separate merge operation (merge_rows_separately)
+    unsigned bar_spin_limit;   // polls a grid-barrier wait may take before the pass is aborted (0 = BAR_SPIN_LIMIT)
 };
 
 // Whether a pass of M rows merges its attention partials in the separate operation: when an attention task carries
@@ -95,7 +96,8 @@ __device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long
 }
 
 // Called by all 256 consumer threads.  Returns false once the pass has been aborted.
-__device__ __forceinline__ bool grid_barrier(const Model &md, const Ring &r, unsigned long long target, int tid, bool alive) {
+__device__ __forceinline__ bool grid_barrier(const Model &md, const Ring &r, unsigned long long target, int tid, bool alive,
+                                             unsigned spin_limit) {
     asm volatile("bar.sync 1, %0;" ::"n"(NCW * 32) : "memory");
     if (tid == 0 && alive) {
         __threadfence();                       // cumulative: covers the writes of the CTA's other threads ordered by the bar.sync
@@ -103,7 +105,7 @@ __device__ __forceinline__ bool grid_barrier(const Model &md, const Ring &r, uns
         unsigned spins = 0;
         while (ld_acquire_u64(md.bar) < target) {
             if (*r.abort_flag || *reinterpret_cast<volatile int *>(md.gabort)) { *r.abort_flag = 1; break; }
-            if (++spins > BAR_SPIN_LIMIT) {
+            if (++spins > spin_limit) {
                 *r.abort_flag = 1;
                 atomicExch(md.gabort, 1);
                 atomicExch(md.err, 7);
@@ -133,7 +135,12 @@ __device__ __forceinline__ void embed_phase(const Model &md, const Op &op, const
     if (cta >= pr.M) return;                               // whole CTAs only: the named barrier below is CTA-local
     // row m = cta: residual stream in fp32, its pre-split form times the first RMSNorm's gain, its sum of squares
     const int m = cta, lane = tid & 31, warp = tid >> 5;
-    const bf16_t *row = md.tok_embed + (size_t)pr.tok[m] * d;
+    int t = pr.tok[m];
+    if (t < 0 || t >= md.vocab) {                          // never gather outside the table: report and read row 0 instead
+        if (tid == 0) atomicExch(md.err, ERR_BAD_TOKEN);
+        t = 0;
+    }
+    const bf16_t *row = md.tok_embed + (size_t)t * d;
     float ss = 0.f;
     for (int i = tid; i < d; i += NCW * 32) {
         const float v = bf16_bits_to_float(row[i]);
@@ -215,7 +222,7 @@ __device__ __forceinline__ void argmax_phase(const Model &md, const Params &pr, 
                     const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
                     argmax_fold(bv, bi, ov, oi);
                 }
-                if (lane == 0) pr.argmax_out[m] = bi;
+                if (lane == 0) pr.argmax_out[m] = argmax_checked(bi, V, md.err);
             }
         }
         if (tid == 0) *md.amax_cnt = 0;
@@ -310,9 +317,6 @@ __device__ __forceinline__ void attn_merge_row(const Model &md, const Op &op, in
     for (int e = 0; e < DPL; ++e) stream::store_split(op.lin.ys, (H * HD) >> 7, m, h * HD + d0 + e, acc[e] / L);
 }
 
-#ifndef KNNSSD_ATT_STAMP
-#define KNNSSD_ATT_STAMP(i)
-#endif
 
 // Tensor-core form.  Lane (g8, t4) = (lane / 4, lane % 4).  The pass's rows are the rows 0..7 of the 16-row MMA
 // operand (row m = g8), so the cost does not depend on how many rows the pass carries.
@@ -374,8 +378,6 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
         // pass row g8's own position lies in this segment and is not in the cache yet: this lane rotates / rounds its K, V
         const bool row_new = !all_cached && g8 < M && P0 + g8 >= p_begin && P0 + g8 < p_end;
         const bool row_live = row_in && rm >= m_first;
-
-        KNNSSD_ATT_STAMP(0);
         // ---- this lane's run of q (row g8), of the new K row and of the new V row: load, rotate, round / split ----
         float qf[DL], kf[DL];
         {
@@ -429,8 +431,6 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
             const uint32_t l1 = float_to_bf16_rne(qf[2 * w + 1] - __uint_as_float(h1 << 16));
             qh[w] = h0 | (h1 << 16); ql[w] = l0 | (l1 << 16);
         }
-
-        KNNSSD_ATT_STAMP(1);
         // ---- scores: one tile = 8 positions; K rows are fetched two tiles ahead ----
         auto load_k = [&](int nt, uint4 (&dst)[NW / 4]) {
             const int p = p_begin + 8 * nt + g8;
@@ -462,7 +462,6 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
                 if (nt + KR < NT) load_k(nt + KR, kq);
             }
         }
-        KNNSSD_ATT_STAMP(2);
         // ---- V rows of the first tiles start moving while the softmax runs ----
         auto load_v = [&](int nt, uint4 (&dst)[2][(VW + 3) / 4]) {
 #pragma unroll
@@ -483,8 +482,6 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
         uint4 vb[VR][2][(VW + 3) / 4];
 #pragma unroll
         for (int i = 0; i < VR; ++i) load_v(i, vb[i]);
-
-        KNNSSD_ATT_STAMP(3);
         // ---- softmax over the segment for row g8 (the four lanes of a row share it) ----
         float mx = -INFINITY;
 #pragma unroll
@@ -509,8 +506,6 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
             }
         lsum += __shfl_xor_sync(0xffffffffu, lsum, 1);
         lsum += __shfl_xor_sync(0xffffffffu, lsum, 2);
-
-        KNNSSD_ATT_STAMP(4);
         // ---- o += p V ----
         float o[VJ][4];
 #pragma unroll
@@ -543,8 +538,6 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
             if (np + VR < NT) load_v(np + VR, vb[np % VR]);
             if (np + 1 + VR < NT) load_v(np + 1 + VR, vb[(np + 1) % VR]);
         }
-
-        KNNSSD_ATT_STAMP(5);
         // ---- partials out (row g8: dimensions DL*t4 + j and DL*t4 + VJ + j); the last warp of a (row, head) merges ----
         if (row_live) {
             const size_t pidx = ((size_t)rm * H + h) * md.n_seg_max + seg;
@@ -559,13 +552,11 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
         if (defer_merge) continue;                            // a separate merge operation follows a grid barrier
         __threadfence();
         __syncwarp();
-        KNNSSD_ATT_STAMP(6);
         bool last = false;
         if (row_live && t4 == 0) {
             const int n_seg_m = (P0 + rm + SEGP) / SEGP;                  // segments row rm sees
             last = atomicAdd(md.attn_cnt + rm * H + h, 1) == n_seg_m - 1;
         }
-        KNNSSD_ATT_STAMP(7);
         const unsigned last_mask = __ballot_sync(0xffffffffu, last);     // bit 4*g set: this warp finishes the (row, head) of lane row g
         if (last_mask) {
             __threadfence();
@@ -577,7 +568,6 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
                 if (lane == 0) md.attn_cnt[mg * H + hg] = 0;
             }
         }
-        KNNSSD_ATT_STAMP(8);
     }
 }
 
@@ -683,7 +673,8 @@ __global__ void __launch_bounds__(stream::NTHREADS, 1) pass_kernel(const Model m
         if (md.trace && cta == 0 && tid == 0) md.trace[2 * i] = globaltimer_ns();
         if (op.barrier_after && ran) {
             ++n_bar;
-            alive = grid_barrier(md, r, pr.bar_base + n_bar * (unsigned long long)n_cta, tid, alive);
+            alive = grid_barrier(md, r, pr.bar_base + n_bar * (unsigned long long)n_cta, tid, alive,
+                                 pr.bar_spin_limit ? pr.bar_spin_limit : BAR_SPIN_LIMIT);
         }
         if (md.trace && cta == 0 && tid == 0) md.trace[2 * i + 1] = globaltimer_ns();
     }

@@ -27,26 +27,13 @@ def _blobs(seed, n, per, d, spread):
     return X[rng.permutation(X.shape[0])].astype(np.float32)
 
 
-def _check(kb, X, init, max_rounds, k, tied=False):
-    """tied: the case has members at exactly equal distances in exact arithmetic (duplicated points mirrored about
-    their centroid).  The kernel measures distances against the fp32-rounded centroid, which can split such a tie, so
-    there the anchors are compared by what is unique - the distances - and checked to be members, nearest first."""
+def _check(kb, X, init, max_rounds, k):
     want = oa.build_anchors(X, init.astype(np.float64), max_rounds, k)
     got = kb.knnssd_build_anchors(torch.tensor(X).cuda(), torch.tensor(init).cuda(), max_rounds, k)
     assert got["rounds"] == want["rounds"]
     assert np.array_equal(got["labels"], want["labels"])
     assert np.abs(got["centroids"].cpu().numpy() - want["centroids"]).max() < 1e-10
-    if not tied:
-        assert np.array_equal(got["anchors"], want["anchors"])
-    else:
-        assert np.array_equal(got["anchors"] < 0, want["anchors"] < 0)
-        for c in range(want["anchors"].shape[0]):
-            g, w = got["anchors"][c], want["anchors"][c]
-            g, w = g[g >= 0], w[w >= 0]
-            assert len(set(g.tolist())) == len(g) and (want["labels"][g] == c).all()
-            dg = np.linalg.norm(X[g].astype(np.float64) - want["centroids"][c], axis=1)
-            dw = np.linalg.norm(X[w].astype(np.float64) - want["centroids"][c], axis=1)
-            assert np.abs(dg - dw).max() < 1e-5 * max(1.0, dw.max())
+    assert np.array_equal(got["anchors"], want["anchors"])
     return want, got
 
 
@@ -83,7 +70,7 @@ def test_round_limit_small_and_empty_clusters(kb):
     assert (want["anchors"][2] == -1).all()
     assert np.array_equal(got["centroids"][2].cpu().numpy(), far[2].astype(np.float64))
     tiny = np.concatenate([X[:5], X[:5]])                              # duplicates: equal distances, lowest index first
-    _check(kb, tiny, tiny[:2].copy(), 20, 6, tied=True)
+    _check(kb, tiny, tiny[:2].copy(), 20, 6)
 
 
 def test_build_anchors_rejects_bad_arguments(kb):

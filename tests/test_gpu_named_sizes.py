@@ -1,0 +1,129 @@
+"""The full-size workloads against token streams the CPU oracle wrote beforehand (``tests/golden/tokens_*.json``).
+
+The oracle needs seconds per pass on 32 / 40 / 48-layer models, so its output is stored once by
+``tests/golden/make_token_goldens.py`` (which calls only ``oracle/`` and ``synthetic_inputs/``); here the same seeded
+inputs are rebuilt on the GPU from the recipe in each file and run through the C ABI as a user would: prompt pass,
+cosine selection of the domain's mask, self-speculative decoding.  Exact: first token, selected domain and anchor,
+every generated token, every round's accept count.  Within 2e-2: the pooled last hidden state and the logits of one
+teacher-forced verification pass at the end of the prompt, on the entries the file samples.  Depth, width, prompt
+length and draft length are the workloads' own; a file whose ``cut`` field is set generated fewer tokens than the
+workload names (oracle time), nothing else.
+"""
+import glob
+import json
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import synthetic_inputs as si
+
+pytestmark = pytest.mark.gpu
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+FILES = sorted(glob.glob(os.path.join(HERE, "golden", "tokens_*.json")),
+               key=lambda p: (json.load(open(p))["shape"], json.load(open(p)).get("gamma", 1.0), p))
+TOL = 2e-2
+
+_weights = {}          # at most one model resident: (shape, seed, damp key) -> weights
+
+
+@pytest.fixture(scope="module")
+def kb():
+    if not torch.cuda.is_available():
+        pytest.fail("the gpu tests need a CUDA device")
+    from paper_2505_16162_b200 import build
+    build.build()
+    from paper_2505_16162_b200 import binding
+    return binding
+
+
+def _model_weights(shape, seed, damp):
+    key = (shape.name, seed, tuple(sorted((damp or {}).items())))
+    if key not in _weights:
+        _weights.clear()
+        torch.cuda.empty_cache()
+        _weights[key] = si.make_model_weights(shape, seed, device="cuda", damp=damp)
+    return _weights[key]
+
+
+def _masks(rec, shape):
+    seed, skip = rec["seed"], rec["skip"]
+    if "pool" in rec:
+        return si.nested_skip_masks(seed + 100, shape.n_layers, rec["n_domains"], rec["pool"][0], rec["pool"][1], skip[0], skip[1])[1]
+    return np.stack([si.skip_mask_split(seed + 100 + i, shape.n_layers, skip[0], skip[1]) for i in range(rec["n_domains"])])
+
+
+def test_golden_files_are_present():
+    assert FILES, "no tests/golden/tokens_*.json"
+
+
+@pytest.mark.parametrize("path", FILES, ids=[os.path.basename(p)[7:-5] for p in FILES])
+def test_workload_matches_the_oracles_stored_output(kb, path):
+    rec = json.load(open(path))
+    shape = si.SHAPES[rec["shape"]]
+    seed, k, max_new = rec["seed"], rec["k"], rec["max_new"]
+    nd, per = rec["n_domains"], rec["anchors_per_domain"]
+    masks = _masks(rec, shape)
+    damp = None
+    if "gamma" in rec:
+        damp = {int(j): rec["gamma"] for j in np.nonzero(masks[rec["shaped_domain"]])[0]}
+    w = _model_weights(shape, seed, damp)
+    anchors = si.anchors(seed, nd, per, shape.d_model, rec["sigma_a"]).cuda()
+    stream = "requests_per_domain" in rec
+    if stream:
+        labels = si.request_stream(seed, nd, rec["requests_per_domain"], rec["mix_ratio"])
+        lengths = si.prompt_lengths(seed, nd * rec["requests_per_domain"], *rec["prompt_range"])
+        cen = si.domain_centroids(seed, nd, shape.d_model).cuda()
+    max_seq = max(r["prompt_len"] for r in rec["requests"]) + max_new + 64
+    sess = kb.Session.from_shape(shape, w, max_seq, max_draft=max(k, 8), anchors=anchors, skip_masks=masks,
+                                 anchors_per_domain=per)
+    worst_logit, worst_pooled = 0.0, 0.0
+    for r in rec["requests"]:
+        P = r["prompt_len"]
+        if stream:
+            i = r["index"]
+            assert labels[i] == r["label"] and lengths[i] == P
+            prompt = si.uniform_tokens(seed, 1 + i, P, shape.vocab).numpy()
+        else:
+            prompt = si.uniform_tokens(seed, 0, P, shape.vocab).numpy()
+        first, pooled = sess.prefill(prompt, want_pooled=True)
+        assert first == r["first_token"], f"first token; oracle margin {r['first_margin']}"
+        pg = pooled[torch.tensor(r["pooled_index"], device="cuda")].cpu().numpy()
+        worst_pooled = max(worst_pooled, float(np.abs(pg - np.array(r["pooled"], dtype=np.float32)).max()))
+        assert worst_pooled < TOL
+        if stream:
+            c = cen[r["label"]]
+            query = (pooled + 4.0 * pooled.norm() / c.norm() * c).contiguous()   # a draw from the domain's cluster
+            dom, anc, cos = sess.select_skipset(query)
+            assert dom == r["label"]
+        else:
+            dom, anc, cos = sess.select_skipset()
+        assert (dom, anc) == (r["domain"], r["anchor"]), f"selection; oracle gap between domains {r['domain_gap']}"
+        assert abs(cos - r["cosine"]) < 1e-4
+        if "explicit_mask_domain" in rec:
+            sess.set_skipmask(masks[rec["explicit_mask_domain"]])
+        got = sess.decode(max_new, k)
+        want_tokens, want_accepts = np.array(r["tokens"], np.int32), np.array(r["accepts"], np.int32)
+        bad = np.nonzero(got["tokens"] != want_tokens)[0]
+        assert bad.size == 0, f"first differing token at {bad[0]}; oracle's smallest decisive margin {r['min_margin']}"
+        assert np.array_equal(got["accepts"], want_accepts)
+        st = got["stats"]
+        assert (st["rounds"], st["drafted"], st["accepted"]) == (r["rounds"], r["drafted"], r["accepted"])
+        # one teacher-forced verification pass at the prompt's end: sampled logits of every row
+        sess.set_length(P)
+        sess.set_pending(first)
+        rows = r["verify_rows"]
+        assert rows[0] == first
+        g = sess.verify(rows[1:], want_logits=True)
+        lg = g["logits"][:, torch.tensor(r["logit_index"], device="cuda")].cpu().numpy()
+        worst_logit = max(worst_logit, float(np.abs(lg - np.array(r["logits"], dtype=np.float32)).max()))
+        assert worst_logit < TOL
+        n_acc = 0
+        while n_acc < len(rows) - 1 and r["verify_argmax"][n_acc] == rows[n_acc + 1]:
+            n_acc += 1
+        assert (g["n_accepted"], g["next_token"]) == (n_acc, r["verify_argmax"][n_acc])
+    sess.close()
+    print(f"\n[{rec['case']}] max |logit - oracle| on sampled entries {worst_logit:.3e}, pooled {worst_pooled:.3e}, "
+          f"oracle min margin {min(r['min_margin'] for r in rec['requests']):.3e}")

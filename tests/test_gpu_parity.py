@@ -355,3 +355,42 @@ def test_rollback_then_replay_gives_the_same_tokens(kb):
     sess.set_pending(first)
     b = [sess.verify(sess.draft(4))["next_token"] for _ in range(3)]
     assert a == b and sess.length == len_after
+
+
+# ---- contexts beyond 2048 positions ------------------------------------------------------------------
+
+@pytest.mark.parametrize("shape_name", ["stream64-bf16", "stream-bf16"])
+def test_context_beyond_2048_positions_matches_oracle(kb, shape_name):
+    """A 2100-token prompt (three chunks of the prompt pass; 33 attention segments, so the merge's second set of segment
+    statistics is in use), then teacher-forced verification rows and a generated stretch against the live oracle."""
+    P, max_seq = 2100, 2300
+    base = si.SHAPES[shape_name]
+    mask = si.skip_mask(0, 2 * base.n_layers, 2)
+    damp = {int(j): 0.05 for j in np.nonzero(mask)[0]}
+    shape, om, sess = _pair(kb, shape_name, max_seq=max_seq, damp=damp)
+    prompt = si.uniform_tokens(3, 0, P, shape.vocab).numpy()
+    pooled_o, first_o, _ = om.prefill(prompt)
+    first_g, pooled_g = sess.prefill(prompt, want_pooled=True)
+    assert first_g == first_o
+    assert np.abs(pooled_g.cpu().numpy() - pooled_o).max() < TOL["bf16"]
+    sess.set_skipmask(mask)
+    n, pending = P, first_o
+    forced = si.uniform_tokens(9, 1, 40, shape.vocab).numpy()
+    fi = 0
+    for k in (4, 8, 0, 2):
+        rows = forced[fi:fi + k]
+        fi += k
+        o = om.forward(np.concatenate([[pending], rows]).astype(np.int32), n, want_hidden=True)
+        g = sess.verify(rows, want_logits=True, want_hidden=True)
+        assert np.abs(g["logits"].cpu().numpy() - o["logits"]).max() < TOL["bf16"]
+        assert np.abs(g["hidden"].cpu().numpy() - o["hidden"]).max() < TOL["bf16"]
+        a, nxt = oracle.accept(rows, o["argmax"])
+        assert (g["n_accepted"], g["next_token"]) == (a, nxt)
+        n += a + 1
+        om.length = n
+        pending = nxt
+    want = om.generate(pending, 20, 4, mask)
+    got = sess.decode(20, 4)
+    assert np.array_equal(got["tokens"], want["tokens"]), f"oracle min margin {want['min_margin']}"
+    assert np.array_equal(got["accepts"], want["accepts"])
+    assert sess.length == om.length > 2048 + 64

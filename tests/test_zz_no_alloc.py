@@ -1,4 +1,4 @@
-"""The allocation-free cosine search against the ordinary one (collected last on purpose).
+"""The allocation-free cosine search against the ordinary one and against the CPU oracle (collected last on purpose).
 
 Some callers cannot call cudaMalloc: a serving loop that lives inside a memory pool sized at start-up, a process
 under a fixed GPU memory reservation, a latency path that cannot afford cudaFree's implicit synchronisation.
@@ -10,6 +10,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 import synthetic_inputs as si
 
 pytestmark = pytest.mark.gpu
@@ -30,6 +31,9 @@ def _same(kb, query, anchors):
     got = kb.knnssd_cosine_top1_static(query, anchors)
     assert got[0] == want[0]
     assert abs(got[1] - want[1]) < 1e-5          # the tolerance the cosine parity tests use; same kernels, so equal
+    # ... and both against the oracle's Eq. (4) on the same inputs (one domain holding all the anchors)
+    dom, anc, cs = oracle.knn_select(query.cpu().numpy(), anchors.cpu().numpy(), 1, anchors.shape[0])
+    assert got[0] == anc and abs(got[1] - cs) < 1e-5
     return got
 
 
@@ -56,5 +60,7 @@ def test_static_scratch_variant_refuses_more_anchors_than_it_holds(kb):
     with pytest.raises(kb.KnnssdError) as e:
         kb.knnssd_cosine_top1_static(q, anchors)
     assert e.value.status == 3
-    # at the limit it still works and agrees with the allocating call (all cosines equal: lowest index wins)
+    # at the limit it still works and agrees with the allocating call and the oracle (all cosines equal: lowest index wins)
     assert _same(kb, q, anchors[:-1].contiguous())[0] == 0
+    with pytest.raises(ValueError):                   # the binding refuses a query shorter than the anchors' rows
+        kb.knnssd_cosine_top1_static(q[:4].contiguous(), anchors[:-1].contiguous())
