@@ -18,6 +18,7 @@ from .generators import (  # noqa: F401
     normal_f32,
     normal_weight,
     uniform_tokens,
+    uniforms,
     skip_mask,
     skip_mask_split,
     nested_skip_masks,

@@ -107,6 +107,13 @@ def uniform_tokens(seed: int, stream_id: int, n: int, vocab: int, device="cpu") 
     return (_lsr(h, 1) % vocab).to(torch.int32)
 
 
+def uniforms(seed: int, stream_id: int, n: int) -> np.ndarray:
+    """n uniforms in [0, 1) as fp64 multiples of 2**-24 (exactly representable in fp32 too): the top 24 bits of the
+    hash of (seed, UNIFORM + stream_id, index).  The random draws a sampling method consumes are handed to it as inputs."""
+    return np.array([(hash_u64_int(seed, TensorId.UNIFORM + stream_id, i) >> 40) / float(1 << 24) for i in range(n)],
+                    dtype=np.float64)
+
+
 def _ranks(seed: int, tensor_id: int, n: int) -> np.ndarray:
     keys = [hash_u64_int(seed, tensor_id, j) for j in range(n)]
     return np.argsort(np.array(keys, dtype=np.uint64), kind="stable")
@@ -217,6 +224,7 @@ class TensorId:
     STREAM = 7
     LENGTH = 8
     LAYER0 = 64          # layer l uses LAYER0 + 8*l + {0 wq, 1 wk, 2 wv, 3 wo, 4 gate, 5 up, 6 down, 7 gains}
+    UNIFORM = 1 << 19    # + stream id
     PROMPT = 1 << 20     # + stream id
 
 
