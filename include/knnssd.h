@@ -298,6 +298,40 @@ knnssd_status knnssd_build_anchors(const float *x_dev, int n_points, int d, int 
                                    void *cuda_stream);
 
 /*
+ * Sampled decoding (App. C.1 lists temperature 0.2 and top-p 0.85 in the decoding set-up; Sec. 1 and Sec. 3.1: the
+ * method leaves the distribution of the generated tokens unchanged).  The paper prints no acceptance rule for the sampled
+ * case; these three operators implement the rule of speculative sampling that has that property, on the logits that
+ * knnssd_draft / knnssd_verify return.  Random numbers are INPUTS: one uniform in [0, 1) per draw.
+ *
+ * knnssd_filtered_probs: probs[r] = softmax(logits[r] / temperature) restricted to its nucleus and renormalised; a
+ *   token is kept iff the probability of the tokens ranked before it (higher probability first, lower id first among
+ *   equals) is below top_p, so at least one token is kept.  logits_dev, probs_dev DEVICE fp32 [rows][vocab] (may not
+ *   overlap); temperature > 0, top_p > 0 (top_p > 1 keeps every token).  Asynchronous on the stream.
+ */
+knnssd_status knnssd_filtered_probs(const float *logits_dev, int rows, int vocab, float temperature, float top_p,
+                                    float *probs_dev, void *cuda_stream);
+
+/*
+ * knnssd_sample_token: inverse CDF in token-id order - the smallest id x with w_0 + .. + w_x > u * sum(w).
+ *   weights_dev DEVICE fp32 [vocab], non-negative, not necessarily normalised, with a positive sum; 0 <= u < 1;
+ *   token_host HOST output.  Synchronises the stream.
+ */
+knnssd_status knnssd_sample_token(const float *weights_dev, int vocab, float u, int *token_host, void *cuda_stream);
+
+/*
+ * knnssd_spec_accept: one verification round.  p_dev DEVICE [k+1][vocab]: the full model's filtered distributions of
+ *   the rows [pending, d_0 .. d_{k-1}]; q_dev DEVICE [k][vocab]: the draft model's filtered distributions the drafts
+ *   were drawn from; drafts_host HOST int32 [k]; u_accept_host HOST [k] and u_final uniforms in [0, 1).
+ *   Draft j is kept iff u_accept[j] * q_j(d_j) < p_j(d_j), i.e. with probability min(1, p_j(d_j) / q_j(d_j)); at the
+ *   first rejected j the emitted token is drawn with u_final from max(0, p_j - q_j) (from p_j if that is zero
+ *   everywhere); if all k are kept it is drawn from p_k.  k = 0 draws one token from p_0.
+ *   n_accepted, next_token HOST outputs.  0 <= k <= 15.  Synchronises the stream.
+ */
+knnssd_status knnssd_spec_accept(const float *p_dev, const float *q_dev, const int *drafts_host, int k, int vocab,
+                                 const float *u_accept_host, float u_final, int *n_accepted, int *next_token,
+                                 void *cuda_stream);
+
+/*
  * Cosine top-1 (Sec. 4.2, Eq. (4)) of one query against n anchors of dimension d, all DEVICE fp32; HOST outputs.
  * KNNSSD_ERR_DEGENERATE for a zero / non-finite query or anchor.
  */

@@ -24,7 +24,7 @@ EXPORTS = ["knnssd_init", "knnssd_destroy", "knnssd_prefill", "knnssd_select_ski
            "knnssd_draft", "knnssd_verify", "knnssd_generate", "knnssd_decode", "knnssd_get_launch_count", "knnssd_get_length", "knnssd_set_length",
            "knnssd_set_pending", "knnssd_mask_objective", "knnssd_get_stats", "knnssd_last_error", "knnssd_time_pass", "knnssd_trace_pass", "knnssd_linear",
            "knnssd_gemm_split", "knnssd_linear_tc", "knnssd_build_anchors", "knnssd_cosine_top1", "knnssd_cosine_top1_static",
-           "knnssd_debug_barrier_timeout"]
+           "knnssd_debug_barrier_timeout", "knnssd_filtered_probs", "knnssd_sample_token", "knnssd_spec_accept"]
 
 
 class KnnssdError(RuntimeError):
@@ -84,6 +84,9 @@ def _load():
         "knnssd_cosine_top1": (I, [P, P, I, I, PI, PF, P]),
         "knnssd_cosine_top1_static": (I, [P, P, I, I, PI, PF, P]),
         "knnssd_debug_barrier_timeout": (I, [P, C.c_uint]),
+        "knnssd_filtered_probs": (I, [P, I, I, F, F, P, P]),
+        "knnssd_sample_token": (I, [P, I, F, PI, P]),
+        "knnssd_spec_accept": (I, [P, P, P, I, I, P, F, PI, PI, P]),
     }
     for name, (res, args) in sigs.items():
         fn = getattr(lib, name)
@@ -193,6 +196,46 @@ def knnssd_cosine_top1(query: torch.Tensor, anchors: torch.Tensor):
     if rc:
         raise KnnssdError(rc, "knnssd_cosine_top1")
     return best.value, cs.value
+
+
+def knnssd_filtered_probs(logits: torch.Tensor, temperature: float, top_p: float) -> torch.Tensor:
+    """Temperature + nucleus filtering of logits [rows][vocab] (App. C.1's decoding settings); returns probabilities."""
+    rows, V = logits.shape
+    probs = torch.empty_like(logits)
+    with torch.cuda.device(logits.device):
+        rc = _lib.knnssd_filtered_probs(_dev_ptr(logits, torch.float32), rows, V, float(temperature), float(top_p), _dev_ptr(probs),
+                                        torch.cuda.current_stream().cuda_stream)
+    if rc:
+        raise KnnssdError(rc, "knnssd_filtered_probs")
+    return probs
+
+
+def knnssd_sample_token(weights: torch.Tensor, u: float) -> int:
+    """Inverse-CDF draw in token-id order from non-negative weights [vocab] with the uniform u."""
+    tok = C.c_int()
+    with torch.cuda.device(weights.device):
+        rc = _lib.knnssd_sample_token(_dev_ptr(weights, torch.float32), weights.shape[0], float(u), C.byref(tok),
+                                      torch.cuda.current_stream().cuda_stream)
+    if rc:
+        raise KnnssdError(rc, "knnssd_sample_token")
+    return tok.value
+
+
+def knnssd_spec_accept(p: torch.Tensor, q: Optional[torch.Tensor], drafts, u_accept, u_final: float):
+    """One verification round of speculative sampling: (n_accepted, next_token).  p [k+1][V], q [k][V] filtered."""
+    d = _host_i32(drafts)
+    k = d.shape[0]
+    ua = np.ascontiguousarray(np.asarray(u_accept, dtype=np.float32))
+    if p.dim() != 2 or p.shape[0] != k + 1 or (k > 0 and (q is None or tuple(q.shape) != (k, p.shape[1]))) or ua.shape[0] != k:
+        raise ValueError("p must be [k+1][V], q [k][V], drafts and u_accept [k]")
+    a, nx = C.c_int(), C.c_int()
+    with torch.cuda.device(p.device):
+        rc = _lib.knnssd_spec_accept(_dev_ptr(p, torch.float32), _dev_ptr(q, torch.float32) if k else None,
+                                     d.ctypes.data if k else None, k, p.shape[1], ua.ctypes.data if k else None, float(u_final),
+                                     C.byref(a), C.byref(nx), torch.cuda.current_stream().cuda_stream)
+    if rc:
+        raise KnnssdError(rc, "knnssd_spec_accept")
+    return a.value, nx.value
 
 
 STATIC_MAX_ANCHORS = 4096

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libknnssd.so")
 SOURCES = ["knnssd.cu"]
-HEADERS = ["kernels.cuh", "linear_stream.cuh", "linear_presplit.cuh", "pass_kernel.cuh", "prefill.cuh", "prefill_host.cuh", "anchors.cuh", "linear_tc.cuh", os.path.join("..", "..", "include", "knnssd.h")]
+HEADERS = ["kernels.cuh", "linear_stream.cuh", "linear_presplit.cuh", "pass_kernel.cuh", "prefill.cuh", "prefill_host.cuh", "anchors.cuh", "linear_tc.cuh", "sampling.cuh", os.path.join("..", "..", "include", "knnssd.h")]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "-shared", "--use_fast_math=false"]
 

@@ -8,6 +8,7 @@
 #include "prefill_host.cuh"
 #include "anchors.cuh"
 #include "linear_tc.cuh"
+#include "sampling.cuh"
 
 #include <cmath>
 #include <cstdio>
@@ -1414,6 +1415,64 @@ knnssd_status knnssd_build_anchors(const float *x_dev, int n_points, int d, int 
     if (e != cudaSuccess) { cudaGetLastError(); return KNNSSD_ERR_CUDA; }
     if (rounds_host) *rounds_host = rounds;
     if (ms_rounds_host) *ms_rounds_host = ms_total;
+    return KNNSSD_OK;
+}
+
+knnssd_status knnssd_filtered_probs(const float *logits_dev, int rows, int vocab, float temperature, float top_p,
+                                    float *probs_dev, void *cuda_stream) {
+    if (!logits_dev || !probs_dev || rows < 1 || vocab < 1 || !(temperature > 0.f) || !(top_p > 0.f) || !std::isfinite(temperature) ||
+        !std::isfinite(top_p))
+        return KNNSSD_ERR_INVALID_ARG;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+    sampling::filtered_probs_kernel<<<rows, sampling::NT, 0, s>>>(logits_dev, vocab, 1.0f / temperature, top_p, probs_dev);
+    return cudaGetLastError() == cudaSuccess ? KNNSSD_OK : KNNSSD_ERR_CUDA;
+}
+
+knnssd_status knnssd_sample_token(const float *weights_dev, int vocab, float u, int *token_host, void *cuda_stream) {
+    if (!weights_dev || !token_host || vocab < 1 || !(u >= 0.f) || !(u < 1.f)) return KNNSSD_ERR_INVALID_ARG;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+    int *tok = nullptr;
+    if (cudaMalloc(reinterpret_cast<void **>(&tok), sizeof(int)) != cudaSuccess) { cudaGetLastError(); return KNNSSD_ERR_CUDA; }
+    sampling::sample_kernel<<<1, sampling::NT, 0, s>>>(weights_dev, vocab, u, tok);
+    cudaError_t e = cudaMemcpyAsync(token_host, tok, sizeof(int), cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e == cudaSuccess) e = cudaGetLastError();
+    cudaFree(tok);
+    return e == cudaSuccess ? KNNSSD_OK : KNNSSD_ERR_CUDA;
+}
+
+knnssd_status knnssd_spec_accept(const float *p_dev, const float *q_dev, const int *drafts_host, int k, int vocab,
+                                 const float *u_accept_host, float u_final, int *n_accepted, int *next_token, void *cuda_stream) {
+    if (!p_dev || !n_accepted || !next_token || k < 0 || k > kMaxRows - 1 || vocab < 1 || !(u_final >= 0.f) || !(u_final < 1.f) ||
+        (k > 0 && (!q_dev || !drafts_host || !u_accept_host)))
+        return KNNSSD_ERR_INVALID_ARG;
+    for (int j = 0; j < k; ++j)
+        if (drafts_host[j] < 0 || drafts_host[j] >= vocab || !(u_accept_host[j] >= 0.f) || !(u_accept_host[j] < 1.f))
+            return KNNSSD_ERR_INVALID_ARG;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+    int *buf = nullptr;                       // [0..1] result, [2 .. 2 + k) drafts, then k floats of uniforms
+    if (cudaMalloc(reinterpret_cast<void **>(&buf), sizeof(int) * (2 + 2 * (size_t)kMaxRows)) != cudaSuccess) {
+        cudaGetLastError();
+        return KNNSSD_ERR_CUDA;
+    }
+    int *d_dev = buf + 2;
+    float *u_dev = reinterpret_cast<float *>(buf + 2 + kMaxRows);
+    cudaError_t e = cudaSuccess;
+    if (k > 0) {
+        e = cudaMemcpyAsync(d_dev, drafts_host, sizeof(int) * k, cudaMemcpyHostToDevice, s);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(u_dev, u_accept_host, sizeof(float) * k, cudaMemcpyHostToDevice, s);
+    }
+    int host[2] = {0, 0};
+    if (e == cudaSuccess) {
+        sampling::spec_accept_kernel<<<1, sampling::NT, 0, s>>>(p_dev, q_dev, d_dev, k, vocab, u_dev, u_final, buf);
+        e = cudaMemcpyAsync(host, buf, sizeof(int) * 2, cudaMemcpyDeviceToHost, s);
+    }
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e == cudaSuccess) e = cudaGetLastError();
+    cudaFree(buf);
+    if (e != cudaSuccess) return KNNSSD_ERR_CUDA;
+    *n_accepted = host[0];
+    *next_token = host[1];
     return KNNSSD_OK;
 }
 
