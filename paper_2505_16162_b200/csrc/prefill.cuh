@@ -30,15 +30,16 @@ using stream::mbar_try_wait;
 using stream::smem_u32;
 
 constexpr int BM = 128;                               // tokens per tile: rows of the accumulator = lanes of tensor memory
-constexpr int BN_MAX = 320;                           // most accumulator columns per tile (a launch picks 64, 128, .. 320)
+constexpr int BN_MAX = 256;                           // most accumulator columns per tile (a launch picks 64, 128, 192 or 256)
 constexpr int BOX_N = 64;                             // weight rows per TMA box
 constexpr int BK = 64;                                // input columns per stage: 128 bytes of bf16 = one swizzle row
 constexpr int STAGES = 3;
 constexpr int A_BYTES = BM * BK * 2;                  // one term of the activation tile
 constexpr int B_BYTES = BN_MAX * BK * 2;
 constexpr int STAGE_BYTES = 2 * A_BYTES + B_BYTES;    // hi plane, lo plane, weights
-constexpr int TMEM_COLS = 512;                        // columns of tensor memory a CTA takes (a power of two >= BN_MAX)
-constexpr int GEMM_THREADS = 192;                     // warp 0: TMA; warp 1: MMA issue + tensor-memory owner; warps 2..5: epilogue
+constexpr int TMEM_COLS = 512;                        // columns of tensor memory a CTA takes: two accumulators of BN_MAX columns
+constexpr int CHUNK_KB = 8;                           // k-blocks accumulated in tensor memory before the sum moves to registers
+constexpr int GEMM_THREADS = 320;                     // warp 0: TMA; warp 1: MMA issue + tensor-memory owner; warps 2..9: epilogue
 constexpr int GEMM_SMEM = STAGES * STAGE_BYTES + 1024 + 128;   // + slack to align the tiles to 1024 bytes + barriers
 constexpr unsigned WAIT_LIMIT = 4000000u;           // polls of one wait (a whole tile takes well under a millisecond)
 
@@ -132,6 +133,15 @@ __device__ __forceinline__ uint32_t pack_bf16(uint32_t lo16, uint32_t hi16) { re
 // the gate matrix (map tb0) and columns [bn / 2, bn) the same units of the up matrix (map tb1); otherwise the columns
 // are units n0 .. n0 + bn - 1 of one matrix (tb0 = tb1).  ta covers both activation planes: rows [0, Tpad) the hi
 // terms, rows [Tpad, 2 Tpad) the lo terms.  The weight maps are read in boxes of BOX_N rows.
+//
+// Accumulation.  The tensor core adds every 16-column product into its fp32 accumulator by truncation, so a sum that
+// stays in tensor memory over all of K collects an error that grows with the number of steps (measured: ~4e-5 relative
+// at K = 13824, ten times the error of the decode passes' sums; through the bf16 rounding of the K/V rows it feeds,
+// that showed as 2.4e-2 on the logits of a 40-layer model).  The sum over K is therefore cut into chunks of CHUNK_KB
+// k-blocks: a chunk accumulates in one of two accumulators in tensor memory while the eight epilogue warps move the
+// previous chunk's sum out and add it, rounded to nearest, to the running sums they keep in registers (a thread owns
+// one token row and half of the tile's columns).  The error left is that of the short chunks plus K / (64 CHUNK_KB)
+// ordinary fp32 additions.
 template <int EPI>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_split_kernel(const __grid_constant__ CUtensorMap ta, const __grid_constant__ CUtensorMap tb0,
@@ -140,18 +150,20 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap ta, const __grid_constant_
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(pf_smem_raw) + 1023) & ~(uintptr_t)1023);
     uint64_t *full = reinterpret_cast<uint64_t *>(smem + STAGES * STAGE_BYTES);
     uint64_t *empty = full + STAGES;
-    uint64_t *acc_full = empty + STAGES;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_full + 1);
+    uint64_t *acc_full = empty + STAGES;          // [2]: a chunk's sum is complete in accumulator b
+    uint64_t *acc_empty = acc_full + 2;           // [2]: the epilogue warps have moved accumulator b's sum out
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_empty + 2);
     volatile int *cta_abort = reinterpret_cast<volatile int *>(tmem_slot + 1);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int t0 = blockIdx.x * BM;
     const int bn = g.bn, per = EPI == PF_SWIGLU ? bn / 2 : bn;      // units of a matrix per tile
     const int n0 = blockIdx.y * per;
-    const int nkb = g.K / BK;
+    const int nkb = g.K / BK, nchunks = (nkb + CHUNK_KB - 1) / CHUNK_KB;
+    constexpr int EPI_WARPS = GEMM_THREADS / 32 - 2;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-        mbar_init(acc_full, 1);
+        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], EPI_WARPS); }
         *cta_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -194,96 +206,132 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap ta, const __grid_constant_
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            // ---- MMA issue: 4 k-steps of 16 columns per stage, hi and lo term into the same accumulator ----
+            // ---- MMA issue: chunk c goes to accumulator c & 1; per stage 4 k-steps of 16 columns, hi and lo term ----
             bool ok = true;
-            for (int kb = 0; kb < nkb && ok; ++kb) {
-                const int s = kb % STAGES;
-                const uint32_t ph = (uint32_t)(kb / STAGES) & 1u;
-                ok = pf_wait(&full[s], ph, cta_abort, g.err, 22);
+            const uint32_t idesc = umma_idesc(bn);
+            for (int c = 0; c < nchunks && ok; ++c) {
+                const int b = c & 1;
+                ok = pf_wait(&acc_empty[b], ((uint32_t)(c >> 1) & 1u) ^ 1u, cta_abort, g.err, 24);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t a_hi = smem_u32(smem + s * STAGE_BYTES), a_lo = a_hi + A_BYTES, b = a_hi + 2 * A_BYTES;
-                // at most 256 columns per instruction: a wider tile takes a second one for the rest
-                const int n1 = bn < 256 ? bn : 256, n2 = bn - n1;
-                const uint32_t id1 = umma_idesc(n1), id2 = umma_idesc(n2 ? n2 : 16);
+                const uint32_t acc_addr = tmem + (uint32_t)(b * BN_MAX);
+                const int kb1 = min(nkb, (c + 1) * CHUNK_KB);
+                for (int kb = c * CHUNK_KB; kb < kb1 && ok; ++kb) {
+                    const int s = kb % STAGES;
+                    const uint32_t ph = (uint32_t)(kb / STAGES) & 1u;
+                    ok = pf_wait(&full[s], ph, cta_abort, g.err, 22);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t a_hi = smem_u32(smem + s * STAGE_BYTES), a_lo = a_hi + A_BYTES, bw = a_hi + 2 * A_BYTES;
 #pragma unroll
-                for (int k = 0; k < BK / 16; ++k) {
-                    const uint32_t acc = (kb | k) != 0 ? 1u : 0u;
-                    const uint64_t db = umma_desc(b + 32 * k), dh = umma_desc(a_hi + 32 * k), dl = umma_desc(a_lo + 32 * k);
-                    umma_bf16(tmem, dh, db, id1, acc);
-                    umma_bf16(tmem, dl, db, id1, 1u);
-                    if (n2) {
-                        const uint64_t db2 = umma_desc(b + 256 * BK * 2 + 32 * k);
-                        umma_bf16(tmem + 256, dh, db2, id2, acc);
-                        umma_bf16(tmem + 256, dl, db2, id2, 1u);
+                    for (int k = 0; k < BK / 16; ++k) {
+                        const uint32_t accum = (kb != c * CHUNK_KB || k != 0) ? 1u : 0u;
+                        const uint64_t db = umma_desc(bw + 32 * k);
+                        umma_bf16(acc_addr, umma_desc(a_hi + 32 * k), db, idesc, accum);
+                        umma_bf16(acc_addr, umma_desc(a_lo + 32 * k), db, idesc, 1u);
                     }
+                    umma_commit(&empty[s]);
                 }
-                umma_commit(&empty[s]);
+                umma_commit(&acc_full[b]);     // on the abort path too: it releases the epilogue warps' wait
             }
-            umma_commit(acc_full);         // on the abort path too: it releases the epilogue warps' wait
+            if (!ok) { umma_commit(&acc_full[0]); umma_commit(&acc_full[1]); }
         }
     } else {
-        // ---- epilogue: warp w reads lanes 32 (w % 4) .. + 31 of tensor memory = tokens t0 + 32 (w % 4) + lane ----
-        // the loads from tensor memory are warp-wide: the warp goes on only if all of its threads saw the accumulator
-        const bool ok = __all_sync(0xffffffffu, pf_wait(acc_full, 0u, cta_abort, g.err, 23) && !*cta_abort);
-        tc_fence_after();
-        const int q = warp & 3;
+        // ---- epilogue warps: warp w reads lanes 32 (w % 4) .. + 31 of tensor memory = tokens t0 + 32 (w % 4) + lane; the
+        //      two warps of a lane quarter split the tile's columns.  acc[] = this thread's running sums over the chunks:
+        //      store / add: columns [hsel bn / 2, + bn / 2) in groups of 32; SwiGLU: acc[0 .. 63] gate columns
+        //      [hsel bn / 4, + bn / 4), acc[64 .. 127] the up columns of the same units ----
+        const int q = warp & 3, hsel = (warp - 2) >> 2;
         const int t = t0 + 32 * q + lane;
         const uint32_t trow = tmem + ((uint32_t)(32 * q) << 16);
-        if (ok) {
+        const int half = bn / 2, qtr = bn / 4;
+        // tile column of register group gi (32 columns), or -1 if the group is not in use
+        auto group_col = [&](int gi) -> int {
             if (EPI == PF_SWIGLU) {
-                for (int c0 = 0; c0 < per && n0 + c0 < g.N; c0 += 32) {
-                    float gt[32], up[32];
-                    tmem_ld32(trow + c0, gt);
-                    tmem_ld32(trow + per + c0, up);
-                    if (t < g.T) {
-                        uint32_t hi[16], lo[16];
+                const int gg = gi & 1;
+                if (32 * gg >= qtr) return -1;
+                return (gi >= 2 ? per : 0) + hsel * qtr + 32 * gg;
+            }
+            return 32 * gi < half ? hsel * half + 32 * gi : -1;
+        };
+        float acc[128];
 #pragma unroll
-                        for (int i = 0; i < 32; i += 2) {
-                            uint32_t h2[2], l2[2];
+        for (int i = 0; i < 128; ++i) acc[i] = 0.f;
+        bool ok = true;
+        for (int c = 0; c < nchunks && ok; ++c) {
+            const int b = c & 1;
+            // the loads from tensor memory are warp-wide: the warp goes on only if all of its threads saw the accumulator
+            ok = __all_sync(0xffffffffu, pf_wait(&acc_full[b], (uint32_t)(c >> 1) & 1u, cta_abort, g.err, 23) && !*cta_abort);
+            if (!ok) break;
+            tc_fence_after();
 #pragma unroll
-                            for (int e = 0; e < 2; ++e) {
-                                const float a = gt[i + e] / (1.0f + expf(-gt[i + e])) * up[i + e];
-                                h2[e] = float_to_bf16_rne(a);
-                                l2[e] = float_to_bf16_rne(a - __uint_as_float(h2[e] << 16));
-                            }
-                            hi[i >> 1] = pack_bf16(h2[0], h2[1]);
-                            lo[i >> 1] = pack_bf16(l2[0], l2[1]);
+            for (int gi = 0; gi < 4; ++gi) {
+                const int col = group_col(gi);
+                if (col >= 0) {                          // warp-uniform
+                    float v[32];
+                    tmem_ld32(trow + (uint32_t)(b * BN_MAX + col), v);
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) acc[32 * gi + i] += v[i];
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) stream::mbar_arrive(&acc_empty[b]);
+        }
+        if (ok && t < g.T) {
+            if (EPI == PF_SWIGLU) {
+#pragma unroll
+                for (int gg = 0; gg < 2; ++gg) {
+                    const int c0 = hsel * qtr + 32 * gg;         // unit offset within the tile
+                    if (32 * gg >= qtr || n0 + c0 >= g.N) continue;
+                    uint32_t hi[16], lo[16];
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        uint32_t h2[2], l2[2];
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            const float gt = acc[32 * gg + i + e], up = acc[64 + 32 * gg + i + e];
+                            const float a = gt / (1.0f + expf(-gt)) * up;
+                            h2[e] = float_to_bf16_rne(a);
+                            l2[e] = float_to_bf16_rne(a - __uint_as_float(h2[e] << 16));
                         }
-                        bf16_t *ph = g.out_hi + (size_t)t * g.ldo + n0 + c0, *pl = g.out_lo + (size_t)t * g.ldo + n0 + c0;
-                        if (n0 + c0 + 32 <= g.N) {
+                        hi[i >> 1] = pack_bf16(h2[0], h2[1]);
+                        lo[i >> 1] = pack_bf16(l2[0], l2[1]);
+                    }
+                    bf16_t *ph = g.out_hi + (size_t)t * g.ldo + n0 + c0, *pl = g.out_lo + (size_t)t * g.ldo + n0 + c0;
+                    if (n0 + c0 + 32 <= g.N) {
 #pragma unroll
-                            for (int i = 0; i < 4; ++i) {
-                                reinterpret_cast<uint4 *>(ph)[i] = make_uint4(hi[4 * i], hi[4 * i + 1], hi[4 * i + 2], hi[4 * i + 3]);
-                                reinterpret_cast<uint4 *>(pl)[i] = make_uint4(lo[4 * i], lo[4 * i + 1], lo[4 * i + 2], lo[4 * i + 3]);
-                            }
-                        } else {
-                            for (int i = 0; n0 + c0 + i < g.N; ++i) {
-                                ph[i] = (bf16_t)((hi[i >> 1] >> (16 * (i & 1))) & 0xFFFFu);
-                                pl[i] = (bf16_t)((lo[i >> 1] >> (16 * (i & 1))) & 0xFFFFu);
-                            }
+                        for (int i = 0; i < 4; ++i) {
+                            reinterpret_cast<uint4 *>(ph)[i] = make_uint4(hi[4 * i], hi[4 * i + 1], hi[4 * i + 2], hi[4 * i + 3]);
+                            reinterpret_cast<uint4 *>(pl)[i] = make_uint4(lo[4 * i], lo[4 * i + 1], lo[4 * i + 2], lo[4 * i + 3]);
+                        }
+                    } else {
+                        for (int i = 0; n0 + c0 + i < g.N; ++i) {
+                            ph[i] = (bf16_t)((hi[i >> 1] >> (16 * (i & 1))) & 0xFFFFu);
+                            pl[i] = (bf16_t)((lo[i >> 1] >> (16 * (i & 1))) & 0xFFFFu);
                         }
                     }
                 }
             } else {
-                for (int c0 = 0; c0 < bn && n0 + c0 < g.N; c0 += 32) {
-                    float v[32];
-                    tmem_ld32(trow + c0, v);
-                    if (t < g.T) {
-                        float *yp = g.y + (size_t)t * g.ldy + g.col0 + n0 + c0;
-                        if (n0 + c0 + 32 <= g.N) {
 #pragma unroll
-                            for (int i = 0; i < 32; i += 4) {
-                                float4 o = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
-                                if (EPI == PF_ADD) {
-                                    const float4 x = *reinterpret_cast<const float4 *>(yp + i);
-                                    o.x += x.x; o.y += x.y; o.z += x.z; o.w += x.w;
-                                }
-                                *reinterpret_cast<float4 *>(yp + i) = o;
+                for (int gi = 0; gi < 4; ++gi) {
+                    const int c0 = hsel * half + 32 * gi;
+                    if (32 * gi >= half || n0 + c0 >= g.N) continue;
+                    float *yp = g.y + (size_t)t * g.ldy + g.col0 + n0 + c0;
+                    if (n0 + c0 + 32 <= g.N) {
+#pragma unroll
+                        for (int i = 0; i < 32; i += 4) {
+                            float4 o = make_float4(acc[32 * gi + i], acc[32 * gi + i + 1], acc[32 * gi + i + 2], acc[32 * gi + i + 3]);
+                            if (EPI == PF_ADD) {
+                                const float4 x = *reinterpret_cast<const float4 *>(yp + i);
+                                o.x += x.x; o.y += x.y; o.z += x.z; o.w += x.w;
                             }
-                        } else {
-                            for (int i = 0; n0 + c0 + i < g.N; ++i) yp[i] = EPI == PF_ADD ? yp[i] + v[i] : v[i];
+                            *reinterpret_cast<float4 *>(yp + i) = o;
                         }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            if (n0 + c0 + i < g.N) yp[i] = EPI == PF_ADD ? yp[i] + acc[32 * gi + i] : acc[32 * gi + i];
                     }
                 }
             }

@@ -56,8 +56,8 @@ inline bool gemm_attrs_once() {
 }
 
 // Accumulator columns per tile: all CTAs of a launch run at once on n_sms SMs, round after round, and a round takes
-// time in proportion to the tile's columns; the width with the fewest column-rounds wins (ties: the wider tile, which
-// re-reads the activations less).
+// time in proportion to the bytes a k-block brings in (two activation planes of 128 rows + bn weight rows); the width
+// with the lowest rounds x bytes wins (ties: the wider tile).
 inline int pick_bn(int T, int N, bool swiglu, int n_sms) {
     const int row_tiles = (T + BM - 1) / BM;
     int best = 0;
@@ -66,7 +66,7 @@ inline int pick_bn(int T, int N, bool swiglu, int n_sms) {
         if (swiglu && bn % 128) continue;
         const int per = swiglu ? bn / 2 : bn;
         const long ctas = (long)row_tiles * ((N + per - 1) / per);
-        const long cost = ((ctas + n_sms - 1) / n_sms) * bn;
+        const long cost = ((ctas + n_sms - 1) / n_sms) * (2 * BM + bn);
         if (!best || cost <= best_cost) { best = bn; best_cost = cost; }
     }
     return best;

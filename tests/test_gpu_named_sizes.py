@@ -55,6 +55,49 @@ def _masks(rec, shape):
     return np.stack([si.skip_mask_split(seed + 100 + i, shape.n_layers, skip[0], skip[1]) for i in range(rec["n_domains"])])
 
 
+def _decode_following_the_oracle(sess, P, want_tokens, want_accepts, r, k, max_new):
+    """Decodes max_new tokens and compares them with the oracle's.  Both sides' logits carry an error of up to TOL, so
+    where the full model's two best logits are closer than 2 TOL the arg-max is not unique: at a first differing token
+    the oracle's choice must be within 2 TOL of this side's best logit at that step (checked on the logits of a
+    teacher-forced one-row pass), after which decoding continues from the oracle's token, so that every later token is
+    still compared.  Returns the substitutions made: [(token index, logit gap)].  Accept counts are compared for the
+    rounds before the first substitution (afterwards the rounds no longer line up)."""
+    subs, start = [], 0
+    first_run = True
+    while start < max_new:
+        got = sess.decode(max_new - start, k)
+        seg = want_tokens[start:]
+        bad = np.nonzero(got["tokens"] != seg)[0]
+        if first_run:
+            n_ok_rounds = len(want_accepts)
+            if bad.size:                        # rounds that emitted only tokens before the first difference
+                emitted, n_ok_rounds = 1, 0
+                for a in want_accepts:
+                    if emitted + a + 1 > bad[0]:
+                        break
+                    emitted += a + 1
+                    n_ok_rounds += 1
+            assert np.array_equal(got["accepts"][:n_ok_rounds], want_accepts[:n_ok_rounds])
+            if not bad.size:
+                st = got["stats"]
+                assert (st["rounds"], st["drafted"], st["accepted"]) == (r["rounds"], r["drafted"], r["accepted"])
+            first_run = False
+        if not bad.size:
+            break
+        i = start + int(bad[0])                 # token i differs; tokens before it agree, so their K/V rows are valid
+        assert i >= 1
+        sess.set_length(P + i - 1)
+        sess.set_pending(int(want_tokens[i - 1]))
+        g = sess.verify([], want_logits=True)   # the full model's logits for token i, given the oracle's prefix
+        lg = g["logits"][0]
+        gap = float(lg.max() - lg[int(want_tokens[i])])
+        assert gap < 2 * TOL, f"token {i}: the oracle's token is {gap} below this side's best logit - not a near-tie"
+        subs.append((i, gap))
+        sess.set_pending(int(want_tokens[i]))   # follow the oracle
+        start = i
+    return subs
+
+
 def test_golden_files_are_present():
     assert FILES, "no tests/golden/tokens_*.json"
 
@@ -80,6 +123,7 @@ def test_workload_matches_the_oracles_stored_output(kb, path):
     sess = kb.Session.from_shape(shape, w, max_seq, max_draft=max(k, 8), anchors=anchors, skip_masks=masks,
                                  anchors_per_domain=per)
     worst_logit, worst_pooled = 0.0, 0.0
+    near_ties = []
     for r in rec["requests"]:
         P = r["prompt_len"]
         if stream:
@@ -104,13 +148,9 @@ def test_workload_matches_the_oracles_stored_output(kb, path):
         assert abs(cos - r["cosine"]) < 1e-4
         if "explicit_mask_domain" in rec:
             sess.set_skipmask(masks[rec["explicit_mask_domain"]])
-        got = sess.decode(max_new, k)
         want_tokens, want_accepts = np.array(r["tokens"], np.int32), np.array(r["accepts"], np.int32)
-        bad = np.nonzero(got["tokens"] != want_tokens)[0]
-        assert bad.size == 0, f"first differing token at {bad[0]}; oracle's smallest decisive margin {r['min_margin']}"
-        assert np.array_equal(got["accepts"], want_accepts)
-        st = got["stats"]
-        assert (st["rounds"], st["drafted"], st["accepted"]) == (r["rounds"], r["drafted"], r["accepted"])
+        subs = _decode_following_the_oracle(sess, P, want_tokens, want_accepts, r, k, max_new)
+        near_ties.extend(subs)
         # one teacher-forced verification pass at the prompt's end: sampled logits of every row
         sess.set_length(P)
         sess.set_pending(first)
@@ -125,5 +165,8 @@ def test_workload_matches_the_oracles_stored_output(kb, path):
             n_acc += 1
         assert (g["n_accepted"], g["next_token"]) == (n_acc, r["verify_argmax"][n_acc])
     sess.close()
-    print(f"\n[{rec['case']}] max |logit - oracle| on sampled entries {worst_logit:.3e}, pooled {worst_pooled:.3e}, "
+    n_tok = sum(len(r["tokens"]) for r in rec["requests"])
+    print(f"\n[{rec['case']}] {n_tok} tokens, {len(near_ties)} near-tie substitution(s) {[(i, round(g, 5)) for i, g in near_ties]}; "
+          f"max |logit - oracle| on sampled entries {worst_logit:.3e}, pooled {worst_pooled:.3e}, "
           f"oracle min margin {min(r['min_margin'] for r in rec['requests']):.3e}")
+    assert len(near_ties) <= max(3, n_tok // 16)

@@ -29,10 +29,12 @@ def _oracle_linear(W, x):
 
 
 def _tol(n_in, want):
-    """Two bf16 terms carry 16 mantissa bits of x (2e-5 of the largest output covers that, as for the decode kernel);
-    the tensor core adds each 16-column product to its fp32 accumulator with truncation, one ulp of the running sum
-    at most per step: n_in / 16 steps of 2^-23 relative."""
-    return (2e-5 + n_in / 16 * 2.0 ** -23) * max(1.0, float(np.abs(want).max()))
+    """Two bf16 terms carry 16 mantissa bits of x (2e-5 of the largest output covers that, as for the decode kernel).
+    The tensor core adds each 16-column product to its fp32 accumulator with truncation, one ulp of the running sum
+    at most per step; a sum stays in tensor memory for a chunk of 512 columns only (64 steps of 2^-23 relative) and the
+    chunks are added in registers with ordinary rounding (n_in / 512 steps of 2^-24).  An observed bound of this
+    kernel's arithmetic, not one the method fixes; the whole-path tolerance on logits stays 2e-2."""
+    return (2e-5 + 64 * 2.0 ** -23 + n_in / 512 * 2.0 ** -24) * max(1.0, float(np.abs(want).max()))
 
 
 def _inputs(n_out, n_in, T, seed=3):
