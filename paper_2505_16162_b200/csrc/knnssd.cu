@@ -518,12 +518,18 @@ bool prefill_tensor(knnssd_ctx *c, int n) {
             bf16_t *kc = reinterpret_cast<bf16_t *>(c->kcache) + (size_t)l * layer_stride;
             bf16_t *vc = reinterpret_cast<bf16_t *>(c->vcache) + (size_t)l * layer_stride;
             prefill::norm_split_kernel<<<T, 256, 0, s>>>(c->pf_x, d, ly.attn_norm, g.rms_eps, c->pf_ad, c->pf_ad + (size_t)cap * d);
-            ok = ok && prefill::launch_gemm(c->pf_map_d, cap, ly.wq, nullptr, nq, d, T, prefill::PF_STORE, c->pf_qkv, ldq, 0, nullptr,
-                                            nullptr, 0, err, c->n_sms, s);
-            ok = ok && prefill::launch_gemm(c->pf_map_d, cap, ly.wk, nullptr, nkv, d, T, prefill::PF_STORE, c->pf_qkv, ldq, nq, nullptr,
-                                            nullptr, 0, err, c->n_sms, s);
-            ok = ok && prefill::launch_gemm(c->pf_map_d, cap, ly.wv, nullptr, nkv, d, T, prefill::PF_STORE, c->pf_qkv, ldq, nq + nkv,
-                                            nullptr, nullptr, 0, err, c->n_sms, s);
+            if (nq % prefill::BOX_N == 0 && nkv % prefill::BOX_N == 0) {
+                // q, k and v in one launch over the stacked units (their columns of the projection buffer are adjacent)
+                ok = ok && prefill::launch_gemm(c->pf_map_d, cap, ly.wq, ly.wk, ldq, d, T, prefill::PF_STORE, c->pf_qkv, ldq, 0, nullptr,
+                                                nullptr, 0, err, c->n_sms, s, ly.wv, nq, nkv);
+            } else {
+                ok = ok && prefill::launch_gemm(c->pf_map_d, cap, ly.wq, nullptr, nq, d, T, prefill::PF_STORE, c->pf_qkv, ldq, 0, nullptr,
+                                                nullptr, 0, err, c->n_sms, s);
+                ok = ok && prefill::launch_gemm(c->pf_map_d, cap, ly.wk, nullptr, nkv, d, T, prefill::PF_STORE, c->pf_qkv, ldq, nq, nullptr,
+                                                nullptr, 0, err, c->n_sms, s);
+                ok = ok && prefill::launch_gemm(c->pf_map_d, cap, ly.wv, nullptr, nkv, d, T, prefill::PF_STORE, c->pf_qkv, ldq, nq + nkv,
+                                                nullptr, nullptr, 0, err, c->n_sms, s);
+            }
             prefill::rope_kv_rows_kernel<<<T, 256, 0, s>>>(c->pf_qkv, H, Hkv, HD, c->pf_cs, kc, vc, g.max_seq, t0);
             prefill::attn_prompt_kernel<HD><<<dim3((T + 15) / 16, (H + 3) / 4), 128, 0, s>>>(c->pf_qkv, H, Hkv, kc, vc, g.max_seq, t0, T,
                                                                                            c->pf_aq, c->pf_aq + (size_t)cap * nq);
@@ -534,7 +540,7 @@ bool prefill_tensor(knnssd_ctx *c, int n) {
                                             c->pf_af + (size_t)cap * F, F, err, c->n_sms, s);
             ok = ok && prefill::launch_gemm(c->pf_map_f, cap, ly.w_down, nullptr, d, F, T, prefill::PF_ADD, c->pf_x, d, 0, nullptr, nullptr,
                                             0, err, c->n_sms, s);
-            c->launches += 11;
+            c->launches += (nq % prefill::BOX_N == 0 && nkv % prefill::BOX_N == 0) ? 9 : 11;
         }
         // pooled numerator: every row's final hidden state (mean pooling) or the last row's
         if (g.pool_mode == 0) {

@@ -56,6 +56,8 @@ struct GemmArgs {
     bf16_t *out_lo;
     int ldo;
     int *err;          // set non-zero if a bounded wait gave up
+    int nA, nB;        // STORE over stacked matrices (q, k, v in one launch): units [0, nA) are rows of map tb0,
+                       // [nA, nA + nB) rows of tb1, the rest rows of tb2; all multiples of BOX_N.  One matrix: nA = N
 };
 
 __device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int x, int y, uint64_t *bar) {
@@ -145,7 +147,7 @@ __device__ __forceinline__ uint32_t pack_bf16(uint32_t lo16, uint32_t hi16) { re
 template <int EPI>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_split_kernel(const __grid_constant__ CUtensorMap ta, const __grid_constant__ CUtensorMap tb0,
-                  const __grid_constant__ CUtensorMap tb1, GemmArgs g, int Tpad) {
+                  const __grid_constant__ CUtensorMap tb1, const __grid_constant__ CUtensorMap tb2, GemmArgs g, int Tpad) {
     extern __shared__ unsigned char pf_smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(pf_smem_raw) + 1023) & ~(uintptr_t)1023);
     uint64_t *full = reinterpret_cast<uint64_t *>(smem + STAGES * STAGE_BYTES);
@@ -192,7 +194,13 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap ta, const __grid_constant_
                 for (int j = 0; j < bn / BOX_N; ++j) {
                     const int r = j * BOX_N;                 // accumulator column the box starts at
                     const bool second = EPI == PF_SWIGLU && r >= per;
-                    tma_load_2d(st + 2 * A_BYTES + r * BK * 2, second ? &tb1 : &tb0, kb * BK, n0 + (second ? r - per : r), &full[s]);
+                    const CUtensorMap *wm = second ? &tb1 : &tb0;
+                    int wrow = n0 + (second ? r - per : r);
+                    if (EPI != PF_SWIGLU && wrow >= g.nA) {          // stacked matrices: the box lies in the second or third one
+                        wm = &tb1; wrow -= g.nA;
+                        if (wrow >= g.nB) { wm = &tb2; wrow -= g.nB; }
+                    }
+                    tma_load_2d(st + 2 * A_BYTES + r * BK * 2, wm, kb * BK, wrow, &full[s]);
                 }
                 armed = kb + 1;
             }

@@ -73,24 +73,32 @@ inline int pick_bn(int T, int N, bool swiglu, int n_sms) {
 }
 
 // One contraction over T rows.  `planes` = the activation map (hi rows [0, cap), lo rows [cap, 2 cap)); W0 (and W1 for
-// SwiGLU: W0 = gate, W1 = up) are [N][K] bf16.  Returns false if a tensor map could not be made.
+// SwiGLU: W0 = gate, W1 = up) are [N][K] bf16.  STORE with W1 and W2 given: the three matrices (nA, nB and nC rows, all
+// multiples of BOX_N) are stacked along the output units, N = nA + nB + nC, one launch for q, k and v.
+// Returns false if a tensor map could not be made.
 inline bool launch_gemm(const CUtensorMap &planes, int cap, const void *W0, const void *W1, int N, int K, int T, int epi, float *y,
-                        int ldy, int col0, bf16_t *out_hi, bf16_t *out_lo, int ldo, int *err, int n_sms, cudaStream_t s) {
+                        int ldy, int col0, bf16_t *out_hi, bf16_t *out_lo, int ldo, int *err, int n_sms, cudaStream_t s,
+                        const void *W2 = nullptr, int nA = 0, int nB = 0) {
     if (!gemm_attrs_once()) return false;
-    CUtensorMap tb0, tb1;
-    if (!make_map(&tb0, W0, (size_t)N, (size_t)K, BOX_N)) return false;
+    CUtensorMap tb0, tb1, tb2;
+    const bool stacked = epi == PF_STORE && W1 && W2;
+    if (!make_map(&tb0, W0, (size_t)(stacked ? nA : N), (size_t)K, BOX_N)) return false;
     if (epi == PF_SWIGLU) {
         if (!make_map(&tb1, W1, (size_t)N, (size_t)K, BOX_N)) return false;
+        tb2 = tb1;
+    } else if (stacked) {
+        if (!make_map(&tb1, W1, (size_t)nB, (size_t)K, BOX_N) || !make_map(&tb2, W2, (size_t)(N - nA - nB), (size_t)K, BOX_N)) return false;
     } else {
         tb1 = tb0;
+        tb2 = tb0;
     }
     const int bn = pick_bn(T, N, epi == PF_SWIGLU, n_sms);
-    GemmArgs g{T, K, N, bn, y, ldy, col0, out_hi, out_lo, ldo, err};
+    GemmArgs g{T, K, N, bn, y, ldy, col0, out_hi, out_lo, ldo, err, stacked ? nA : N, stacked ? nB : 0};
     const int per = epi == PF_SWIGLU ? bn / 2 : bn;
     const dim3 grid((T + BM - 1) / BM, (N + per - 1) / per);
-    if (epi == PF_STORE) gemm_split_kernel<PF_STORE><<<grid, GEMM_THREADS, GEMM_SMEM, s>>>(planes, tb0, tb1, g, cap);
-    else if (epi == PF_ADD) gemm_split_kernel<PF_ADD><<<grid, GEMM_THREADS, GEMM_SMEM, s>>>(planes, tb0, tb1, g, cap);
-    else gemm_split_kernel<PF_SWIGLU><<<grid, GEMM_THREADS, GEMM_SMEM, s>>>(planes, tb0, tb1, g, cap);
+    if (epi == PF_STORE) gemm_split_kernel<PF_STORE><<<grid, GEMM_THREADS, GEMM_SMEM, s>>>(planes, tb0, tb1, tb2, g, cap);
+    else if (epi == PF_ADD) gemm_split_kernel<PF_ADD><<<grid, GEMM_THREADS, GEMM_SMEM, s>>>(planes, tb0, tb1, tb2, g, cap);
+    else gemm_split_kernel<PF_SWIGLU><<<grid, GEMM_THREADS, GEMM_SMEM, s>>>(planes, tb0, tb1, tb2, g, cap);
     return true;
 }
 
