@@ -332,6 +332,22 @@ knnssd_status knnssd_spec_accept(const float *p_dev, const float *q_dev, const i
                                  void *cuda_stream);
 
 /*
+ * The draft-and-verify loop of Sec. 4.2 with sampled instead of greedy decoding, built from the three operators above
+ * (App. C.1's temperature / top-p; the keep-or-resample rule described there), on an already prefilled session with an
+ * active mask.  Emits exactly max_new tokens, the first being the pending token as it stands (the prompt pass leaves the
+ * greedy one).  Each round drafts k_eff = min(k, remaining - 1) tokens: draft step j runs M(z), filters its logits into
+ * q_j and draws d_j from q_j; one verification pass gives p_0 .. p_{k_eff}; the round keeps a prefix of the drafts and
+ * emits one more token (knnssd_spec_accept's rule) and commits len += kept + 1.
+ *   uniforms_host  HOST fp32 [n_uniforms], each in [0, 1); round r (0-based) uses entries r (2k + 1) + j for draw j of its
+ *                  drafts (j < k), r (2k + 1) + k + j for the keep test of draft j, r (2k + 1) + 2k for its last draw;
+ *                  n_uniforms >= (max_new - 1) (2k + 1) (a round emits at least one token)
+ *   other arguments as knnssd_decode.  Errors as knnssd_decode; one host read-back per round.
+ */
+knnssd_status knnssd_decode_sampled(knnssd_ctx *ctx, int max_new, int k, float temperature, float top_p,
+                                    const float *uniforms_host, int n_uniforms, int *out_tokens_host, int *n_out,
+                                    int *accepts_host_or_null, knnssd_stats *stats_or_null);
+
+/*
  * Cosine top-1 (Sec. 4.2, Eq. (4)) of one query against n anchors of dimension d, all DEVICE fp32; HOST outputs.
  * KNNSSD_ERR_DEGENERATE for a zero / non-finite query or anchor.
  */

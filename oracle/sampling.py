@@ -114,3 +114,44 @@ def accept_margin(p, q, drafts, u_accept) -> float:
         if not a < b:
             break
     return float(best)
+
+
+def generate_sampled(model, first_token: int, max_new: int, k: int, skip_mask, temperature: float, top_p: float,
+                     uniforms: Sequence[float]):
+    """The draft-and-verify loop (Sec. 4.2) with sampled decoding on an ``oracle.OracleModel`` that has been prefilled.
+    Emits exactly max_new tokens, the first being ``first_token``.  Round r uses uniforms[r (2k + 1) + j] for the draw
+    of draft j, [r (2k + 1) + k + j] for its keep test and [r (2k + 1) + 2k] for the round's last draw.  Returns
+    dict(tokens, accepts, margin): margin = how close any decision of the run came to flipping (the smallest of the
+    nucleus margins, the draw gaps and the keep-test margins), for tests that compare another implementation."""
+    stride = 2 * k + 1
+    tokens: List[int] = [int(first_token)]
+    accepts: List[int] = []
+    pending, n, rnd, margin = int(first_token), model.length, 0, np.inf
+    while len(tokens) < max_new:
+        keff = min(k, max_new - len(tokens) - 1)
+        u = uniforms[rnd * stride:(rnd + 1) * stride]
+        q, drafts, cur = [], [], pending
+        for j in range(keff):
+            lg = model.forward([cur], n + j, skip_mask=skip_mask)["logits"][0]
+            qj = filtered_distribution(lg, temperature, top_p)
+            d = sample(qj, u[j])
+            margin = min(margin, nucleus_margin(lg, temperature, top_p), sample_gap(qj, u[j]))
+            q.append(qj)
+            drafts.append(d)
+            cur = d
+        lgs = model.forward([pending] + drafts, n)["logits"]
+        p = [filtered_distribution(lgs[j], temperature, top_p) for j in range(keff + 1)]
+        a, nxt = accept_or_resample(p, q, drafts, u[k:k + keff], u[2 * k])
+        for j in range(keff + 1):
+            margin = min(margin, nucleus_margin(lgs[j], temperature, top_p))
+        if keff:
+            margin = min(margin, accept_margin(p, q, drafts, u[k:k + keff]))
+        resid = np.maximum(p[a] - q[a], 0.0) if a < keff else p[keff]
+        margin = min(margin, sample_gap(resid if resid.sum() > 0 else p[a], u[2 * k]))
+        tokens.extend(drafts[:a] + [nxt])
+        accepts.append(a)
+        pending = nxt
+        n += a + 1
+        model.length = n
+        rnd += 1
+    return {"tokens": np.array(tokens, dtype=np.int32), "accepts": np.array(accepts, dtype=np.int32), "margin": float(margin)}

@@ -24,7 +24,8 @@ EXPORTS = ["knnssd_init", "knnssd_destroy", "knnssd_prefill", "knnssd_select_ski
            "knnssd_draft", "knnssd_verify", "knnssd_generate", "knnssd_decode", "knnssd_get_launch_count", "knnssd_get_length", "knnssd_set_length",
            "knnssd_set_pending", "knnssd_mask_objective", "knnssd_get_stats", "knnssd_last_error", "knnssd_time_pass", "knnssd_trace_pass", "knnssd_linear",
            "knnssd_gemm_split", "knnssd_linear_tc", "knnssd_build_anchors", "knnssd_cosine_top1", "knnssd_cosine_top1_static",
-           "knnssd_debug_barrier_timeout", "knnssd_filtered_probs", "knnssd_sample_token", "knnssd_spec_accept"]
+           "knnssd_debug_barrier_timeout", "knnssd_filtered_probs", "knnssd_sample_token", "knnssd_spec_accept",
+           "knnssd_decode_sampled"]
 
 
 class KnnssdError(RuntimeError):
@@ -87,6 +88,7 @@ def _load():
         "knnssd_filtered_probs": (I, [P, I, I, F, F, P, P]),
         "knnssd_sample_token": (I, [P, I, F, PI, P]),
         "knnssd_spec_accept": (I, [P, P, P, I, I, P, F, PI, PI, P]),
+        "knnssd_decode_sampled": (I, [P, I, I, F, F, P, I, P, PI, P, C.POINTER(Stats)]),
     }
     for name, (res, args) in sigs.items():
         fn = getattr(lib, name)
@@ -369,6 +371,17 @@ class Session:
         self._check(_lib.knnssd_decode(self.h, max_new, k, int(use_selection), out.ctypes.data, C.byref(n_out),
                                        acc.ctypes.data, C.byref(dom), C.byref(st)))
         return {"tokens": out[:n_out.value], "accepts": acc[:st.rounds].copy(), "domain": dom.value,
+                "stats": {f: getattr(st, f) for f, _ in Stats._fields_}}
+
+    def decode_sampled(self, max_new: int, k: int, temperature: float, top_p: float, uniforms):
+        """Sampled draft-and-verify loop; ``uniforms``: (max_new - 1) * (2k + 1) values in [0, 1), layout as in the header."""
+        u = np.ascontiguousarray(np.asarray(uniforms, dtype=np.float32))
+        out = np.zeros(max_new, dtype=np.int32)
+        acc = np.full(max_new, -1, dtype=np.int32)
+        n_out, st = C.c_int(), Stats()
+        self._check(_lib.knnssd_decode_sampled(self.h, max_new, k, float(temperature), float(top_p), u.ctypes.data, u.shape[0],
+                                               out.ctypes.data, C.byref(n_out), acc.ctypes.data, C.byref(st)))
+        return {"tokens": out[:n_out.value], "accepts": acc[:st.rounds].copy(),
                 "stats": {f: getattr(st, f) for f, _ in Stats._fields_}}
 
     @property

@@ -54,6 +54,8 @@ struct knnssd_ctx {
     int *chain = nullptr, *target = nullptr, *prompt = nullptr, *out_tokens = nullptr, *accept_log = nullptr;
     int *amax_i = nullptr, *flag = nullptr, *knn_out = nullptr;
     DeviceState *state = nullptr;
+    float *samp_p = nullptr, *samp_q = nullptr;   // sampled decoding: filtered distributions [kMaxRows][vocab], made on first use
+    int *samp_res = nullptr;                      // [2] result of a keep-or-resample round
     int *err_word = nullptr;   // this device's error word (bounded waits that gave up, bad token ids, non-finite logits)
     bool enqueue_failed = false;   // a pass could not be enqueued (its operation list did not reach the device)
     unsigned bar_spin_limit = 0;   // grid-barrier poll limit handed to the pass kernel (0 = its default)
@@ -473,7 +475,8 @@ void free_all(knnssd_ctx *c) {
                     c->anchor_inv_norm, c->cosines, c->amax_v, c->part_ml, c->rope_cs, c->pool_sum, c->inv_freq, c->chain,
                     c->target, c->prompt, c->out_tokens, c->accept_log, c->amax_i, c->flag, c->knn_out, c->state,
                     c->ops_full, c->ops_draft, c->bar, c->gabort, c->attn_cnt, c->amax_cnt, c->mpart_o, c->mamax_v, c->mpart_ml,
-                    c->mamax_i, c->trace, c->xs_x, c->xs_attn, c->xs_act, c->ssp, c->pf_x, c->pf_qkv, c->pf_ad, c->pf_aq, c->pf_af, c->pf_cs};
+                    c->mamax_i, c->trace, c->xs_x, c->xs_attn, c->xs_act, c->ssp, c->pf_x, c->pf_qkv, c->pf_ad, c->pf_aq, c->pf_af, c->pf_cs,
+                    c->samp_p, c->samp_q, c->samp_res};
     for (void *p : ptrs)
         if (p) cudaFree(p);
     if (c->pinned) cudaFreeHost(c->pinned);
@@ -985,6 +988,98 @@ knnssd_status knnssd_decode(knnssd_ctx *c, int max_new, int k, int use_selection
                      stats_or_null);
 }
 
+knnssd_status knnssd_decode_sampled(knnssd_ctx *c, int max_new, int k, float temperature, float top_p, const float *uniforms_host,
+                                    int n_uniforms, int *out_tokens_host, int *n_out, int *accepts_host_or_null,
+                                    knnssd_stats *stats_or_null) {
+    if (!c) return KNNSSD_ERR_INVALID_ARG;
+    DeviceGuard dg(c->device);
+    const knnssd_config &g = c->cfg;
+    const int stride = 2 * k + 1;
+    if (!out_tokens_host || !n_out || !uniforms_host || max_new < 1 || k < 0 || k > g.max_draft || !(temperature > 0.f) ||
+        !(top_p > 0.f) || !std::isfinite(temperature) || !std::isfinite(top_p) || (long long)n_uniforms < (long long)(max_new - 1) * stride)
+        return fail(c, KNNSSD_ERR_INVALID_ARG, "decode_sampled: bad arguments (need (max_new - 1) * (2k + 1) uniforms)");
+    for (int i = 0; i < (max_new - 1) * stride; ++i)
+        if (!(uniforms_host[i] >= 0.f) || !(uniforms_host[i] < 1.f))
+            return fail(c, KNNSSD_ERR_INVALID_ARG, "decode_sampled: uniforms must lie in [0, 1)");
+    if (!c->prefilled) return fail(c, KNNSSD_ERR_STATE, "decode_sampled: prefill first");
+    if (!c->has_mask) return fail(c, KNNSSD_ERR_STATE, "decode_sampled: no active skip mask");
+    if (c->len + max_new + 1 > g.max_seq) return fail(c, KNNSSD_ERR_CAPACITY, "decode_sampled: length + max_new + 1 exceeds max_seq");
+    const size_t V = (size_t)g.vocab;
+    if (!c->samp_p) {
+        if (dev_alloc(&c->samp_p, (size_t)kMaxRows * V) != cudaSuccess || dev_alloc(&c->samp_q, (size_t)kMaxRows * V) != cudaSuccess ||
+            dev_alloc(&c->samp_res, 2) != cudaSuccess) {
+            cudaGetLastError();
+            return fail(c, KNNSSD_ERR_CUDA, "decode_sampled: cannot allocate the distribution buffers");
+        }
+    }
+    cudaStream_t s = c->stream;
+    float *u_dev = nullptr;
+    const size_t n_u = (size_t)(max_new > 1 ? (max_new - 1) * stride : 1);
+    if (dev_alloc(&u_dev, n_u) != cudaSuccess) { cudaGetLastError(); return fail(c, KNNSSD_ERR_CUDA, "decode_sampled: cannot allocate the uniforms"); }
+    knnssd_status st = KNNSSD_OK;
+    auto finish = [&](knnssd_status r) { cudaStreamSynchronize(s); cudaFree(u_dev); return r; };
+    if (max_new > 1 && cudaMemcpyAsync(u_dev, uniforms_host, sizeof(float) * n_u, cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return finish(fail(c, KNNSSD_ERR_CUDA, "decode_sampled: cannot copy the uniforms"));
+    emit_first_token_kernel<<<1, 1, 0, s>>>(c->chain, c->state, c->out_tokens, c->len);
+    c->launches++;
+    int produced = 1, round = 0;
+    c->stats.rounds = c->stats.drafted = c->stats.accepted = 0;
+    c->stats.ms_draft = c->stats.ms_verify = 0.f;
+    const float inv_t = 1.0f / temperature;
+    while (produced < max_new) {
+        const int remaining = max_new - produced;
+        const int keff = k < remaining - 1 ? k : remaining - 1;
+        const float *u = u_dev + (size_t)round * stride;
+        cudaEventRecord(c->ev0, s);
+        for (int j = 0; j < keff; ++j) {
+            // draft step j: the draft model's logits of the row, filtered into q_j, the draft drawn from it
+            run_pass(c, 1, c->chain + j, j, c->active_mask.data(), 0, c->target, false);
+            sampling::filtered_probs_kernel<<<1, sampling::NT, 0, s>>>(c->logits, g.vocab, inv_t, top_p, c->samp_q + (size_t)j * V);
+            sampling::sample_kernel<<<1, sampling::NT, 0, s>>>(c->samp_q + (size_t)j * V, g.vocab, u + j, 0.f, c->chain + j + 1);
+            c->launches += 2;
+        }
+        cudaEventRecord(c->ev1, s);
+        run_pass(c, keff + 1, c->chain, 0, nullptr, 0, c->target, false);
+        sampling::filtered_probs_kernel<<<keff + 1, sampling::NT, 0, s>>>(c->logits, g.vocab, inv_t, top_p, c->samp_p);
+        sampling::spec_accept_kernel<<<1, sampling::NT, 0, s>>>(c->samp_p, c->samp_q, c->chain + 1, keff, g.vocab, u + k, u + 2 * k, 0.f,
+                                                                c->samp_res);
+        sampling::commit_sampled_kernel<<<1, 32, 0, s>>>(c->chain, c->samp_res, c->state, c->out_tokens, g.max_seq, c->accept_log, round);
+        c->launches += 3;
+        cudaEventRecord(c->ev2, s);
+        if (cudaMemcpyAsync(c->pinned, c->state, sizeof(DeviceState), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+            cudaMemcpyAsync(c->pinned + 8, c->err_word, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess)
+            return finish(fail(c, KNNSSD_ERR_CUDA, "decode_sampled: read-back failed"));
+        st = sync_check(c, "decode_sampled");
+        if (st != KNNSSD_OK) return finish(st);
+        if (c->pinned[8]) return finish(fail_device_code(c, "decode_sampled", c->pinned[8]));
+        const DeviceState *hs = reinterpret_cast<const DeviceState *>(c->pinned);
+        float ms = 0.f;
+        cudaEventElapsedTime(&ms, c->ev0, c->ev1);
+        c->stats.ms_draft += ms;
+        cudaEventElapsedTime(&ms, c->ev1, c->ev2);
+        c->stats.ms_verify += ms;
+        produced = hs->produced;
+        c->len = hs->len;
+        c->pending = hs->last_next;
+        c->stats.rounds += 1;
+        c->stats.drafted += keff;
+        c->stats.accepted += hs->last_accept;
+        ++round;
+    }
+    c->stats.tokens = produced;
+    if (cudaMemcpyAsync(out_tokens_host, c->out_tokens, sizeof(int) * max_new, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return finish(fail(c, KNNSSD_ERR_CUDA, "decode_sampled: read-back failed"));
+    if (accepts_host_or_null && round > 0 &&
+        cudaMemcpyAsync(accepts_host_or_null, c->accept_log, sizeof(int) * round, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return finish(fail(c, KNNSSD_ERR_CUDA, "decode_sampled: read-back failed"));
+    st = sync_check(c, "decode_sampled");
+    if (st == KNNSSD_OK) st = check_stream_err(c, "decode_sampled");
+    if (st != KNNSSD_OK) return finish(st);
+    *n_out = max_new;
+    if (stats_or_null) *stats_or_null = c->stats;
+    return finish(KNNSSD_OK);
+}
+
 knnssd_status knnssd_generate(knnssd_ctx *c, const int *prompt_host, int n_prompt, int max_new, int k, int use_selection,
                               int *out_tokens_host, int *n_out, int *accepts_host_or_null, int *domain_or_null,
                               knnssd_stats *stats_or_null) {
@@ -1439,7 +1534,7 @@ knnssd_status knnssd_sample_token(const float *weights_dev, int vocab, float u, 
     cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
     int *tok = nullptr;
     if (cudaMalloc(reinterpret_cast<void **>(&tok), sizeof(int)) != cudaSuccess) { cudaGetLastError(); return KNNSSD_ERR_CUDA; }
-    sampling::sample_kernel<<<1, sampling::NT, 0, s>>>(weights_dev, vocab, u, tok);
+    sampling::sample_kernel<<<1, sampling::NT, 0, s>>>(weights_dev, vocab, nullptr, u, tok);
     cudaError_t e = cudaMemcpyAsync(token_host, tok, sizeof(int), cudaMemcpyDeviceToHost, s);
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     if (e == cudaSuccess) e = cudaGetLastError();
@@ -1470,7 +1565,7 @@ knnssd_status knnssd_spec_accept(const float *p_dev, const float *q_dev, const i
     }
     int host[2] = {0, 0};
     if (e == cudaSuccess) {
-        sampling::spec_accept_kernel<<<1, sampling::NT, 0, s>>>(p_dev, q_dev, d_dev, k, vocab, u_dev, u_final, buf);
+        sampling::spec_accept_kernel<<<1, sampling::NT, 0, s>>>(p_dev, q_dev, d_dev, k, vocab, u_dev, nullptr, u_final, buf);
         e = cudaMemcpyAsync(host, buf, sizeof(int) * 2, cudaMemcpyDeviceToHost, s);
     }
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);

@@ -183,19 +183,22 @@ __device__ __forceinline__ int block_sample(const float *__restrict__ a, const f
     return 0;
 }
 
-// token <- draw from weights w[V] with uniform u.  One block.
-__global__ void __launch_bounds__(NT) sample_kernel(const float *__restrict__ w, int V, float u, int *__restrict__ token) {
+// token <- draw from weights w[V] with the uniform *u_ptr (u_val if u_ptr is null).  One block.
+__global__ void __launch_bounds__(NT) sample_kernel(const float *__restrict__ w, int V, const float *__restrict__ u_ptr, float u_val,
+                                                    int *__restrict__ token) {
     __shared__ float shf[NT / 32];
     __shared__ int shi[NT / 32];
-    const int tok = block_sample(w, nullptr, V, u, shf, shi);
+    const int tok = block_sample(w, nullptr, V, u_ptr ? *u_ptr : u_val, shf, shi);
     if (threadIdx.x == 0) *token = tok < 0 ? 0 : tok;
 }
 
 // One verification round of speculative sampling.  p [k+1][V], q [k][V] filtered distributions, drafts [k] (device),
-// u_accept [k] (device), u_final.  out[0] = number of drafts kept, out[1] = the token emitted after them.  One block.
+// u_accept [k] (device), u_final (*u_final_ptr if given).  out[0] = number of drafts kept, out[1] = the token emitted
+// after them.  One block.
 __global__ void __launch_bounds__(NT) spec_accept_kernel(const float *__restrict__ p, const float *__restrict__ q, const int *__restrict__ drafts,
-                                                         int k, int V, const float *__restrict__ u_accept, float u_final,
-                                                         int *__restrict__ out) {
+                                                         int k, int V, const float *__restrict__ u_accept,
+                                                         const float *__restrict__ u_final_ptr, float u_final, int *__restrict__ out) {
+    if (u_final_ptr) u_final = *u_final_ptr;
     __shared__ float shf[NT / 32];
     __shared__ int shi[NT / 32];
     __shared__ int s_rej;
@@ -213,6 +216,23 @@ __global__ void __launch_bounds__(NT) spec_accept_kernel(const float *__restrict
     const int tok = j < k ? block_sample(p + (size_t)j * V, q + (size_t)j * V, V, u_final, shf, shi)
                           : block_sample(p + (size_t)k * V, nullptr, V, u_final, shf, shi);
     if (threadIdx.x == 0) { out[0] = j; out[1] = tok < 0 ? 0 : tok; }
+}
+
+// The round's result into the session (one thread): res[0] = drafts kept, res[1] = the token after them; chain[1 .. k]
+// the drafts.  Same bookkeeping as the greedy accept step.
+__global__ void commit_sampled_kernel(int *__restrict__ chain, const int *__restrict__ res, DeviceState *__restrict__ st,
+                                      int *__restrict__ out_tokens, int out_cap, int *__restrict__ accept_log, int round_idx) {
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    const int a = res[0], next = res[1];
+    int p = st->produced;
+    for (int j = 0; j < a && p < out_cap; ++j) out_tokens[p++] = chain[j + 1];
+    if (p < out_cap) out_tokens[p++] = next;
+    st->produced = p;
+    st->len += a + 1;
+    st->last_accept = a;
+    st->last_next = next;
+    chain[0] = next;
+    if (accept_log) accept_log[round_idx] = a;
 }
 
 }  // namespace sampling

@@ -133,3 +133,87 @@ def test_round_without_drafts_and_bad_arguments(kb):
     with pytest.raises(E) as e:
         kb.knnssd_spec_accept(torch.cat([p, p]), p, [500], [0.5], 0.5)          # draft outside the vocabulary
     assert e.value.status == 1
+
+
+# ---- the sampled draft-and-verify loop ------------------------------------------------------------------------------
+
+def _to_dev(w):
+    return {k: ([t.cuda() for t in v] if isinstance(v, list) else v.cuda()) for k, v in w.items()}
+
+
+@pytest.mark.parametrize("shape_name", ["tiny", "stream-bf16"])
+def test_sampled_loop_at_vanishing_temperature_is_the_greedy_loop(kb, shape_name):
+    shape = si.SHAPES[shape_name]
+    mask = si.skip_mask(0, 2 * shape.n_layers, 3)
+    damp = {int(j): 0.05 for j in np.nonzero(mask)[0]}
+    w = _to_dev(si.make_model_weights(shape, 0, damp=damp, gain_spread=0.1))
+    sess = kb.Session.from_shape(shape, w, 160, max_draft=8)
+    sess.set_skipmask(mask)
+    prompt = si.uniform_tokens(0, 0, 33, shape.vocab).numpy()
+    for k in (0, 3, 8):
+        first = sess.prefill(prompt)
+        want = sess.decode(24, k)
+        assert sess.prefill(prompt) == first
+        got = sess.decode_sampled(24, k, 1e-6, 0.85, si.uniforms(k, 5, 23 * (2 * k + 1)))
+        assert np.array_equal(got["tokens"], want["tokens"]) and np.array_equal(got["accepts"], want["accepts"])
+        assert got["stats"]["accepted"] == want["stats"]["accepted"]
+
+
+@pytest.mark.parametrize("shape_name,T,need", [("tiny", 0.5, 1e-4), ("stream-bf16", 0.05, 2e-2)])
+def test_sampled_loop_matches_oracle_on_a_run_with_clear_decisions(kb, shape_name, T, need):
+    """Same uniforms on both sides.  A draw within rounding of a CDF step is a coin toss between the two sides' slightly
+    different logits, so the oracle reports how close any decision of a run came to flipping and the first seeded
+    streams of uniforms whose runs stay clear of that are the ones compared.  top_p = 2 keeps every token: over a
+    thousand tokens some nucleus boundary always lies within rounding of top_p (the filter has its own parity test
+    above).  The fp32 model (logits equal to ~1e-5) is compared at temperature 0.5; the bf16 one, whose logits differ
+    by a few 1e-4 between the sides, at a temperature low enough that the CDF's steps are far larger than that."""
+    import oracle
+    from oracle import sampling as osamp
+    shape = si.SHAPES[shape_name]
+    mask = si.skip_mask(0, 2 * shape.n_layers, 3)
+    damp = {int(j): 0.05 for j in np.nonzero(mask)[0]}
+    w = si.make_model_weights(shape, 0, damp=damp, gain_spread=0.1)
+    prompt = si.uniform_tokens(0, 0, 21, shape.vocab).numpy()
+    k, max_new, top_p = 3, 14, 2.0
+    sess = kb.Session.from_shape(shape, _to_dev(w), 96, max_draft=4)
+    sess.set_skipmask(mask)
+    compared = 0
+    for stream in range(80):
+        us = si.uniforms(11, 100 + stream, (max_new - 1) * (2 * k + 1))
+        om = oracle.OracleModel(shape, w, 96)
+        _, first, _ = om.prefill(prompt)
+        want = osamp.generate_sampled(om, first, max_new, k, mask, T, top_p, us)
+        if want["margin"] < need:
+            continue
+        assert sess.prefill(prompt) == first
+        got = sess.decode_sampled(max_new, k, T, top_p, us)
+        assert np.array_equal(got["tokens"], want["tokens"]), f"stream {stream}, oracle margin {want['margin']}"
+        assert np.array_equal(got["accepts"], want["accepts"])
+        compared += 1
+        if compared == 3:
+            break
+    assert compared >= 1, "no stream of uniforms gave a run clear of near-ties"
+
+
+def test_sampled_loop_rejects_bad_arguments(kb):
+    shape = si.SHAPES["tiny"]
+    sess = kb.Session.from_shape(shape, _to_dev(si.make_model_weights(shape, 0)), 64, max_draft=4)
+    prompt = si.uniform_tokens(0, 0, 10, shape.vocab).numpy()
+    E = kb.KnnssdError
+    with pytest.raises(E) as e:
+        sess.decode_sampled(8, 2, 0.5, 0.9, si.uniforms(0, 0, 35))         # before prefill
+    assert e.value.status == 4
+    sess.prefill(prompt)
+    sess.set_skipmask(np.zeros(8, np.uint8))
+    with pytest.raises(E) as e:
+        sess.decode_sampled(8, 2, 0.5, 0.9, si.uniforms(0, 0, 34))         # one uniform short
+    assert e.value.status == 1
+    with pytest.raises(E) as e:
+        sess.decode_sampled(8, 2, 0.0, 0.9, si.uniforms(0, 0, 35))
+    assert e.value.status == 1
+    bad = si.uniforms(0, 0, 35); bad[3] = 1.0
+    with pytest.raises(E) as e:
+        sess.decode_sampled(8, 2, 0.5, 0.9, bad)
+    assert e.value.status == 1
+    got = sess.decode_sampled(8, 2, 0.5, 0.9, si.uniforms(0, 0, 35))
+    assert len(got["tokens"]) == 8 and (got["tokens"] >= 0).all() and (got["tokens"] < shape.vocab).all()

@@ -113,3 +113,23 @@ def test_all_drafts_kept_when_the_models_agree_and_bonus_token_comes_from_p():
     p0 = np.array([0.5, 0.5, 0.0]); q0 = np.array([0.0, 0.5, 0.5])
     for ua, uf in itertools.product((0.0, 0.5, 0.99), (0.0, 0.5, 0.99)):
         assert osamp.accept_or_resample([p0, p0], [q0], [2], [ua], uf) == (0, 0)
+
+
+def test_sampled_loop_is_the_greedy_loop_as_temperature_goes_to_zero():
+    """With all mass on the arg-max the sampled draft-and-verify loop must emit the greedy loop's tokens and accept
+    counts, whatever the uniforms (the greedy loop itself is pinned to plain greedy decoding elsewhere)."""
+    import synthetic_inputs as si
+    shape = si.SHAPES["tiny"]
+    mask = si.skip_mask(0, 2 * shape.n_layers, 3)
+    damp = {int(j): 0.02 for j in np.nonzero(mask)[0]}
+    w = si.make_model_weights(shape, 0, gain_spread=0.1, damp=damp)
+    prompt = si.uniform_tokens(0, 0, 12, shape.vocab).numpy()
+    for k in (0, 2, 4):
+        om = oracle.OracleModel(shape, w, 96)
+        _, first, _ = om.prefill(prompt)
+        want = om.generate(first, 20, k, mask)
+        om2 = oracle.OracleModel(shape, w, 96)
+        om2.prefill(prompt)
+        got = osamp.generate_sampled(om2, first, 20, k, mask, 1e-7, 0.85, si.uniforms(k, 3, 19 * (2 * k + 1)))
+        assert np.array_equal(got["tokens"], want["tokens"]) and np.array_equal(got["accepts"], want["accepts"])
+        assert len(got["tokens"]) == 20
