@@ -9,6 +9,13 @@
 // NB = row blocks of eight: 1 for passes of up to 8 rows, 2 for 9..16 rows (the second block is a second 8-column
 // operand for the same weight fragments; every row is computed exactly as it would be in a one-row pass).
 //
+// PAIRED (NB = 1, passes of up to 4 rows - every draft step): the two bf16 terms of a row sit in neighbouring columns
+// of ONE 8-column operand (column 2 r = hi term of row r, 2 r + 1 = its lo term), so a weight fragment takes one MMA
+// instead of two.  The tensor pipe is what bounds the consumers' rate at these row counts, and a consumer that is
+// faster than the HBM stream drains the ring after a barrier and lets the producer run ahead again.  An output is
+// still (sum of the lo products) + (sum of the hi products), each sum accumulated over the same k-steps in the same
+// order as in the unpaired form: the numbers do not depend on which form computed them.
+//
 // The epilogue writes what the NEXT map needs: the fp32 result where something reads it as fp32 (projection buffer,
 // residual stream, logits) and, for the residual update and the SwiGLU product, the pre-split form (times the next
 // RMSNorm's gain) plus this CTA's partial sums of squares.
@@ -20,9 +27,11 @@ namespace stream {
 
 __device__ __forceinline__ uint4 ld_frag4(const uint32_t *p) { return __ldcg(reinterpret_cast<const uint4 *>(p)); }
 
-template <int NB>
+template <int NB, bool PAIRED>
 __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring &r, int cta, int n_cta, int warp, int lane,
                                                    int &w_use, bool &alive) {
+    static_assert(!PAIRED || NB == 1, "the paired form serves passes of up to 4 rows");
+    constexpr int NTM = PAIRED ? 1 : NTERM;                 // operand sets (MMAs) per weight fragment and row block
     // groups per batch: the tile loop is unrolled over them and has to stay small (instruction cache), so two row
     // blocks take half as many groups; the producer is told the same number through LinPhase::gb
     constexpr int GBN = GB / NB;
@@ -37,8 +46,10 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
     bool row_live[NB];
 #pragma unroll
     for (int nb = 0; nb < NB; ++nb) {
-        row_live[nb] = nb * 8 + g8 < p.M;
-        xsrow[nb] = p.xs + (size_t)min(nb * 8 + g8, p.M - 1) * nslots * SLOT_WORDS + t4 * 4;
+        // this lane's operand column: row nb * 8 + g8, both terms; PAIRED: term g8 & 1 of row g8 / 2
+        const int row = PAIRED ? (g8 >> 1) : nb * 8 + g8;
+        row_live[nb] = row < p.M;
+        xsrow[nb] = p.xs + (size_t)min(row, p.M - 1) * nslots * SLOT_WORDS + (PAIRED ? (g8 & 1) * 64 : 0) + t4 * 4;
     }
     int ws = w_use % WS, it = w_use / WS;
     float *red = r.red, *red_ss = r.red_ss;
@@ -54,14 +65,14 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
         for (int i = 0; i < GBN; ++i)
 #pragma unroll
             for (int nb = 0; nb < NB; ++nb) { acc[i][nb][0] = acc[i][nb][1] = acc[i][nb][2] = acc[i][nb][3] = 0.f; }
-        uint4 nx[NB][NTERM][4];                              // fragments of the next column tile, block by block, term by term
+        uint4 nx[NB][NTM][4];                                // fragments of the next column tile, block by block, term by term
         auto fetch = [&](int kt) {
             const int slot = kt * NCW + warp;
 #pragma unroll
             for (int nb = 0; nb < NB; ++nb) {
                 const bool ld = alive && row_live[nb] && slot < nslots;
 #pragma unroll
-                for (int t = 0; t < NTERM; ++t)
+                for (int t = 0; t < NTM; ++t)
 #pragma unroll
                     for (int q = 0; q < 4; ++q)
                         nx[nb][t][q] = ld ? ld_frag4(xsrow[nb] + (size_t)slot * SLOT_WORDS + t * 64 + q * 16) : make_uint4(0u, 0u, 0u, 0u);
@@ -102,11 +113,11 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
         }
         for (int kt = 0; kt < s.n_kt; ++kt) {
             const bool slot_valid = kt * NCW + warp < nslots;
-            uint32_t bf[NB][NTERM][KSTEPS][2];                // operand registers: block, term, k-step, (b0, b1)
+            uint32_t bf[NB][NTM][KSTEPS][2];                  // operand registers: block, term, k-step, (b0, b1)
 #pragma unroll
             for (int nb = 0; nb < NB; ++nb)
 #pragma unroll
-                for (int t = 0; t < NTERM; ++t)
+                for (int t = 0; t < NTM; ++t)
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
                         bf[nb][t][2 * q][0] = nx[nb][t][q].x; bf[nb][t][2 * q][1] = nx[nb][t][q].y;
@@ -120,7 +131,7 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
                 if (alive && slot_valid) {
                     const uint32_t base = smem_u32(r.wring + ws * WSTAGE) + lm_row * WPITCH + (warp * SLOT + lm_col) * 2;
                     // independent accumulator chains: block x term x parity of the k-step; smallest terms are added first
-                    float tc[NB][NTERM][2][4] = {};
+                    float tc[NB][NTM][2][4] = {};
 #pragma unroll
                     for (int j = 0; j < KSTEPS; ++j) {
                         uint32_t a0, a1, a2, a3;
@@ -128,18 +139,30 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
 #pragma unroll
                         for (int nb = 0; nb < NB; ++nb)
 #pragma unroll
-                            for (int t = NTERM - 1; t >= 0; --t)
+                            for (int t = NTM - 1; t >= 0; --t)
                                 mma_bf16(tc[nb][t][j & 1], a0, a1, a2, a3, bf[nb][t][j][0], bf[nb][t][j][1]);
                     }
+                    if (PAIRED) {
+                        // registers 0 / 1 = hi / lo part of (unit g8, row t4), 2 / 3 = of (unit g8 + 8, row t4): the sum of the
+                        // lo products first, then the hi products, as in the unpaired form; acc[..][0], [1] = the two units
+                        static_assert(NTERM == 2, "the paired form packs two terms");
 #pragma unroll
-                    for (int nb = 0; nb < NB; ++nb)
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            float sum = tc[nb][NTERM - 1][0][e] + tc[nb][NTERM - 1][1][e];
-#pragma unroll
-                            for (int t = NTERM - 2; t >= 0; --t) sum += tc[nb][t][0][e] + tc[nb][t][1][e];
-                            acc[gi][nb][e] += sum;
+                        for (int h = 0; h < 2; ++h) {
+                            float sum = tc[0][0][0][2 * h + 1] + tc[0][0][1][2 * h + 1];
+                            sum += tc[0][0][0][2 * h] + tc[0][0][1][2 * h];
+                            acc[gi][0][h] += sum;
                         }
+                    } else {
+#pragma unroll
+                        for (int nb = 0; nb < NB; ++nb)
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                float sum = tc[nb][NTM - 1][0][e] + tc[nb][NTM - 1][1][e];
+#pragma unroll
+                                for (int t = NTM - 2; t >= 0; --t) sum += tc[nb][t][0][e] + tc[nb][t][1][e];
+                                acc[gi][nb][e] += sum;
+                            }
+                    }
                 }
                 __syncwarp();
                 if (alive && lane == 0) mbar_arrive(&r.empty_w[ws]);
@@ -163,15 +186,18 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
                 const int n = idx % p.M, ur = idx / p.M, gi = ur >> gshift, rr = ur & ((1 << gshift) - 1);
                 if (rr >= s.group_size(g0 + gi)) continue;
                 // token n sits in block n / 8, column n % 8; rows 0..7 of the tile: regs 0,1; rows 8..15: regs 2,3
-                const int nb = n >> 3, n8 = n & 7;
-                const int src_lane = (rr & 7) * 4 + (n8 >> 1), reg = n8 & 1;
-                const int e0 = s.swiglu ? reg : (rr >> 3) * 2 + reg;
+                // where the eight warps left this item's partial sums.  Unpaired: lane (unit % 8, token / 2), register
+                // (unit / 8) * 2 + token % 2; paired: lane (unit % 8, token), register unit / 8
+                const int nb = PAIRED ? 0 : n >> 3, n8 = n & 7;
+                const int src_lane = (rr & 7) * 4 + (PAIRED ? n8 : (n8 >> 1)), reg = PAIRED ? 0 : (n8 & 1);
+                const int e0 = PAIRED ? (s.swiglu ? 0 : (rr >> 3)) : (s.swiglu ? reg : (rr >> 3) * 2 + reg);
+                const int e1 = PAIRED ? 1 : 2 + reg;            // SwiGLU: the up row of the unit (tile rows 8..15)
                 float s0 = 0.f, s1 = 0.f;
 #pragma unroll
                 for (int w = 0; w < NCW; ++w) {
                     const float *q = red + ((((w * GBN + gi) * NB + nb) * 32) + src_lane) * 4;
                     s0 += q[e0];
-                    if (s.swiglu) s1 += q[2 + reg];
+                    if (s.swiglu) s1 += q[e1];
                 }
                 const float ri = normed ? red_ss[n] : 1.0f;
                 const int u = s.u_lo + s.group_lo(g0 + gi) + rr;
@@ -202,7 +228,8 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
                     for (int i = lane; i < (ng << gshift); i += 32) {
                         const int gi = i >> gshift, rr = i & ((1 << gshift) - 1);
                         if (rr < s.group_size(g0 + gi))
-                            part += red[((((0 * GBN + gi) * NB + nb) * 32) + (rr & 7) * 4 + (n8 >> 1)) * 4 + (rr >> 3) * 2 + (n8 & 1)];
+                            part += PAIRED ? red[((((0 * GBN + gi) * NB + nb) * 32) + (rr & 7) * 4 + n8) * 4 + (rr >> 3)]
+                                           : red[((((0 * GBN + gi) * NB + nb) * 32) + (rr & 7) * 4 + (n8 >> 1)) * 4 + (rr >> 3) * 2 + (n8 & 1)];
                     }
                     part = warp_sum(part);
                     ss_acc[nb] += part;
