@@ -310,15 +310,15 @@ knnssd_status upload_ops(knnssd_ctx *c, const std::vector<pass::Op> &ops, pass::
     return KNNSSD_OK;
 }
 
-template <int HD, int NB, bool PAIRED> cudaError_t launch_pass_t(knnssd_ctx *c, const pass::Params &pr) {
+template <int HD, int NB, int NP> cudaError_t launch_pass_t(knnssd_ctx *c, const pass::Params &pr) {
     static bool configured[kMaxDevices] = {};          // function attributes are per device
     const int dev = current_device_slot();
     if (!configured[dev]) {
-        cudaFuncSetAttribute(pass::pass_kernel<HD, NB, PAIRED>, cudaFuncAttributeMaxDynamicSharedMemorySize, stream::SMEM_BYTES);
+        cudaFuncSetAttribute(pass::pass_kernel<HD, NB, NP>, cudaFuncAttributeMaxDynamicSharedMemorySize, stream::SMEM_BYTES);
         configured[dev] = true;
     }
     void *args[] = {const_cast<pass::Model *>(&c->model), const_cast<pass::Params *>(&pr)};
-    return cudaLaunchCooperativeKernel(reinterpret_cast<void *>(pass::pass_kernel<HD, NB, PAIRED>), dim3(c->n_sms),
+    return cudaLaunchCooperativeKernel(reinterpret_cast<void *>(pass::pass_kernel<HD, NB, NP>), dim3(c->n_sms),
                                        dim3(stream::NTHREADS), args, stream::SMEM_BYTES, c->stream);
 }
 
@@ -349,9 +349,10 @@ void run_pass_mega(knnssd_ctx *c, int M, const int *tok_dev, int pos_off, const 
     if (pr.merge_op) bars += n_attn;
     if (M > pass::BLKM) bars += n_attn;
     cudaError_t e;
-    if (M > pass::BLKM) e = c->cfg.head_dim == 128 ? launch_pass_t<128, 2, false>(c, pr) : launch_pass_t<64, 2, false>(c, pr);
-    else if (M > pass::BLKM / 2) e = c->cfg.head_dim == 128 ? launch_pass_t<128, 1, false>(c, pr) : launch_pass_t<64, 1, false>(c, pr);
-    else e = c->cfg.head_dim == 128 ? launch_pass_t<128, 1, true>(c, pr) : launch_pass_t<64, 1, true>(c, pr);
+    if (M > 12) e = c->cfg.head_dim == 128 ? launch_pass_t<128, 2, 0>(c, pr) : launch_pass_t<64, 2, 0>(c, pr);
+    else if (M > pass::BLKM) e = c->cfg.head_dim == 128 ? launch_pass_t<128, 2, 3>(c, pr) : launch_pass_t<64, 2, 3>(c, pr);
+    else if (M > pass::BLKM / 2) e = c->cfg.head_dim == 128 ? launch_pass_t<128, 1, 0>(c, pr) : launch_pass_t<64, 1, 0>(c, pr);
+    else e = c->cfg.head_dim == 128 ? launch_pass_t<128, 1, 1>(c, pr) : launch_pass_t<64, 1, 1>(c, pr);
     if (e == cudaSuccess) c->bar_total += (unsigned long long)bars * (unsigned long long)c->n_sms;
     c->launches++;
 }
@@ -1303,7 +1304,7 @@ knnssd_status knnssd_debug_barrier_timeout(knnssd_ctx *c, unsigned spin_limit) {
     pr.ops = c->ops_draft; pr.n_ops = 1; pr.M = 1; pr.tok = c->chain; pr.pos_off = 0; pr.head_row0 = 1;
     pr.argmax_out = c->target; pr.bar_spin_limit = spin_limit;
     pr.bar_base = c->bar_total + (unsigned long long)c->n_sms;   // one CTA-count beyond what this launch can reach
-    const cudaError_t le = c->cfg.head_dim == 128 ? launch_pass_t<128, 1, false>(c, pr) : launch_pass_t<64, 1, false>(c, pr);
+    const cudaError_t le = c->cfg.head_dim == 128 ? launch_pass_t<128, 1, 0>(c, pr) : launch_pass_t<64, 1, 0>(c, pr);
     c->launches++;
     if (le != cudaSuccess) return fail(c, KNNSSD_ERR_CUDA, std::string("debug_barrier_timeout: ") + cudaGetErrorString(le));
     st = sync_check(c, "debug_barrier_timeout");

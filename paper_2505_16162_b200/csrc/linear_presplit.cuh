@@ -9,9 +9,10 @@
 // NB = row blocks of eight: 1 for passes of up to 8 rows, 2 for 9..16 rows (the second block is a second 8-column
 // operand for the same weight fragments; every row is computed exactly as it would be in a one-row pass).
 //
-// PAIRED (NB = 1, passes of up to 4 rows - every draft step): the two bf16 terms of a row sit in neighbouring columns
-// of ONE 8-column operand (column 2 r = hi term of row r, 2 r + 1 = its lo term), so a weight fragment takes one MMA
-// instead of two.  The tensor pipe is what bounds the consumers' rate at these row counts, and a consumer that is
+// NP > 0 (the paired form; NP = 1: passes of up to 4 rows - every draft step; NP = 3: passes of 9..12 rows): the rows
+// are taken four at a time and the two bf16 terms of a row sit in neighbouring columns of ONE 8-column operand
+// (column 2 r = hi term of row 4 b + r, 2 r + 1 = its lo term), so a weight fragment takes one MMA per four rows
+// instead of two per eight: 1 instead of 2 for up to 4 rows, 3 instead of 4 for 9..12.  The tensor pipe is what bounds the consumers' rate at these row counts, and a consumer that is
 // faster than the HBM stream drains the ring after a barrier and lets the producer run ahead again.  An output is
 // still (sum of the lo products) + (sum of the hi products), each sum accumulated over the same k-steps in the same
 // order as in the unpaired form: the numbers do not depend on which form computed them.
@@ -27,11 +28,13 @@ namespace stream {
 
 __device__ __forceinline__ uint4 ld_frag4(const uint32_t *p) { return __ldcg(reinterpret_cast<const uint4 *>(p)); }
 
-template <int NB, bool PAIRED>
+template <int NB, int NP>
 __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring &r, int cta, int n_cta, int warp, int lane,
                                                    int &w_use, bool &alive) {
-    static_assert(!PAIRED || NB == 1, "the paired form serves passes of up to 4 rows");
-    constexpr int NTM = PAIRED ? 1 : NTERM;                 // operand sets (MMAs) per weight fragment and row block
+    constexpr bool PAIRED = NP > 0;
+    static_assert(NP * 4 <= NB * 8, "paired blocks of four rows cover at most the pass's rows");
+    constexpr int NX = PAIRED ? NP : NB;                    // operand blocks: of 4 rows (paired) or of 8 rows
+    constexpr int NTM = PAIRED ? 1 : NTERM;                 // operand sets (MMAs) per weight fragment and operand block
     // groups per batch: the tile loop is unrolled over them and has to stay small (instruction cache), so two row
     // blocks take half as many groups; the producer is told the same number through LinPhase::gb
     constexpr int GBN = GB / NB;
@@ -42,12 +45,12 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
     const bool normed = p.ss_in != nullptr;
     const int nslots = p.K >> 7;
     // this lane's 16-byte pieces: row nb*8 + g8, lane group t4; + slot * SLOT_WORDS + term * 64 + piece * 16
-    const uint32_t *xsrow[NB];
-    bool row_live[NB];
+    const uint32_t *xsrow[NX];
+    bool row_live[NX];
 #pragma unroll
-    for (int nb = 0; nb < NB; ++nb) {
-        // this lane's operand column: row nb * 8 + g8, both terms; PAIRED: term g8 & 1 of row g8 / 2
-        const int row = PAIRED ? (g8 >> 1) : nb * 8 + g8;
+    for (int nb = 0; nb < NX; ++nb) {
+        // this lane's operand column: row nb * 8 + g8, both terms; PAIRED: term g8 & 1 of row nb * 4 + g8 / 2
+        const int row = PAIRED ? nb * 4 + (g8 >> 1) : nb * 8 + g8;
         row_live[nb] = row < p.M;
         xsrow[nb] = p.xs + (size_t)min(row, p.M - 1) * nslots * SLOT_WORDS + (PAIRED ? (g8 & 1) * 64 : 0) + t4 * 4;
     }
@@ -60,16 +63,16 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
 
     for (int b = 0; b < s.n_batches; ++b) {
         const int g0 = b * GBN, ng = min(s.n_groups - g0, GBN);
-        float acc[GBN][NB][4];
+        float acc[GBN][NX][4];
 #pragma unroll
         for (int i = 0; i < GBN; ++i)
 #pragma unroll
-            for (int nb = 0; nb < NB; ++nb) { acc[i][nb][0] = acc[i][nb][1] = acc[i][nb][2] = acc[i][nb][3] = 0.f; }
-        uint4 nx[NB][NTM][4];                                // fragments of the next column tile, block by block, term by term
+            for (int nb = 0; nb < NX; ++nb) { acc[i][nb][0] = acc[i][nb][1] = acc[i][nb][2] = acc[i][nb][3] = 0.f; }
+        uint4 nx[NX][NTM][4];                                // fragments of the next column tile, block by block, term by term
         auto fetch = [&](int kt) {
             const int slot = kt * NCW + warp;
 #pragma unroll
-            for (int nb = 0; nb < NB; ++nb) {
+            for (int nb = 0; nb < NX; ++nb) {
                 const bool ld = alive && row_live[nb] && slot < nslots;
 #pragma unroll
                 for (int t = 0; t < NTM; ++t)
@@ -113,9 +116,9 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
         }
         for (int kt = 0; kt < s.n_kt; ++kt) {
             const bool slot_valid = kt * NCW + warp < nslots;
-            uint32_t bf[NB][NTM][KSTEPS][2];                  // operand registers: block, term, k-step, (b0, b1)
+            uint32_t bf[NX][NTM][KSTEPS][2];                  // operand registers: block, term, k-step, (b0, b1)
 #pragma unroll
-            for (int nb = 0; nb < NB; ++nb)
+            for (int nb = 0; nb < NX; ++nb)
 #pragma unroll
                 for (int t = 0; t < NTM; ++t)
 #pragma unroll
@@ -131,27 +134,29 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
                 if (alive && slot_valid) {
                     const uint32_t base = smem_u32(r.wring + ws * WSTAGE) + lm_row * WPITCH + (warp * SLOT + lm_col) * 2;
                     // independent accumulator chains: block x term x parity of the k-step; smallest terms are added first
-                    float tc[NB][NTM][2][4] = {};
+                    float tc[NX][NTM][2][4] = {};
 #pragma unroll
                     for (int j = 0; j < KSTEPS; ++j) {
                         uint32_t a0, a1, a2, a3;
                         ldmatrix_x4(base + j * 32, a0, a1, a2, a3);
 #pragma unroll
-                        for (int nb = 0; nb < NB; ++nb)
+                        for (int nb = 0; nb < NX; ++nb)
 #pragma unroll
                             for (int t = NTM - 1; t >= 0; --t)
                                 mma_bf16(tc[nb][t][j & 1], a0, a1, a2, a3, bf[nb][t][j][0], bf[nb][t][j][1]);
                     }
                     if (PAIRED) {
-                        // registers 0 / 1 = hi / lo part of (unit g8, row t4), 2 / 3 = of (unit g8 + 8, row t4): the sum of the
+                        // registers 0 / 1 = hi / lo part of (unit g8, row 4 nb + t4), 2 / 3 = of (unit g8 + 8, same row): the sum of the
                         // lo products first, then the hi products, as in the unpaired form; acc[..][0], [1] = the two units
                         static_assert(NTERM == 2, "the paired form packs two terms");
 #pragma unroll
-                        for (int h = 0; h < 2; ++h) {
-                            float sum = tc[0][0][0][2 * h + 1] + tc[0][0][1][2 * h + 1];
-                            sum += tc[0][0][0][2 * h] + tc[0][0][1][2 * h];
-                            acc[gi][0][h] += sum;
-                        }
+                        for (int nb = 0; nb < NX; ++nb)
+#pragma unroll
+                            for (int h = 0; h < 2; ++h) {
+                                float sum = tc[nb][0][0][2 * h + 1] + tc[nb][0][1][2 * h + 1];
+                                sum += tc[nb][0][0][2 * h] + tc[nb][0][1][2 * h];
+                                acc[gi][nb][h] += sum;
+                            }
                     } else {
 #pragma unroll
                         for (int nb = 0; nb < NB; ++nb)
@@ -174,8 +179,8 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
 #pragma unroll
         for (int gi = 0; gi < GBN; ++gi)
 #pragma unroll
-            for (int nb = 0; nb < NB; ++nb)
-                *reinterpret_cast<float4 *>(red + ((((warp * GBN + gi) * NB + nb) * 32) + lane) * 4) =
+            for (int nb = 0; nb < NX; ++nb)
+                *reinterpret_cast<float4 *>(red + ((((warp * GBN + gi) * NX + nb) * 32) + lane) * 4) =
                     make_float4(acc[gi][nb][0], acc[gi][nb][1], acc[gi][nb][2], acc[gi][nb][3]);
         asm volatile("bar.sync 1, %0;" ::"n"(NCW * 32) : "memory");
         if (alive) {
@@ -188,14 +193,14 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
                 // token n sits in block n / 8, column n % 8; rows 0..7 of the tile: regs 0,1; rows 8..15: regs 2,3
                 // where the eight warps left this item's partial sums.  Unpaired: lane (unit % 8, token / 2), register
                 // (unit / 8) * 2 + token % 2; paired: lane (unit % 8, token), register unit / 8
-                const int nb = PAIRED ? 0 : n >> 3, n8 = n & 7;
+                const int nb = PAIRED ? n >> 2 : n >> 3, n8 = PAIRED ? (n & 3) : (n & 7);
                 const int src_lane = (rr & 7) * 4 + (PAIRED ? n8 : (n8 >> 1)), reg = PAIRED ? 0 : (n8 & 1);
                 const int e0 = PAIRED ? (s.swiglu ? 0 : (rr >> 3)) : (s.swiglu ? reg : (rr >> 3) * 2 + reg);
                 const int e1 = PAIRED ? 1 : 2 + reg;            // SwiGLU: the up row of the unit (tile rows 8..15)
                 float s0 = 0.f, s1 = 0.f;
 #pragma unroll
                 for (int w = 0; w < NCW; ++w) {
-                    const float *q = red + ((((w * GBN + gi) * NB + nb) * 32) + src_lane) * 4;
+                    const float *q = red + ((((w * GBN + gi) * NX + nb) * 32) + src_lane) * 4;
                     s0 += q[e0];
                     if (s.swiglu) s1 += q[e1];
                 }
@@ -211,7 +216,7 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
                     __stcg(yp, v);
                     if (p.ys) store_split(p.ys, p.units >> 7, n, u, v * gnext[it4]);
                     // leave v^2 where this thread alone read its first partial: warp n % 8 adds them up below
-                    red[((((0 * GBN + gi) * NB + nb) * 32) + src_lane) * 4 + e0] = v * v;
+                    red[((((0 * GBN + gi) * NX + nb) * 32) + src_lane) * 4 + e0] = v * v;
                 } else {
                     __stcg(yp, s0 * ri);
                 }
@@ -222,14 +227,15 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
             if (alive) {
 #pragma unroll
                 for (int nb = 0; nb < NB; ++nb) {
-                    if (nb * 8 + warp >= p.M) continue;
+                    const int row = nb * 8 + warp;              // this warp adds up the squares of pass row `row`
+                    if (row >= p.M) continue;
                     const int n8 = warp;
                     float part = 0.f;
                     for (int i = lane; i < (ng << gshift); i += 32) {
                         const int gi = i >> gshift, rr = i & ((1 << gshift) - 1);
                         if (rr < s.group_size(g0 + gi))
-                            part += PAIRED ? red[((((0 * GBN + gi) * NB + nb) * 32) + (rr & 7) * 4 + n8) * 4 + (rr >> 3)]
-                                           : red[((((0 * GBN + gi) * NB + nb) * 32) + (rr & 7) * 4 + (n8 >> 1)) * 4 + (rr >> 3) * 2 + (n8 & 1)];
+                            part += PAIRED ? red[((((0 * GBN + gi) * NX + (row >> 2)) * 32) + (rr & 7) * 4 + (row & 3)) * 4 + (rr >> 3)]
+                                           : red[((((0 * GBN + gi) * NX + nb) * 32) + (rr & 7) * 4 + (n8 >> 1)) * 4 + (rr >> 3) * 2 + (n8 & 1)];
                     }
                     part = warp_sum(part);
                     ss_acc[nb] += part;

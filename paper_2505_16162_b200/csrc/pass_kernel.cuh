@@ -612,8 +612,9 @@ __device__ __forceinline__ void attn_merge_phase(const Model &md, const Op &op, 
 
 // ---- the pass ---------------------------------------------------------------------------------------------------
 // NB = 1: passes of up to BLKM rows; NB = 2: 9..16 rows (a kernel of its own, so that the common one stays small).
-// PAIRED (NB = 1): passes of up to 4 rows - every draft step - whose linear maps take one MMA per weight fragment.
-template <int HD, int NB, bool PAIRED>
+// NP > 0: the linear maps take the rows four at a time with both terms in one operand (NP = 1: passes of up to 4 rows -
+// every draft step; NP = 3 with NB = 2: passes of 9..12 rows); NP = 0: eight at a time, one operand per term.
+template <int HD, int NB, int NP>
 __global__ void __launch_bounds__(stream::NTHREADS, 1) pass_kernel(const Model md, const Params pr) {
     extern __shared__ __align__(128) unsigned char smem[];
     Ring r;
@@ -656,7 +657,7 @@ __global__ void __launch_bounds__(stream::NTHREADS, 1) pass_kernel(const Model m
                 lp.ss_in += (size_t)pr.head_row0 * n_cta;
                 lp.y += (size_t)(pr.out_row0 + pr.head_row0) * lp.units;
             }
-            if (ran) stream::consume_linear_pre<NB, PAIRED>(lp, r, cta, n_cta, warp, lane, w_use, alive);
+            if (ran) stream::consume_linear_pre<NB, NP>(lp, r, cta, n_cta, warp, lane, w_use, alive);
         } else if (alive) {
             if (op.type == OP_EMBED) embed_phase(md, op, pr, r, cta, n_cta, tid);
             else if (op.type == OP_KV_APPEND) { if (NB > 1) kv_append_phase<HD>(md, op, pr, cta, n_cta, warp, lane); else ran = false; }

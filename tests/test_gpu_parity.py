@@ -402,13 +402,14 @@ def test_context_beyond_2048_positions_matches_oracle(kb, shape_name):
 def test_a_row_is_bit_identical_whatever_the_pass_carries(kb, shape_name):
     """The same token at the same position gives the same logits and hidden state, bit for bit, whether it is verified
     alone (1 row), with 1..3 more rows (the form that packs both terms of a row into one product), with 4..7 more (one
-    product per term) or in a pass of 9..16 rows: losslessness on the GPU rests on this."""
+    product per term), in a pass of 9..12 rows (three packed products) or of 13..16: losslessness on the GPU rests on
+    this."""
     shape, om, sess = _pair(kb, shape_name, max_seq=160, max_draft=15)
     prompt = si.uniform_tokens(5, 0, 70, shape.vocab).numpy()
     first = sess.prefill(prompt)
     rows = si.uniform_tokens(6, 1, 15, shape.vocab).numpy()
     ref = None
-    for k in (0, 1, 3, 4, 7, 8, 15):
+    for k in (0, 1, 3, 4, 7, 8, 11, 12, 15):
         sess.set_length(70)
         sess.set_pending(first)
         g = sess.verify(rows[:k], want_logits=True, want_hidden=True)
@@ -420,7 +421,7 @@ def test_a_row_is_bit_identical_whatever_the_pass_carries(kb, shape_name):
         if k == 15:
             wide = (g["logits"].clone(), g["hidden"].clone())
     # and the other rows of the widest pass against narrower passes that contain them
-    for k in (1, 3, 4, 7, 8):
+    for k in (1, 3, 4, 7, 8, 11, 12):
         sess.set_length(70)
         sess.set_pending(first)
         g = sess.verify(rows[:k], want_logits=True, want_hidden=True)
