@@ -536,8 +536,8 @@ bool prefill_tensor(knnssd_ctx *c, int n) {
                                                 nullptr, nullptr, 0, err, c->n_sms, s);
             }
             prefill::rope_kv_rows_kernel<<<T, 256, 0, s>>>(c->pf_qkv, H, Hkv, HD, c->pf_cs, kc, vc, g.max_seq, t0);
-            prefill::attn_prompt_kernel<HD><<<dim3((T + 15) / 16, (H + 3) / 4), 128, 0, s>>>(c->pf_qkv, H, Hkv, kc, vc, g.max_seq, t0, T,
-                                                                                           c->pf_aq, c->pf_aq + (size_t)cap * nq);
+            prefill::attn_prompt_kernel<HD><<<dim3(H, (T + 63) / 64), 128, prefill::attn_smem_bytes<HD>(), s>>>(
+                c->pf_qkv, H, Hkv, kc, vc, g.max_seq, t0, T, c->pf_aq, c->pf_aq + (size_t)cap * nq);
             ok = ok && prefill::launch_gemm(c->pf_map_q, cap, ly.wo, nullptr, d, nq, T, prefill::PF_ADD, c->pf_x, d, 0, nullptr, nullptr, 0,
                                             err, c->n_sms, s);
             prefill::norm_split_kernel<<<T, 256, 0, s>>>(c->pf_x, d, ly.mlp_norm, g.rms_eps, c->pf_ad, c->pf_ad + (size_t)cap * d);

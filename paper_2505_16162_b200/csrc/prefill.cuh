@@ -11,8 +11,9 @@
 //                       SwiGLU of a gate tile and an up tile.
 //   norm_split_kernel   RMSNorm of each row, written as the two bf16 planes the next map reads.
 //   rope_kv_kernel      rotary embedding of q and k, K/V rows rounded to bf16 into the cache.
-//   attn_prompt_kernel  causal attention of 16 query rows per warp over the cached K/V, on mma.sync (the sizes are
-//                       small next to the linear maps), output written as bf16 planes for the O projection.
+//   attn_prompt_kernel  causal attention of 64 query rows per CTA (16 per warp) over the cached K/V, staged segment by
+//                       segment in shared memory, on mma.sync (the sizes are small next to the linear maps), output
+//                       written as bf16 planes for the O projection.
 //
 // Every wait in these kernels is bounded; a wait that gives up sets the error word and the kernel returns after
 // releasing its tensor memory.
@@ -456,193 +457,222 @@ __global__ void split_rows_kernel(const float *__restrict__ x, int n, bf16_t *__
 // Causal attention over the prompt
 // ---------------------------------------------------------------------------------------------
 
-// One warp per (head, block of 16 consecutive prompt rows); it walks the positions 0 .. (its last row's position) in
-// segments of 64 with a running maximum and sum per row (the softmax of a row is taken over all its positions at once
-// in exact arithmetic; the running form differs from it by rounding only).  K and V, this chunk's rows included, are
-// already in the cache in bf16; q is rotated fp32 and is split into hi + lo bf16 here (kept in shared memory, one
-// 16-row tile per warp), as are the probabilities.  m16n8k16 bf16 products, fp32 accumulation.
-// Lane (g8, t4) = (lane / 4, lane % 4) holds rows g8 and g8 + 8 of the block.  Index conventions of the two products:
-//   scores  column n = g8 of a tile is position 8 nt + g8; k-step s of the lane covers dimensions DL t4 + 4 s .. + 3
-//           for q and K alike (a dot product may take its terms in any order), so a lane reads one contiguous run of
-//           DL = HD / 4 dimensions of a K row;
-//   output  over pairs of tiles, k-indices (2 t4, 2 t4 + 1) = the lane's two positions of the first tile and
-//           (2 t4 + 8, 2 t4 + 9) those of the second; column n = g8 of V-tile j is dimension (HD / 8) g8 + j.
-// grid = (ceil(T / 16), ceil(H / 4)), 128 threads; the last row blocks (longest walks) are scheduled first.
+// One CTA of four warps per (head, block of 64 consecutive prompt rows), one warp per 16 of the rows.  The CTA walks
+// the positions 0 .. (its last row's position) in segments of 64: the segment's K and V rows (bf16, as cached; this
+// chunk's rows are in the cache already) are brought into shared memory with 16-byte asynchronous copies, two segments
+// in flight, and are read from there by all four warps with `ldmatrix` - every cached row crosses the L2 -> SM path
+// once per 64 query rows.  A shared-memory row keeps its 16-byte pieces at (piece ^ (row & 7)), so the eight rows of
+// an `ldmatrix` matrix fall into distinct banks.  Rows past the block's last position are filled with zeros.
+//
+// Arithmetic per warp: q (rotated fp32) is split into hi + lo bf16 once and stays in registers as the 16-row operand
+// of m16n8k16; scores = q . K^T with the lo term added before the hi term at every k-step; the softmax of a row is a
+// running maximum and sum over the segments (it differs from the softmax over all positions at once by rounding
+// only); the probabilities are split into hi + lo bf16 in registers (the accumulator layout of two position tiles is
+// the operand layout of one k-step) and o += p . V with V read through `ldmatrix.trans`.  fp32 accumulation.
+// The exponentials are exp2 of scores scaled by log2(e) / sqrt(HD) (`ex2.approx`, 2 ulp), the bf16 splits use the
+// hardware's round-to-nearest-even pair conversion.
+// grid = (H, ceil(T / 64)), 128 threads, attn_smem_bytes<HD>() of dynamic shared memory; the last row blocks (longest
+// walks) of all heads are scheduled first.
+constexpr int ATTN_SEG = 64;
+template <int HD> constexpr int attn_smem_bytes() { return 2 * 2 * ATTN_SEG * HD * 2; }      // 2 stages x (K, V)
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, bool valid) {
+    const int n = valid ? 16 : 0;                           // 0 bytes read: the 16 bytes are filled with zeros
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t &a0, uint32_t &a1, uint32_t &a2, uint32_t &a3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(a0), "=r"(a1), "=r"(a2), "=r"(a3) : "r"(addr));
+}
+
+// (v0, v1) -> packed bf16 pair (v0 in the low half), round to nearest even; hi part and what is left of it
+__device__ __forceinline__ uint32_t cvt_bf16x2(float v0, float v1) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(v1), "f"(v0));
+    return r;
+}
+__device__ __forceinline__ void split_pair(float v0, float v1, uint32_t &hi, uint32_t &lo) {
+    hi = cvt_bf16x2(v0, v1);
+    lo = cvt_bf16x2(v0 - __uint_as_float(hi << 16), v1 - __uint_as_float(hi & 0xffff0000u));
+}
+// c += a . b (m16n8k16, bf16 operands, fp32 accumulation); a pure function of its registers, free to be scheduled
+__device__ __forceinline__ void mma_acc(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
 template <int HD>
-__global__ void __launch_bounds__(128) attn_prompt_kernel(const float *__restrict__ qkv, int H, int Hkv, const bf16_t *__restrict__ kc,
-                                                          const bf16_t *__restrict__ vc, int max_seq, int pos0, int T,
-                                                          bf16_t *__restrict__ out_hi, bf16_t *__restrict__ out_lo) {
-    constexpr int DL = HD / 4, NW = HD / 8, VW = HD / 16, VJ = HD / 8, SEG = 64, NT = SEG / 8, RB = 16;
-    constexpr int QP = HD / 2 + 4;                           // words per q row in shared memory (padded)
-    __shared__ uint32_t qs[4][2][RB][QP];                    // [warp][term][row][word = dimensions (2w, 2w + 1)]
+__global__ void __launch_bounds__(128, 2) attn_prompt_kernel(const float *__restrict__ qkv, int H, int Hkv, const bf16_t *__restrict__ kc,
+                                                             const bf16_t *__restrict__ vc, int max_seq, int pos0, int T,
+                                                             bf16_t *__restrict__ out_hi, bf16_t *__restrict__ out_lo) {
+    constexpr int SEG = ATTN_SEG, NT = SEG / 8, KS = HD / 16, VJ = HD / 8, KP = SEG / 16, RB = 64;
+    constexpr int CH = HD / 8;                               // 16-byte pieces per row
+    constexpr int TILE = SEG * HD * 2;                       // bytes of one K (or V) segment
+    extern __shared__ __align__(128) unsigned char attn_smem[];
+    const uint32_t sm0 = stream::smem_u32(attn_smem);        // stage st: K at sm0 + st * 2 TILE, V one TILE further
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g8 = lane >> 2, t4 = lane & 3;
-    const int h = blockIdx.y * 4 + warp;
-    if (h >= H) return;                                      // whole warps only: nothing below is block-wide
-    const int rb = gridDim.x - 1 - blockIdx.x;
+    const int h = blockIdx.x;
+    const int rb = gridDim.y - 1 - blockIdx.y;               // all heads' longest walks first, the short ones fill the tail
     const int t_first = rb * RB;
-    const int p_last = pos0 + min(t_first + RB - 1, T - 1);
+    const int p_last = pos0 + min(t_first + RB - 1, T - 1);  // the block's last position
     const int n_seg = p_last / SEG + 1;
     const int kvh = h / (H / Hkv);
     const int qstride = (H + 2 * Hkv) * HD;
     const bf16_t *kbase = kc + (size_t)kvh * max_seq * HD, *vbase = vc + (size_t)kvh * max_seq * HD;
-    const float scale = 1.0f / sqrtf((float)HD);
+    const float scale = 1.4426950408889634f / sqrtf((float)HD);      // scores in units of log 2: p = 2^(s - max)
+
+    auto load_segment = [&](int seg) {
+        const uint32_t kdst = sm0 + (uint32_t)(seg & 1) * 2 * TILE, vdst = kdst + TILE;
+        for (int i = threadIdx.x; i < SEG * CH; i += 128) {
+            const int r = i / CH, c = i % CH, p = seg * SEG + r;
+            const bool ok = p <= p_last;
+            const size_t off = (size_t)(ok ? p : 0) * HD + 8 * c;
+            const uint32_t d = (uint32_t)(r * HD * 2 + ((c ^ (r & 7)) << 4));
+            cp_async16(kdst + d, kbase + off, ok);
+            cp_async16(vdst + d, vbase + off, ok);
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    load_segment(0);
+
+    // ---- this warp's rows: g8 and g8 + 8 of its 16 ----
+    const int w_first = t_first + 16 * warp;
+    const bool warp_live = w_first < T;
+    const int wp_last = pos0 + min(w_first + 15, T - 1);     // the warp's last position
     int t_row[2], p_row[2];
     bool live[2];
 #pragma unroll
-    for (int r = 0; r < 2; ++r) { t_row[r] = t_first + g8 + 8 * r; live[r] = t_row[r] < T; p_row[r] = pos0 + t_row[r]; }
+    for (int r = 0; r < 2; ++r) { t_row[r] = w_first + g8 + 8 * r; live[r] = t_row[r] < T; p_row[r] = pos0 + t_row[r]; }
 
-    // ---- the block's q rows, split into hi + lo, into this warp's tile ----
-    for (int idx = lane; idx < RB * (HD / 2); idx += 32) {
-        const int r = idx / (HD / 2), w = idx % (HD / 2);
-        float2 v = make_float2(0.f, 0.f);
-        if (t_first + r < T) v = *reinterpret_cast<const float2 *>(qkv + (size_t)(t_first + r) * qstride + (size_t)h * HD + 2 * w);
-        const uint32_t h0 = float_to_bf16_rne(v.x), h1 = float_to_bf16_rne(v.y);
-        qs[warp][0][r][w] = pack_bf16(h0, h1);
-        qs[warp][1][r][w] = pack_bf16(float_to_bf16_rne(v.x - __uint_as_float(h0 << 16)), float_to_bf16_rne(v.y - __uint_as_float(h1 << 16)));
-    }
-    __syncwarp();
-    const uint32_t *qh0 = &qs[warp][0][g8][(DL / 2) * t4], *qh1 = &qs[warp][0][g8 + 8][(DL / 2) * t4];
-    const uint32_t *ql0 = &qs[warp][1][g8][(DL / 2) * t4], *ql1 = &qs[warp][1][g8 + 8][(DL / 2) * t4];
+    // q as operand registers: k-step ks covers dimensions 16 ks .. 16 ks + 15; [0] row g8, dims 2 t4 + {0, 1};
+    // [1] row g8 + 8; [2], [3] the same rows, dims + 8
+    uint32_t qh[KS][4], ql[KS][4];
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int r = i & 1, dim = 16 * ks + 2 * t4 + 8 * (i >> 1);
+            float2 v = make_float2(0.f, 0.f);
+            if (live[r]) v = *reinterpret_cast<const float2 *>(qkv + (size_t)t_row[r] * qstride + (size_t)h * HD + dim);
+            split_pair(v.x, v.y, qh[ks][i], ql[ks][i]);
+        }
 
     float o[VJ][4];
 #pragma unroll
     for (int j = 0; j < VJ; ++j) { o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f; }
     float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};   // l_run: this lane's share of the row's sum
 
+    // ldmatrix sources of this lane.  K (plain): matrix lane / 8 = 16-byte piece (lane / 8) of the two k-steps, row
+    // lane % 8 of the position tile.  V (transposed): matrices 0, 1 = positions 0-7, 8-15 of the k-step, piece j;
+    // 2, 3 = the same positions, piece j + 1.
+    const int k_row = lane & 7, k_piece = lane >> 3;
+    const int v_row = (lane & 7) + ((lane >> 3) & 1) * 8, v_piece = lane >> 4;
+
     for (int seg = 0; seg < n_seg; ++seg) {
-        const int p_begin = seg * SEG, p_end = min(p_begin + SEG, p_last + 1);
-        auto load_k = [&](int nt, uint4 (&dst)[NW / 4]) {
-            const int p = p_begin + 8 * nt + g8;
-            const bf16_t *src = kbase + (size_t)p * HD + DL * t4;
+        if (seg + 1 < n_seg) {
+            load_segment(seg + 1);
+            asm volatile("cp.async.wait_group 1;" ::: "memory");
+        } else {
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+        }
+        __syncthreads();
+        const int p_begin = seg * SEG;
+        if (warp_live && p_begin <= wp_last) {
+            const uint32_t ks0 = sm0 + (uint32_t)(seg & 1) * 2 * TILE, vs0 = ks0 + TILE;
+            // ---- scores of rows (g8: [0], [1]; g8 + 8: [2], [3]) x positions 8 nt + 2 t4 + {0, 1} ----
+            // Four position tiles at a time: their products are independent, so the tensor pipe always has one to start.
+            float sc[NT][4];
 #pragma unroll
-            for (int q = 0; q < NW / 4; ++q)
-                dst[q] = p < p_end ? *reinterpret_cast<const uint4 *>(src + 8 * q) : make_uint4(0u, 0u, 0u, 0u);
-        };
-        float sc[NT][4];               // scores of rows (g8: [0], [1]; g8 + 8: [2], [3]) x positions 8 nt + 2 t4 + {0, 1}
-        {
-            uint4 kb[2][NW / 4];
-            load_k(0, kb[0]);
-            load_k(1, kb[1]);
+            for (int nt = 0; nt < NT; ++nt) { sc[nt][0] = sc[nt][1] = sc[nt][2] = sc[nt][3] = 0.f; }
 #pragma unroll
-            for (int nt = 0; nt < NT; ++nt) {
-                uint4(&kq)[NW / 4] = kb[nt & 1];
-                float c[4] = {0.f, 0.f, 0.f, 0.f};
+            for (int n0 = 0; n0 < NT; n0 += 4)
 #pragma unroll
-                for (int q = 0; q < NW / 4; ++q) {
-                    // words 4q .. 4q+3 of the lane's run: k-steps 2q (x, y) and 2q + 1 (z, w); the lo term first
-                    stream::mma_bf16(c, ql0[4 * q], ql1[4 * q], ql0[4 * q + 1], ql1[4 * q + 1], kq[q].x, kq[q].y);
-                    stream::mma_bf16(c, qh0[4 * q], qh1[4 * q], qh0[4 * q + 1], qh1[4 * q + 1], kq[q].x, kq[q].y);
-                    stream::mma_bf16(c, ql0[4 * q + 2], ql1[4 * q + 2], ql0[4 * q + 3], ql1[4 * q + 3], kq[q].z, kq[q].w);
-                    stream::mma_bf16(c, qh0[4 * q + 2], qh1[4 * q + 2], qh0[4 * q + 3], qh1[4 * q + 3], kq[q].z, kq[q].w);
+                for (int kk = 0; kk < KS; kk += 2) {
+                    uint32_t b[4][4];                        // per tile: (b[0], b[1]) k-step kk; (b[2], b[3]) k-step kk + 1
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int r = 8 * (n0 + i) + k_row;
+                        stream::ldmatrix_x4(ks0 + (uint32_t)(r * HD * 2) + (uint32_t)(((2 * kk + k_piece) ^ (r & 7)) << 4), b[i][0], b[i][1],
+                                            b[i][2], b[i][3]);
+                    }
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) mma_acc(sc[n0 + i], ql[kk], b[i][0], b[i][1]);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) mma_acc(sc[n0 + i], qh[kk], b[i][0], b[i][1]);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) mma_acc(sc[n0 + i], ql[kk + 1], b[i][2], b[i][3]);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) mma_acc(sc[n0 + i], qh[kk + 1], b[i][2], b[i][3]);
                 }
-                sc[nt][0] = c[0]; sc[nt][1] = c[1]; sc[nt][2] = c[2]; sc[nt][3] = c[3];
-                if (nt + 2 < NT) load_k(nt + 2, kq);
+            // ---- running softmax per row: new maximum, old sums and outputs rescaled ----
+            const bool diagonal = p_begin + SEG - 1 > pos0 + w_first;      // some (row, position) of the tile is masked
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+                float mx = -INFINITY;
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const int p = p_begin + 8 * nt + 2 * t4 + e;
+                        float &v = sc[nt][2 * r + e];
+                        v = (!diagonal || (live[r] && p <= p_row[r])) ? v * scale : -INFINITY;
+                        mx = fmaxf(mx, v);
+                    }
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+                const float m_new = fmaxf(m_run[r], mx);
+                const float f = m_run[r] == -INFINITY ? 0.f : exp2f(m_run[r] - m_new);
+                m_run[r] = m_new;
+                l_run[r] *= f;
+                const float m_sub = m_new == -INFINITY ? 0.f : m_new;      // a row with nothing to see yet: 2^(-inf) = 0
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        float &v = sc[nt][2 * r + e];
+                        v = exp2f(v - m_sub);
+                        l_run[r] += v;
+                    }
+#pragma unroll
+                for (int j = 0; j < VJ; ++j) { o[j][2 * r] *= f; o[j][2 * r + 1] *= f; }
+            }
+            // ---- o += p V, 16 positions per k-step ----
+#pragma unroll
+            for (int kp = 0; kp < KP; ++kp) {
+                uint32_t ah[4], al[4];     // [0], [1]: rows g8, g8 + 8, positions 16 kp + 2 t4 + {0, 1}; [2], [3]: positions + 8
+#pragma unroll
+                for (int i = 0; i < 4; ++i) split_pair(sc[2 * kp + (i >> 1)][2 * (i & 1)], sc[2 * kp + (i >> 1)][2 * (i & 1) + 1], ah[i], al[i]);
+                const int r = 16 * kp + v_row;
+                const uint32_t rowaddr = vs0 + (uint32_t)(r * HD * 2);
+#pragma unroll
+                for (int j = 0; j < VJ; j += 4) {
+                    uint32_t b[4][2];                        // dimension tiles j .. j + 3
+                    ldmatrix_x4_trans(rowaddr + (uint32_t)(((j + v_piece) ^ (r & 7)) << 4), b[0][0], b[0][1], b[1][0], b[1][1]);
+                    ldmatrix_x4_trans(rowaddr + (uint32_t)(((j + 2 + v_piece) ^ (r & 7)) << 4), b[2][0], b[2][1], b[3][0], b[3][1]);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) mma_acc(o[j + i], al, b[i][0], b[i][1]);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) mma_acc(o[j + i], ah, b[i][0], b[i][1]);
+                }
             }
         }
-        auto load_v = [&](int nt, uint4 (&dst)[2][(VW + 3) / 4]) {
-#pragma unroll
-            for (int rr = 0; rr < 2; ++rr) {
-                const int p = p_begin + 8 * nt + 2 * t4 + rr;
-                const bf16_t *src = vbase + (size_t)p * HD + 2 * VW * g8;
-                if (VW >= 4) {
-#pragma unroll
-                    for (int q = 0; q < VW / 4; ++q)
-                        dst[rr][q] = p < p_end ? *reinterpret_cast<const uint4 *>(src + 8 * q) : make_uint4(0u, 0u, 0u, 0u);
-                } else {
-                    const uint2 v = p < p_end ? *reinterpret_cast<const uint2 *>(src) : make_uint2(0u, 0u);
-                    dst[rr][0] = make_uint4(v.x, v.y, 0u, 0u);
-                }
-            }
-        };
-        uint4 vb[2][2][(VW + 3) / 4];
-        load_v(0, vb[0]);
-        load_v(1, vb[1]);
-
-        // ---- running softmax per row: new maximum, old sums and outputs rescaled ----
-#pragma unroll
-        for (int r = 0; r < 2; ++r) {
-            float mx = -INFINITY;
-#pragma unroll
-            for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-                for (int e = 0; e < 2; ++e) {
-                    const int p = p_begin + 8 * nt + 2 * t4 + e;
-                    float &v = sc[nt][2 * r + e];
-                    v = (live[r] && p <= p_row[r]) ? v * scale : -INFINITY;
-                    mx = fmaxf(mx, v);
-                }
-            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-            const float m_new = fmaxf(m_run[r], mx);
-            const float f = m_run[r] == -INFINITY ? 0.f : expf(m_run[r] - m_new);
-            m_run[r] = m_new;
-            l_run[r] *= f;
-#pragma unroll
-            for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-                for (int e = 0; e < 2; ++e) {
-                    float &v = sc[nt][2 * r + e];
-                    v = v == -INFINITY ? 0.f : expf(v - m_new);
-                    l_run[r] += v;
-                }
-#pragma unroll
-            for (int j = 0; j < VJ; ++j) { o[j][2 * r] *= f; o[j][2 * r + 1] *= f; }
-        }
-
-        // ---- o += p V ----
-#pragma unroll
-        for (int np = 0; np < NT; np += 2) {
-            uint32_t ah[4], al[4];     // [0], [1]: rows g8, g8 + 8 of tile np; [2], [3]: of tile np + 1
-#pragma unroll
-            for (int i = 0; i < 2; ++i)
-#pragma unroll
-                for (int r = 0; r < 2; ++r) {
-                    const float v0 = sc[np + i][2 * r], v1 = sc[np + i][2 * r + 1];
-                    const uint32_t h0 = float_to_bf16_rne(v0), h1 = float_to_bf16_rne(v1);
-                    ah[2 * i + r] = pack_bf16(h0, h1);
-                    al[2 * i + r] = pack_bf16(float_to_bf16_rne(v0 - __uint_as_float(h0 << 16)), float_to_bf16_rne(v1 - __uint_as_float(h1 << 16)));
-                }
-#pragma unroll
-            for (int j = 0; j < VJ; ++j) {
-                const int wi = (j >> 1) & 3;
-                uint32_t b[2];
-#pragma unroll
-                for (int i = 0; i < 2; ++i) {
-                    const uint4 &wa = vb[i][0][j / 8], &wb = vb[i][1][j / 8];
-                    const uint32_t xa = wi == 0 ? wa.x : wi == 1 ? wa.y : wi == 2 ? wa.z : wa.w;
-                    const uint32_t xb = wi == 0 ? wb.x : wi == 1 ? wb.y : wi == 2 ? wb.z : wb.w;
-                    b[i] = __byte_perm(xa, xb, (j & 1) ? 0x7632 : 0x5410);     // dimension j of the two positions' rows
-                }
-                stream::mma_bf16(o[j], al[0], al[1], al[2], al[3], b[0], b[1]);
-                stream::mma_bf16(o[j], ah[0], ah[1], ah[2], ah[3], b[0], b[1]);
-            }
-            if (np + 2 < NT) { load_v(np + 2, vb[0]); load_v(np + 3, vb[1]); }
-        }
+        __syncthreads();                                     // the stage is refilled by the next round's copies
     }
 
-    // ---- rows g8 ([0], [1]) and g8 + 8 ([2], [3]): dimensions DL t4 + j and DL t4 + VJ + j, divided by the row's sum ----
+    // ---- rows g8 ([0], [1]) and g8 + 8 ([2], [3]) x dimensions 8 j + 2 t4 + {0, 1}, divided by the row's sum ----
 #pragma unroll
     for (int r = 0; r < 2; ++r) {
         float l = l_run[r];
         l += __shfl_xor_sync(0xffffffffu, l, 1);
         l += __shfl_xor_sync(0xffffffffu, l, 2);
         if (!live[r]) continue;
-        const size_t base = (size_t)t_row[r] * ((size_t)H * HD) + (size_t)h * HD + DL * t4;
+        const size_t base = (size_t)t_row[r] * ((size_t)H * HD) + (size_t)h * HD + 2 * t4;
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-            uint32_t hw[VJ / 2], lw[VJ / 2];
-#pragma unroll
-            for (int j = 0; j < VJ; j += 2) {
-                const float v0 = o[j][2 * r + half] / l, v1 = o[j + 1][2 * r + half] / l;
-                const uint32_t h0 = float_to_bf16_rne(v0), h1 = float_to_bf16_rne(v1);
-                hw[j >> 1] = pack_bf16(h0, h1);
-                lw[j >> 1] = pack_bf16(float_to_bf16_rne(v0 - __uint_as_float(h0 << 16)), float_to_bf16_rne(v1 - __uint_as_float(h1 << 16)));
-            }
-#pragma unroll
-            for (int w = 0; w < VJ / 2; w += 4) {
-                *reinterpret_cast<uint4 *>(out_hi + base + half * VJ + 2 * w) = make_uint4(hw[w], hw[w + 1], hw[w + 2], hw[w + 3]);
-                *reinterpret_cast<uint4 *>(out_lo + base + half * VJ + 2 * w) = make_uint4(lw[w], lw[w + 1], lw[w + 2], lw[w + 3]);
-            }
+        for (int j = 0; j < VJ; ++j) {
+            uint32_t hw, lw;
+            split_pair(o[j][2 * r] / l, o[j][2 * r + 1] / l, hw, lw);
+            *reinterpret_cast<uint32_t *>(out_hi + base + 8 * j) = hw;
+            *reinterpret_cast<uint32_t *>(out_lo + base + 8 * j) = lw;
         }
     }
 }
