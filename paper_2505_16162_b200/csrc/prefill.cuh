@@ -354,6 +354,215 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap ta, const __grid_constant_
     }
 }
 
+// 16 consecutive accumulator columns of this thread's lane.
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+          "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// The same contraction on tiles of 128 tokens x 320 units (store and add epilogues), for the maps whose unit count
+// makes 320-wide tiles fill the SMs better (5120 units x 1024 rows: 128 tiles = one round, where 216 tiles of 192 columns
+// take two).  Two double-buffered accumulators of 320 columns do not fit the 512 columns of tensor memory, so the tile
+// is cut into two halves of 160 columns whose chunks are staggered by half a chunk, and three accumulators of 160
+// columns rotate between them: half A's chunk i covers k-blocks [8 i, 8 i + 8) in accumulator i mod 3, half B's chunk j
+// covers [8 j - 4, 8 j + 4) (its first one [0, 4)) in accumulator (j + 1) mod 3.  When a chunk ends, its half goes on
+// in the accumulator the other half left four k-blocks earlier (moved out by then), and the four epilogue warps of
+// the half move the finished sum into their registers while both halves keep the tensor core busy.
+// Same operand staging, maps and arguments as gemm_split_kernel with bn = 320.
+constexpr int WIDE_BN = 320, WIDE_HALF = 160;
+constexpr int WIDE_STAGE = 2 * A_BYTES + WIDE_BN * BK * 2;
+constexpr int WIDE_SMEM = STAGES * WIDE_STAGE + 1024 + 128;
+
+// Accumulator and how many times it was used before: half 0 chunk i / half 1 chunk j (see above).
+__device__ __forceinline__ void wide_slot(int half, int i, int &buf, int &use) {
+    if (half == 0) { buf = i % 3; use = 2 * (i / 3) + (buf == 0 ? 0 : 1); }
+    else { buf = (i + 1) % 3; use = 2 * (i / 3) + (buf == 0 ? 1 : 0); }
+}
+
+template <int EPI>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+gemm_wide_kernel(const __grid_constant__ CUtensorMap ta, const __grid_constant__ CUtensorMap tb0,
+                 const __grid_constant__ CUtensorMap tb1, const __grid_constant__ CUtensorMap tb2, GemmArgs g, int Tpad) {
+    static_assert(EPI == PF_STORE || EPI == PF_ADD, "wide tiles: store and add epilogues");
+    extern __shared__ unsigned char pf_smem_raw[];
+    unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(pf_smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint64_t *full = reinterpret_cast<uint64_t *>(smem + STAGES * WIDE_STAGE);
+    uint64_t *empty = full + STAGES;
+    uint64_t *acc_full = empty + STAGES;          // [3]: a chunk's sum is complete in accumulator b
+    uint64_t *acc_empty = acc_full + 3;           // [3]: the half's epilogue warps have moved accumulator b's sum out
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_empty + 3);
+    volatile int *cta_abort = reinterpret_cast<volatile int *>(tmem_slot + 1);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int t0 = blockIdx.x * BM;
+    const int n0 = blockIdx.y * WIDE_BN;
+    const int nkb = g.K / BK;
+    // chunks per half: A [0, 8), [8, 16), ..; B [0, 4), [4, 12), ..
+    const int n_chunks[2] = {(nkb + CHUNK_KB - 1) / CHUNK_KB, nkb <= CHUNK_KB / 2 ? 1 : 1 + (nkb - CHUNK_KB / 2 + CHUNK_KB - 1) / CHUNK_KB};
+    constexpr int HALF_WARPS = (GEMM_THREADS / 32 - 2) / 2;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        for (int b = 0; b < 3; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], HALF_WARPS); }
+        *cta_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // ---- TMA producer ----
+            int armed = 0;
+            for (int kb = 0; kb < nkb; ++kb) {
+                const int s = kb % STAGES;
+                const uint32_t ph = (uint32_t)(kb / STAGES) & 1u;
+                if (!pf_wait(&empty[s], ph ^ 1u, cta_abort, g.err, 31)) break;
+                unsigned char *st = smem + s * WIDE_STAGE;
+                stream::mbar_expect_tx(&full[s], WIDE_STAGE);
+                tma_load_2d(st, &ta, kb * BK, t0, &full[s]);
+                tma_load_2d(st + A_BYTES, &ta, kb * BK, Tpad + t0, &full[s]);
+#pragma unroll
+                for (int j = 0; j < WIDE_BN / BOX_N; ++j) {
+                    const CUtensorMap *wm = &tb0;
+                    int wrow = n0 + j * BOX_N;
+                    if (wrow >= g.nA) {                              // stacked matrices: the box lies in the second or third one
+                        wm = &tb1; wrow -= g.nA;
+                        if (wrow >= g.nB) { wm = &tb2; wrow -= g.nB; }
+                    }
+                    tma_load_2d(st + 2 * A_BYTES + j * BOX_N * BK * 2, wm, kb * BK, wrow, &full[s]);
+                }
+                armed = kb + 1;
+            }
+            if (*cta_abort) {
+                for (int kb = (armed > STAGES ? armed - STAGES : 0); kb < armed; ++kb) {
+                    unsigned spins = 0;
+                    while (!mbar_try_wait(&full[kb % STAGES], (uint32_t)(kb / STAGES) & 1u) && ++spins < WAIT_LIMIT) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // ---- MMA issue: per stage 4 k-steps x (hi, lo) x (half A, half B) ----
+            bool ok = true;
+            const uint32_t idesc = umma_idesc(WIDE_HALF);
+            int cur[2] = {-1, -1};                 // chunk each half is in
+            uint32_t acc_addr[2] = {0u, 0u};
+            int cur_buf[2] = {0, 0};
+            for (int kb = 0; kb < nkb && ok; ++kb) {
+                // chunk boundaries: A at kb = 0, 8, 16, ..; B at kb = 0, 4, 12, 20, ..
+                bool fresh[2] = {false, false};
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const bool boundary = h == 0 ? (kb % CHUNK_KB == 0) : (kb == 0 || kb % CHUNK_KB == CHUNK_KB / 2);
+                    if (!boundary || !ok) continue;
+                    if (cur[h] >= 0) umma_commit(&acc_full[cur_buf[h]]);
+                    ++cur[h];
+                    int buf, use;
+                    wide_slot(h, cur[h], buf, use);
+                    ok = pf_wait(&acc_empty[buf], ((uint32_t)use & 1u) ^ 1u, cta_abort, g.err, 34);
+                    cur_buf[h] = buf;
+                    acc_addr[h] = tmem + (uint32_t)(buf * WIDE_HALF);
+                    fresh[h] = true;
+                }
+                if (!ok) break;
+                tc_fence_after();
+                const int s = kb % STAGES;
+                const uint32_t ph = (uint32_t)(kb / STAGES) & 1u;
+                ok = pf_wait(&full[s], ph, cta_abort, g.err, 32);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t a_hi = smem_u32(smem + s * WIDE_STAGE), a_lo = a_hi + A_BYTES, bw = a_hi + 2 * A_BYTES;
+#pragma unroll
+                for (int k = 0; k < BK / 16; ++k) {
+                    const uint64_t dah = umma_desc(a_hi + 32 * k), dal = umma_desc(a_lo + 32 * k);
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const uint64_t db = umma_desc(bw + h * (WIDE_HALF * BK * 2) + 32 * k);
+                        umma_bf16(acc_addr[h], dah, db, idesc, (fresh[h] && k == 0) ? 0u : 1u);
+                        umma_bf16(acc_addr[h], dal, db, idesc, 1u);
+                    }
+                }
+                umma_commit(&empty[s]);
+            }
+            // the last chunks; on the abort path every accumulator is signalled so that no epilogue warp keeps waiting
+            if (ok) { umma_commit(&acc_full[cur_buf[0]]); umma_commit(&acc_full[cur_buf[1]]); }
+            else { umma_commit(&acc_full[0]); umma_commit(&acc_full[1]); umma_commit(&acc_full[2]); }
+        }
+    } else {
+        // ---- epilogue warps: warp w reads lanes 32 (w % 4) .. + 31 = tokens t0 + 32 (w % 4) + lane; warps 2..5 own half A
+        //      (tile columns 0 .. 159), warps 6..9 half B; acc[] = this thread's running sums over its half's chunks (the
+        //      compiler keeps a few dozen of the 160 in local memory: touched once per chunk) ----
+        const int q = warp & 3, hsel = (warp - 2) >> 2;
+        const int t = t0 + 32 * q + lane;
+        const uint32_t trow = tmem + ((uint32_t)(32 * q) << 16);
+        float acc[WIDE_HALF];
+#pragma unroll
+        for (int i = 0; i < WIDE_HALF; ++i) acc[i] = 0.f;
+        bool ok = true;
+        for (int c = 0; c < n_chunks[hsel] && ok; ++c) {
+            int buf, use;
+            wide_slot(hsel, c, buf, use);
+            ok = __all_sync(0xffffffffu, pf_wait(&acc_full[buf], (uint32_t)use & 1u, cta_abort, g.err, 33) && !*cta_abort);
+            if (!ok) break;
+            tc_fence_after();
+#pragma unroll
+            for (int gi = 0; gi < WIDE_HALF / 16; ++gi) {
+                float v[16];
+                tmem_ld16(trow + (uint32_t)(buf * WIDE_HALF + 16 * gi), v);
+#pragma unroll
+                for (int i = 0; i < 16; ++i) acc[16 * gi + i] += v[i];
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) stream::mbar_arrive(&acc_empty[buf]);
+        }
+        if (ok && t < g.T) {
+#pragma unroll
+            for (int gi = 0; gi < WIDE_HALF / 16; ++gi) {
+                const int c0 = hsel * WIDE_HALF + 16 * gi;
+                if (n0 + c0 >= g.N) continue;
+                float *yp = g.y + (size_t)t * g.ldy + g.col0 + n0 + c0;
+                if (n0 + c0 + 16 <= g.N) {
+#pragma unroll
+                    for (int i = 0; i < 16; i += 4) {
+                        float4 o = make_float4(acc[16 * gi + i], acc[16 * gi + i + 1], acc[16 * gi + i + 2], acc[16 * gi + i + 3]);
+                        if (EPI == PF_ADD) {
+                            const float4 x = *reinterpret_cast<const float4 *>(yp + i);
+                            o.x += x.x; o.y += x.y; o.z += x.z; o.w += x.w;
+                        }
+                        *reinterpret_cast<float4 *>(yp + i) = o;
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        if (n0 + c0 + i < g.N) yp[i] = EPI == PF_ADD ? yp[i] + acc[16 * gi + i] : acc[16 * gi + i];
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
+    }
+}
+
 // ---------------------------------------------------------------------------------------------
 // Row-wise kernels around the contractions
 // ---------------------------------------------------------------------------------------------

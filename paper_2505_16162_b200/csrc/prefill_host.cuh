@@ -51,24 +51,33 @@ inline bool gemm_attrs_once() {
         cudaFuncSetAttribute(gemm_split_kernel<PF_STORE>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM) == cudaSuccess &&
         cudaFuncSetAttribute(gemm_split_kernel<PF_ADD>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM) == cudaSuccess &&
         cudaFuncSetAttribute(gemm_split_kernel<PF_SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM) == cudaSuccess &&
+        cudaFuncSetAttribute(gemm_wide_kernel<PF_STORE>, cudaFuncAttributeMaxDynamicSharedMemorySize, WIDE_SMEM) == cudaSuccess &&
+        cudaFuncSetAttribute(gemm_wide_kernel<PF_ADD>, cudaFuncAttributeMaxDynamicSharedMemorySize, WIDE_SMEM) == cudaSuccess &&
         cudaFuncSetAttribute(attn_prompt_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_smem_bytes<128>()) == cudaSuccess &&
         cudaFuncSetAttribute(attn_prompt_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_smem_bytes<64>()) == cudaSuccess;
     done[dev] = ok;
     return ok;
 }
 
-// Accumulator columns per tile: all CTAs of a launch run at once on n_sms SMs, round after round, and a round takes
-// time in proportion to the bytes a k-block brings in (two activation planes of 128 rows + bn weight rows); the width
-// with the lowest rounds x bytes wins (ties: the wider tile).
-inline int pick_bn(int T, int N, bool swiglu, int n_sms) {
+// Accumulator columns per tile.  All CTAs of a launch run at once on n_sms SMs, round after round.  The main loop is
+// bound by shared-memory traffic (measured: 0.50 / 0.69 / 0.70 us per k-block at 128 / 192 / 256 columns, 1.0 - 1.3 at
+// 2 x 160): per k-block TMA writes the two activation planes (32 KB) and bn / 8 KB of weights, and the tensor core reads
+// the planes once and the weights twice (hi and lo products), 64 + 3 bn / 8 KB in all; the 320-column tiles of
+// gemm_wide_kernel (returned as WIDE_BN; store and add epilogues only) read the planes once per half and are charged
+// 15 % on top, as measured.  A round also costs a fixed ~10 us (tensor-memory allocation, first copies, epilogue),
+// 1960 KB at that rate.  The width with the lowest rounds x (traffic x k-blocks + fixed) wins (ties: the wider tile).
+inline int pick_bn(int T, int N, int K, bool swiglu, int n_sms) {
     const int row_tiles = (T + BM - 1) / BM;
+    const long nkb = K / BK;
     int best = 0;
     long best_cost = 0;
-    for (int bn = BOX_N; bn <= BN_MAX; bn += BOX_N) {
+    for (int bn = BOX_N; bn <= (swiglu ? BN_MAX : WIDE_BN); bn += BOX_N) {
+        if (bn > BN_MAX && bn != WIDE_BN) continue;
         if (swiglu && bn % 128) continue;
         const int per = swiglu ? bn / 2 : bn;
         const long ctas = (long)row_tiles * ((N + per - 1) / per);
-        const long cost = ((ctas + n_sms - 1) / n_sms) * (2 * BM + bn);
+        const long traffic = bn == WIDE_BN ? 248 : 64 + 3 * bn / 8;
+        const long cost = ((ctas + n_sms - 1) / n_sms) * (traffic * nkb + 1960);
         if (!best || cost <= best_cost) { best = bn; best_cost = cost; }
     }
     return best;
@@ -94,11 +103,13 @@ inline bool launch_gemm(const CUtensorMap &planes, int cap, const void *W0, cons
         tb1 = tb0;
         tb2 = tb0;
     }
-    const int bn = pick_bn(T, N, epi == PF_SWIGLU, n_sms);
+    const int bn = pick_bn(T, N, K, epi == PF_SWIGLU, n_sms);
     GemmArgs g{T, K, N, bn, y, ldy, col0, out_hi, out_lo, ldo, err, stacked ? nA : N, stacked ? nB : 0};
     const int per = epi == PF_SWIGLU ? bn / 2 : bn;
     const dim3 grid((T + BM - 1) / BM, (N + per - 1) / per);
-    if (epi == PF_STORE) gemm_split_kernel<PF_STORE><<<grid, GEMM_THREADS, GEMM_SMEM, s>>>(planes, tb0, tb1, tb2, g, cap);
+    if (bn == WIDE_BN && epi == PF_STORE) gemm_wide_kernel<PF_STORE><<<grid, GEMM_THREADS, WIDE_SMEM, s>>>(planes, tb0, tb1, tb2, g, cap);
+    else if (bn == WIDE_BN) gemm_wide_kernel<PF_ADD><<<grid, GEMM_THREADS, WIDE_SMEM, s>>>(planes, tb0, tb1, tb2, g, cap);
+    else if (epi == PF_STORE) gemm_split_kernel<PF_STORE><<<grid, GEMM_THREADS, GEMM_SMEM, s>>>(planes, tb0, tb1, tb2, g, cap);
     else if (epi == PF_ADD) gemm_split_kernel<PF_ADD><<<grid, GEMM_THREADS, GEMM_SMEM, s>>>(planes, tb0, tb1, tb2, g, cap);
     else gemm_split_kernel<PF_SWIGLU><<<grid, GEMM_THREADS, GEMM_SMEM, s>>>(planes, tb0, tb1, tb2, g, cap);
     return true;

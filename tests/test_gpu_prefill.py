@@ -48,8 +48,11 @@ def _inputs(n_out, n_in, T, seed=3):
 GEMM_CASES = [(512, 256, 128), (1000, 320, 77), (136, 64, 5), (640, 1024, 300), (5120, 5120, 260), (264, 13824, 130),
               (15360, 5120, 1),
               # tile widths other than 128 columns (the launch picks the width with the fewest column-rounds on the
-              # GPU's SMs): 192, 320 (two MMAs per step) and 256 on a 148-SM part
-              (5120, 256, 520), (5120, 256, 900), (4608, 256, 1024)]
+              # GPU's SMs): 192, 320 and 256 on a 148-SM part
+              (5120, 256, 520), (5120, 256, 900), (4608, 256, 1024),
+              # 320-column tiles on three rotating accumulators: several staggered chunks per half with a short last
+              # one; a ragged last tile (136 of 320 columns, a weight box partly past the end)
+              (5120, 2176, 900), (4936, 512, 1000)]
 
 
 @pytest.mark.parametrize("n_out,n_in,T", GEMM_CASES)
