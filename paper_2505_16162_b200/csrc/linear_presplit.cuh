@@ -28,6 +28,9 @@ namespace stream {
 
 __device__ __forceinline__ uint4 ld_frag4(const uint32_t *p) { return __ldcg(reinterpret_cast<const uint4 *>(p)); }
 
+// Column groups (of 16 units) a batch of the consumer takes, by kernel form; LinPhase::gb carries it to the producer.
+template <int NB, int NP> __host__ __device__ constexpr int groups_per_batch() { return NP == 3 ? GB : GB / NB; }
+
 template <int NB, int NP>
 __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring &r, int cta, int n_cta, int warp, int lane,
                                                    int &w_use, bool &alive) {
@@ -36,8 +39,11 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
     constexpr int NX = PAIRED ? NP : NB;                    // operand blocks: of 4 rows (paired) or of 8 rows
     constexpr int NTM = PAIRED ? 1 : NTERM;                 // operand sets (MMAs) per weight fragment and operand block
     // groups per batch: the tile loop is unrolled over them and has to stay small (instruction cache), so two row
-    // blocks take half as many groups; the producer is told the same number through LinPhase::gb
-    constexpr int GBN = GB / NB;
+    // blocks of eight take half as many groups; the producer is told the same number through LinPhase::gb.  The
+    // activation fragments of a column tile are fetched from L2 once per batch, so the 9..12-row form keeps four
+    // groups: at two it would pull 0.75 bytes of activations per byte of weights.
+    constexpr int GBN = groups_per_batch<NB, NP>();
+    constexpr int RW = PAIRED ? 2 : 4;                      // floats a lane leaves per (warp, group, block) for the batch-end sums
     const Share s = make_share(p, cta, n_cta);
     const int tid = warp * 32 + lane;
     const int g8 = lane >> 2, t4 = lane & 3;
@@ -98,6 +104,7 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
         }
         // this thread's epilogue items: (unit, token) pairs, token fastest among the M live tokens.  For a residual
         // update the old value and the next gain are fetched now, long before the epilogue needs them.
+        static_assert(NCW * GBN * NX * 32 * RW * 4 <= RED_BYTES, "the batch-end sums fit the reduction buffer");
         const int gshift = s.swiglu ? 3 : 4, total = (ng << gshift) * p.M;
         constexpr int ITEMS = GBN * 16 * 8 * NB / (NCW * 32);
         float xold[ITEMS], gnext[ITEMS];
@@ -179,9 +186,11 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
 #pragma unroll
         for (int gi = 0; gi < GBN; ++gi)
 #pragma unroll
-            for (int nb = 0; nb < NX; ++nb)
-                *reinterpret_cast<float4 *>(red + ((((warp * GBN + gi) * NX + nb) * 32) + lane) * 4) =
-                    make_float4(acc[gi][nb][0], acc[gi][nb][1], acc[gi][nb][2], acc[gi][nb][3]);
+            for (int nb = 0; nb < NX; ++nb) {
+                float *dst = red + ((((warp * GBN + gi) * NX + nb) * 32) + lane) * RW;
+                if (PAIRED) *reinterpret_cast<float2 *>(dst) = make_float2(acc[gi][nb][0], acc[gi][nb][1]);
+                else *reinterpret_cast<float4 *>(dst) = make_float4(acc[gi][nb][0], acc[gi][nb][1], acc[gi][nb][2], acc[gi][nb][3]);
+            }
         asm volatile("bar.sync 1, %0;" ::"n"(NCW * 32) : "memory");
         if (alive) {
 #pragma unroll
@@ -200,7 +209,7 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
                 float s0 = 0.f, s1 = 0.f;
 #pragma unroll
                 for (int w = 0; w < NCW; ++w) {
-                    const float *q = red + ((((w * GBN + gi) * NX + nb) * 32) + src_lane) * 4;
+                    const float *q = red + ((((w * GBN + gi) * NX + nb) * 32) + src_lane) * RW;
                     s0 += q[e0];
                     if (s.swiglu) s1 += q[e1];
                 }
@@ -216,7 +225,7 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
                     __stcg(yp, v);
                     if (p.ys) store_split(p.ys, p.units >> 7, n, u, v * gnext[it4]);
                     // leave v^2 where this thread alone read its first partial: warp n % 8 adds them up below
-                    red[((((0 * GBN + gi) * NX + nb) * 32) + src_lane) * 4 + e0] = v * v;
+                    red[((((0 * GBN + gi) * NX + nb) * 32) + src_lane) * RW + e0] = v * v;
                 } else {
                     __stcg(yp, s0 * ri);
                 }
@@ -234,8 +243,8 @@ __device__ __forceinline__ void consume_linear_pre(const LinPhase &p, const Ring
                     for (int i = lane; i < (ng << gshift); i += 32) {
                         const int gi = i >> gshift, rr = i & ((1 << gshift) - 1);
                         if (rr < s.group_size(g0 + gi))
-                            part += PAIRED ? red[((((0 * GBN + gi) * NX + (row >> 2)) * 32) + (rr & 7) * 4 + (row & 3)) * 4 + (rr >> 3)]
-                                           : red[((((0 * GBN + gi) * NX + nb) * 32) + (rr & 7) * 4 + (n8 >> 1)) * 4 + (rr >> 3) * 2 + (n8 & 1)];
+                            part += PAIRED ? red[((((0 * GBN + gi) * NX + (row >> 2)) * 32) + (rr & 7) * 4 + (row & 3)) * RW + (rr >> 3)]
+                                           : red[((((0 * GBN + gi) * NX + nb) * 32) + (rr & 7) * 4 + (n8 >> 1)) * RW + (rr >> 3) * 2 + (n8 & 1)];
                     }
                     part = warp_sum(part);
                     ss_acc[nb] += part;

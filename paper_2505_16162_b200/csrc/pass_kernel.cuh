@@ -632,7 +632,7 @@ __global__ void __launch_bounds__(stream::NTHREADS, 1) pass_kernel(const Model m
                 if (op.type != OP_LINEAR) continue;
                 LinPhase lp = op.lin;
                 lp.M = pr.M;
-                lp.gb = stream::GB / NB;
+                lp.gb = stream::groups_per_batch<NB, NP>();
                 if (op.is_head) { if (pr.head_row0 >= pr.M) continue; }
                 stream::produce_linear(lp, r, cta, n_cta, lane, w_use, alive);
             }
@@ -649,7 +649,7 @@ __global__ void __launch_bounds__(stream::NTHREADS, 1) pass_kernel(const Model m
         if (op.type == OP_LINEAR) {
             LinPhase lp = op.lin;
             lp.M = pr.M;
-            lp.gb = stream::GB / NB;
+            lp.gb = stream::groups_per_batch<NB, NP>();
             if (op.is_head) {
                 if (pr.head_row0 >= pr.M) ran = false;
                 lp.M = pr.M - pr.head_row0;
