@@ -274,6 +274,13 @@ __device__ __forceinline__ void mma_bf16_top(float (&c)[4], uint32_t a0, uint32_
                  : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
 }
 
+// The same with both halves of the 16-row operand: rows 0..7 from (a0, a2), rows 8..15 from (a1, a3).
+__device__ __forceinline__ void mma_bf16_rows(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
 // Merge the segment partials of one (row m, head h) in segment order and write the result pre-split (one warp).
 template <int HD>
 __device__ __forceinline__ void attn_merge_row(const Model &md, const Op &op, int P0, int m, int h, int lane) {
@@ -331,7 +338,7 @@ __device__ __forceinline__ void attn_merge_row(const Model &md, const Op &op, in
 //           dimensions of four V rows; an operand register (two positions of one dimension) is one byte-permute of two
 //           loaded words.  p is split into two bf16 terms.
 // A lane ends up with output dimensions [DL*t4, DL*t4 + DL) of row g8, the run it holds of q.
-template <int HD>
+template <int HD, bool R16>
 __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const Params &pr, const Ring &r, int cta, int n_cta,
                                            int warp, int lane, bool defer_merge, int row0, bool all_cached) {
     constexpr int DL = HD / 4;         // dimensions of q / o per lane
@@ -341,6 +348,7 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
     constexpr int VJ = HD / 8;         // V tiles (8 dimensions each)
     constexpr int HALF = HD / 2, DPL = HD / 32;
     constexpr int NT = SEGP / 8;       // position tiles per segment
+    constexpr int NR = R16 ? 2 : 1;    // pass rows per lane: row0 + g8 and, with R16, row0 + g8 + 8 (rows 8..15 of the MMA operand)
     const int g8 = lane >> 2, t4 = lane & 3;
     const int M = pr.M, H = md.H, Hkv = md.Hkv, G = H / Hkv;
     const int P0 = md.state->len + pr.pos_off, Ttot = P0 + M;
@@ -369,17 +377,34 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
         const int rm = all_cached ? row0 + g8 : rr % M;      // the pass row this lane's MMA row stands for
         const int h = all_cached ? grp : kvh * G + min(rr / M, G - 1);   // and its query head
         const bool row_in = all_cached ? rm < M : rr < R;
+        const int rm2 = rm + BLKM;                           // R16: the lane's second row (MMA row g8 + 8), same head
         const int p_begin = seg * SEGP, p_end = min(p_begin + SEGP, Ttot);
         const int m_first = max(0, p_begin - P0);           // first row that sees this segment
         const bool writer = !all_cached && blk == 0;         // one task per (segment, K/V head) puts the new rows into the cache
         bf16_t *kbase = op.kc + (size_t)kvh * md.max_seq * HD;
         bf16_t *vbase = op.vc + (size_t)kvh * md.max_seq * HD;
-        if (all_cached && row0 + BLKM <= m_first) continue;  // none of this block's rows sees the segment
+        if (all_cached && row0 + NR * BLKM <= m_first) continue;  // none of this block's rows sees the segment
         // pass row g8's own position lies in this segment and is not in the cache yet: this lane rotates / rounds its K, V
         const bool row_new = !all_cached && g8 < M && P0 + g8 >= p_begin && P0 + g8 < p_end;
         const bool row_live = row_in && rm >= m_first;
+        const bool row_live2 = R16 && rm2 < M && rm2 >= m_first;
         // ---- this lane's run of q (row g8), of the new K row and of the new V row: load, rotate, round / split ----
         float qf[DL], kf[DL];
+        float qf2[R16 ? DL : 1];                             // R16: the second row's run of q, rotated like the first
+        if constexpr (R16) {
+            const float *qraw2 = md.qkv + (size_t)min(rm2, M - 1) * qstride + (size_t)h * HD + DL * t4;
+#pragma unroll
+            for (int e = 0; e < DL; e += 4) {
+                const float4 a = row_live2 ? __ldcg(reinterpret_cast<const float4 *>(qraw2 + e)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                qf2[e] = a.x; qf2[e + 1] = a.y; qf2[e + 2] = a.z; qf2[e + 3] = a.w;
+            }
+#pragma unroll
+            for (int e = 0; e < DL; ++e) {
+                const float qp = __shfl_xor_sync(0xffffffffu, qf2[e], 2);
+                const float2 cq = row_live2 ? my_cs[rm2 * HALF + ci + e] : make_float2(1.f, 0.f);
+                qf2[e] = upper ? (qf2[e] * cq.x + qp * cq.y) : (qf2[e] * cq.x - qp * cq.y);
+            }
+        }
         {
             const float *qraw = md.qkv + (size_t)min(rm, M - 1) * qstride + (size_t)h * HD + DL * t4;
             const float *kraw = md.qkv + (size_t)min(g8, M - 1) * qstride + (size_t)(H + kvh) * HD + DL * t4;
@@ -431,6 +456,16 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
             const uint32_t l1 = float_to_bf16_rne(qf[2 * w + 1] - __uint_as_float(h1 << 16));
             qh[w] = h0 | (h1 << 16); ql[w] = l0 | (l1 << 16);
         }
+        uint32_t qh2[R16 ? NW : 1], ql2[R16 ? NW : 1];       // R16: the second row's words
+        if constexpr (R16) {
+#pragma unroll
+            for (int w = 0; w < NW; ++w) {
+                const uint32_t h0 = float_to_bf16_rne(qf2[2 * w]), h1 = float_to_bf16_rne(qf2[2 * w + 1]);
+                const uint32_t l0 = float_to_bf16_rne(qf2[2 * w] - __uint_as_float(h0 << 16));
+                const uint32_t l1 = float_to_bf16_rne(qf2[2 * w + 1] - __uint_as_float(h1 << 16));
+                qh2[w] = h0 | (h1 << 16); ql2[w] = l0 | (l1 << 16);
+            }
+        }
         // ---- scores: one tile = 8 positions; K rows are fetched two tiles ahead ----
         auto load_k = [&](int nt, uint4 (&dst)[NW / 4]) {
             const int p = p_begin + 8 * nt + g8;
@@ -439,7 +474,7 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
             for (int q = 0; q < NW / 4; ++q)
                 dst[q] = p < p_end ? *reinterpret_cast<const uint4 *>(src + 8 * q) : make_uint4(0u, 0u, 0u, 0u);
         };
-        float sc[NT][2];                                     // scores of (row g8, positions 8*nt + 2*t4 + {0, 1})
+        float sc[NT][2 * NR];                                // scores of (row g8, positions 8*nt + 2*t4 + {0, 1}); R16: [2], [3] = row g8 + 8
         {
             constexpr int KR = NT < 4 ? NT : 4;              // tiles in flight
             uint4 kb[KR][NW / 4];
@@ -452,13 +487,21 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
 #pragma unroll
                 for (int q = 0; q < NW / 4; ++q) {
                     // words 4q .. 4q+3 of the run: k-steps 2q (x, y) and 2q + 1 (z, w)
-                    mma_bf16_top(cl, ql[4 * q], ql[4 * q + 1], kq[q].x, kq[q].y);
-                    mma_bf16_top(ch, qh[4 * q], qh[4 * q + 1], kq[q].x, kq[q].y);
-                    mma_bf16_top(cl, ql[4 * q + 2], ql[4 * q + 3], kq[q].z, kq[q].w);
-                    mma_bf16_top(ch, qh[4 * q + 2], qh[4 * q + 3], kq[q].z, kq[q].w);
+                    if constexpr (R16) {
+                        mma_bf16_rows(cl, ql[4 * q], ql2[4 * q], ql[4 * q + 1], ql2[4 * q + 1], kq[q].x, kq[q].y);
+                        mma_bf16_rows(ch, qh[4 * q], qh2[4 * q], qh[4 * q + 1], qh2[4 * q + 1], kq[q].x, kq[q].y);
+                        mma_bf16_rows(cl, ql[4 * q + 2], ql2[4 * q + 2], ql[4 * q + 3], ql2[4 * q + 3], kq[q].z, kq[q].w);
+                        mma_bf16_rows(ch, qh[4 * q + 2], qh2[4 * q + 2], qh[4 * q + 3], qh2[4 * q + 3], kq[q].z, kq[q].w);
+                    } else {
+                        mma_bf16_top(cl, ql[4 * q], ql[4 * q + 1], kq[q].x, kq[q].y);
+                        mma_bf16_top(ch, qh[4 * q], qh[4 * q + 1], kq[q].x, kq[q].y);
+                        mma_bf16_top(cl, ql[4 * q + 2], ql[4 * q + 3], kq[q].z, kq[q].w);
+                        mma_bf16_top(ch, qh[4 * q + 2], qh[4 * q + 3], kq[q].z, kq[q].w);
+                    }
                 }
                 sc[nt][0] = cl[0] + ch[0];
                 sc[nt][1] = cl[1] + ch[1];
+                if constexpr (R16) { sc[nt][2] = cl[2] + ch[2]; sc[nt][3] = cl[3] + ch[3]; }
                 if (nt + KR < NT) load_k(nt + KR, kq);
             }
         }
@@ -482,30 +525,38 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
         uint4 vb[VR][2][(VW + 3) / 4];
 #pragma unroll
         for (int i = 0; i < VR; ++i) load_v(i, vb[i]);
-        // ---- softmax over the segment for row g8 (the four lanes of a row share it) ----
-        float mx = -INFINITY;
+        // ---- softmax over the segment for row g8 (the four lanes of a row share it); R16: and for row g8 + 8 ----
+        float mx_r[NR], lsum_r[NR];
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt)
+        for (int r = 0; r < NR; ++r) {
+            const bool live_r = r == 0 ? row_live : row_live2;
+            const int rm_r = r == 0 ? rm : rm2;
+            float mx = -INFINITY;
 #pragma unroll
-            for (int e = 0; e < 2; ++e) {
-                const int p = p_begin + 8 * nt + 2 * t4 + e;
-                const bool valid = row_live && p <= P0 + rm;             // causal; also excludes p >= p_end
-                sc[nt][e] = valid ? sc[nt][e] * scale : -INFINITY;
-                mx = fmaxf(mx, sc[nt][e]);
-            }
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-        float lsum = 0.f;
+            for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt)
+                for (int e = 0; e < 2; ++e) {
+                    const int p = p_begin + 8 * nt + 2 * t4 + e;
+                    const bool valid = live_r && p <= P0 + rm_r;             // causal; also excludes p >= p_end
+                    sc[nt][2 * r + e] = valid ? sc[nt][2 * r + e] * scale : -INFINITY;
+                    mx = fmaxf(mx, sc[nt][2 * r + e]);
+                }
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+            float lsum = 0.f;
 #pragma unroll
-            for (int e = 0; e < 2; ++e) {
-                const float pj = sc[nt][e] == -INFINITY ? 0.f : expf(sc[nt][e] - mx);
-                sc[nt][e] = pj;
-                lsum += pj;
-            }
-        lsum += __shfl_xor_sync(0xffffffffu, lsum, 1);
-        lsum += __shfl_xor_sync(0xffffffffu, lsum, 2);
+            for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const float pj = sc[nt][2 * r + e] == -INFINITY ? 0.f : expf(sc[nt][2 * r + e] - mx);
+                    sc[nt][2 * r + e] = pj;
+                    lsum += pj;
+                }
+            lsum += __shfl_xor_sync(0xffffffffu, lsum, 1);
+            lsum += __shfl_xor_sync(0xffffffffu, lsum, 2);
+            mx_r[r] = mx; lsum_r[r] = lsum;
+        }
+        const float mx = mx_r[0], lsum = lsum_r[0];
         // ---- o += p V ----
         float o[VJ][4];
 #pragma unroll
@@ -514,12 +565,19 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
         for (int np = 0; np < NT; np += 2) {
             // k-indices 2t4, 2t4+1 stand for this lane's two positions of tile np, 2t4+8, 2t4+9 for those of tile np + 1
             uint32_t ah[2], al[2];
+            uint32_t ah2[2] = {0u, 0u}, al2[2] = {0u, 0u};  // R16: the same for row g8 + 8
 #pragma unroll
             for (int i = 0; i < 2; ++i) {
                 const uint32_t h0 = float_to_bf16_rne(sc[np + i][0]), h1 = float_to_bf16_rne(sc[np + i][1]);
                 const uint32_t l0 = float_to_bf16_rne(sc[np + i][0] - __uint_as_float(h0 << 16));
                 const uint32_t l1 = float_to_bf16_rne(sc[np + i][1] - __uint_as_float(h1 << 16));
                 ah[i] = h0 | (h1 << 16); al[i] = l0 | (l1 << 16);
+                if constexpr (R16) {
+                    const uint32_t g0 = float_to_bf16_rne(sc[np + i][2]), g1 = float_to_bf16_rne(sc[np + i][3]);
+                    const uint32_t m0 = float_to_bf16_rne(sc[np + i][2] - __uint_as_float(g0 << 16));
+                    const uint32_t m1 = float_to_bf16_rne(sc[np + i][3] - __uint_as_float(g1 << 16));
+                    ah2[i] = g0 | (g1 << 16); al2[i] = m0 | (m1 << 16);
+                }
             }
 #pragma unroll
             for (int j = 0; j < VJ; ++j) {
@@ -532,8 +590,13 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
                     const uint32_t xb = wi == 0 ? wb.x : wi == 1 ? wb.y : wi == 2 ? wb.z : wb.w;
                     b[i] = __byte_perm(xa, xb, (j & 1) ? 0x7632 : 0x5410);     // dimension j of the two positions' rows
                 }
-                mma_bf16_top(o[j], al[0], al[1], b[0], b[1]);
-                mma_bf16_top(o[j], ah[0], ah[1], b[0], b[1]);
+                if constexpr (R16) {
+                    mma_bf16_rows(o[j], al[0], al2[0], al[1], al2[1], b[0], b[1]);
+                    mma_bf16_rows(o[j], ah[0], ah2[0], ah[1], ah2[1], b[0], b[1]);
+                } else {
+                    mma_bf16_top(o[j], al[0], al[1], b[0], b[1]);
+                    mma_bf16_top(o[j], ah[0], ah[1], b[0], b[1]);
+                }
             }
             if (np + VR < NT) load_v(np + VR, vb[np % VR]);
             if (np + 1 + VR < NT) load_v(np + 1 + VR, vb[(np + 1) % VR]);
@@ -547,6 +610,18 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
             for (int j = 0; j < VJ; j += 4) {
                 __stcg(reinterpret_cast<float4 *>(po + j), make_float4(o[j][0], o[j + 1][0], o[j + 2][0], o[j + 3][0]));
                 __stcg(reinterpret_cast<float4 *>(po + VJ + j), make_float4(o[j][1], o[j + 1][1], o[j + 2][1], o[j + 3][1]));
+            }
+        }
+        if constexpr (R16) {
+            if (row_live2) {                                  // row g8 + 8: accumulator registers 2, 3
+                const size_t pidx = ((size_t)rm2 * H + h) * md.n_seg_max + seg;
+                if (t4 == 0) __stcg(md.part_ml + pidx, make_float2(mx_r[NR - 1], lsum_r[NR - 1]));
+                float *po = md.part_o + pidx * HD + DL * t4;
+#pragma unroll
+                for (int j = 0; j < VJ; j += 4) {
+                    __stcg(reinterpret_cast<float4 *>(po + j), make_float4(o[j][2], o[j + 1][2], o[j + 2][2], o[j + 3][2]));
+                    __stcg(reinterpret_cast<float4 *>(po + VJ + j), make_float4(o[j][3], o[j + 1][3], o[j + 2][3], o[j + 3][3]));
+                }
             }
         }
         if (defer_merge) continue;                            // a separate merge operation follows a grid barrier
@@ -663,9 +738,9 @@ __global__ void __launch_bounds__(stream::NTHREADS, 1) pass_kernel(const Model m
             else if (op.type == OP_KV_APPEND) { if (NB > 1) kv_append_phase<HD>(md, op, pr, cta, n_cta, warp, lane); else ran = false; }
             else if (op.type == OP_ATTN) {
                 if (NB == 1) {
-                    attn_phase<HD>(md, op, pr, r, cta, n_cta, warp, lane, pr.merge_op != 0, 0, false);
+                    attn_phase<HD, false>(md, op, pr, r, cta, n_cta, warp, lane, pr.merge_op != 0, 0, false);
                 } else {
-                    for (int blk = 0; blk < NB; ++blk) attn_phase<HD>(md, op, pr, r, cta, n_cta, warp, lane, true, blk * BLKM, true);
+                    attn_phase<HD, true>(md, op, pr, r, cta, n_cta, warp, lane, true, 0, true);
                 }
             }
             else if (op.type == OP_ATTN_MERGE) { if (pr.merge_op) attn_merge_phase<HD>(md, op, pr, cta, n_cta, warp, lane); else ran = false; }
