@@ -391,20 +391,6 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
         // ---- this lane's run of q (row g8), of the new K row and of the new V row: load, rotate, round / split ----
         float qf[DL], kf[DL];
         float qf2[R16 ? DL : 1];                             // R16: the second row's run of q, rotated like the first
-        if constexpr (R16) {
-            const float *qraw2 = md.qkv + (size_t)min(rm2, M - 1) * qstride + (size_t)h * HD + DL * t4;
-#pragma unroll
-            for (int e = 0; e < DL; e += 4) {
-                const float4 a = row_live2 ? __ldcg(reinterpret_cast<const float4 *>(qraw2 + e)) : make_float4(0.f, 0.f, 0.f, 0.f);
-                qf2[e] = a.x; qf2[e + 1] = a.y; qf2[e + 2] = a.z; qf2[e + 3] = a.w;
-            }
-#pragma unroll
-            for (int e = 0; e < DL; ++e) {
-                const float qp = __shfl_xor_sync(0xffffffffu, qf2[e], 2);
-                const float2 cq = row_live2 ? my_cs[rm2 * HALF + ci + e] : make_float2(1.f, 0.f);
-                qf2[e] = upper ? (qf2[e] * cq.x + qp * cq.y) : (qf2[e] * cq.x - qp * cq.y);
-            }
-        }
         {
             const float *qraw = md.qkv + (size_t)min(rm, M - 1) * qstride + (size_t)h * HD + DL * t4;
             const float *kraw = md.qkv + (size_t)min(g8, M - 1) * qstride + (size_t)(H + kvh) * HD + DL * t4;
@@ -415,6 +401,14 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
                 qf[e] = a.x; qf[e + 1] = a.y; qf[e + 2] = a.z; qf[e + 3] = a.w;
                 kf[e] = b.x; kf[e + 1] = b.y; kf[e + 2] = b.z; kf[e + 3] = b.w;
             }
+            if constexpr (R16) {
+                const float *qraw2 = md.qkv + (size_t)min(rm2, M - 1) * qstride + (size_t)h * HD + DL * t4;
+#pragma unroll
+                for (int e = 0; e < DL; e += 4) {
+                    const float4 a = row_live2 ? __ldcg(reinterpret_cast<const float4 *>(qraw2 + e)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    qf2[e] = a.x; qf2[e + 1] = a.y; qf2[e + 2] = a.z; qf2[e + 3] = a.w;
+                }
+            }
 #pragma unroll
             for (int e = 0; e < DL; ++e) {
                 const float qp = __shfl_xor_sync(0xffffffffu, qf[e], 2), kp = __shfl_xor_sync(0xffffffffu, kf[e], 2);
@@ -422,6 +416,14 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
                 const float2 ck = row_new ? my_cs[g8 * HALF + ci + e] : make_float2(1.f, 0.f);
                 qf[e] = upper ? (qf[e] * cq.x + qp * cq.y) : (qf[e] * cq.x - qp * cq.y);
                 kf[e] = upper ? (kf[e] * ck.x + kp * ck.y) : (kf[e] * ck.x - kp * ck.y);
+            }
+            if constexpr (R16) {
+#pragma unroll
+                for (int e = 0; e < DL; ++e) {
+                    const float qp = __shfl_xor_sync(0xffffffffu, qf2[e], 2);
+                    const float2 cq = row_live2 ? my_cs[rm2 * HALF + ci + e] : make_float2(1.f, 0.f);
+                    qf2[e] = upper ? (qf2[e] * cq.x + qp * cq.y) : (qf2[e] * cq.x - qp * cq.y);
+                }
             }
         }
         __syncwarp();
