@@ -523,10 +523,12 @@ bool prefill_tensor(knnssd_ctx *c, int n) {
             bf16_t *kc = reinterpret_cast<bf16_t *>(c->kcache) + (size_t)l * layer_stride;
             bf16_t *vc = reinterpret_cast<bf16_t *>(c->vcache) + (size_t)l * layer_stride;
             prefill::norm_split_kernel<<<T, 256, 0, s>>>(c->pf_x, d, ly.attn_norm, g.rms_eps, c->pf_ad, c->pf_ad + (size_t)cap * d);
+            bool heads_done = false;     // rotary embedding and K / V rows done by the q / k / v launch's epilogue
             if (nq % prefill::BOX_N == 0 && nkv % prefill::BOX_N == 0) {
                 // q, k and v in one launch over the stacked units (their columns of the projection buffer are adjacent)
+                const prefill::QkvFuse fuse{c->pf_cs, kc, vc, g.max_seq, t0, HD};
                 ok = ok && prefill::launch_gemm(c->pf_map_d, cap, ly.wq, ly.wk, ldq, d, T, prefill::PF_STORE, c->pf_qkv, ldq, 0, nullptr,
-                                                nullptr, 0, err, c->n_sms, s, ly.wv, nq, nkv);
+                                                nullptr, 0, err, c->n_sms, s, ly.wv, nq, nkv, &fuse, &heads_done);
             } else {
                 ok = ok && prefill::launch_gemm(c->pf_map_d, cap, ly.wq, nullptr, nq, d, T, prefill::PF_STORE, c->pf_qkv, ldq, 0, nullptr,
                                                 nullptr, 0, err, c->n_sms, s);
@@ -535,7 +537,7 @@ bool prefill_tensor(knnssd_ctx *c, int n) {
                 ok = ok && prefill::launch_gemm(c->pf_map_d, cap, ly.wv, nullptr, nkv, d, T, prefill::PF_STORE, c->pf_qkv, ldq, nq + nkv,
                                                 nullptr, nullptr, 0, err, c->n_sms, s);
             }
-            prefill::rope_kv_rows_kernel<<<T, 256, 0, s>>>(c->pf_qkv, H, Hkv, HD, c->pf_cs, kc, vc, g.max_seq, t0);
+            if (!heads_done) prefill::rope_kv_rows_kernel<<<T, 256, 0, s>>>(c->pf_qkv, H, Hkv, HD, c->pf_cs, kc, vc, g.max_seq, t0);
             prefill::attn_prompt_kernel<HD><<<dim3(H, (T + 63) / 64), 128, prefill::attn_smem_bytes<HD>(), s>>>(
                 c->pf_qkv, H, Hkv, kc, vc, g.max_seq, t0, T, c->pf_aq, c->pf_aq + (size_t)cap * nq);
             ok = ok && prefill::launch_gemm(c->pf_map_q, cap, ly.wo, nullptr, d, nq, T, prefill::PF_ADD, c->pf_x, d, 0, nullptr, nullptr, 0,
@@ -545,7 +547,7 @@ bool prefill_tensor(knnssd_ctx *c, int n) {
                                             c->pf_af + (size_t)cap * F, F, err, c->n_sms, s);
             ok = ok && prefill::launch_gemm(c->pf_map_f, cap, ly.w_down, nullptr, d, F, T, prefill::PF_ADD, c->pf_x, d, 0, nullptr, nullptr,
                                             0, err, c->n_sms, s);
-            c->launches += (nq % prefill::BOX_N == 0 && nkv % prefill::BOX_N == 0) ? 9 : 11;
+            c->launches += ((nq % prefill::BOX_N == 0 && nkv % prefill::BOX_N == 0) ? 9 : 11) - (heads_done ? 1 : 0);
         }
         // pooled numerator: every row's final hidden state (mean pooling) or the last row's
         if (g.pool_mode == 0) {

@@ -44,7 +44,7 @@ constexpr int GEMM_THREADS = 320;                     // warp 0: TMA; warp 1: MM
 constexpr int GEMM_SMEM = STAGES * STAGE_BYTES + 1024 + 128;   // + slack to align the tiles to 1024 bytes + barriers
 constexpr unsigned WAIT_LIMIT = 4000000u;           // polls of one wait (a whole tile takes well under a millisecond)
 
-enum { PF_STORE = 0, PF_ADD = 1, PF_SWIGLU = 2 };
+enum { PF_STORE = 0, PF_ADD = 1, PF_SWIGLU = 2, PF_QKV = 3 };
 
 struct GemmArgs {
     int T;             // live rows
@@ -59,6 +59,12 @@ struct GemmArgs {
     int *err;          // set non-zero if a bounded wait gave up
     int nA, nB;        // STORE over stacked matrices (q, k, v in one launch): units [0, nA) are rows of map tb0,
                        // [nA, nA + nB) rows of tb1, the rest rows of tb2; all multiples of BOX_N.  One matrix: nA = N
+    // PF_QKV (stacked q, k, v; head dimension 128, bn = 256: an epilogue thread holds one head of its token): the q
+    // heads are rotated and stored to y, the k heads rotated, the k and v heads rounded to bf16 into the cache rows
+    // of position pos0 + t
+    const float2 *rope;    // [T][64] (cos, sin) of the rows' positions
+    bf16_t *kc, *vc;       // this layer's K and V cache, [kv head][max_seq][128]
+    int max_seq, pos0;
 };
 
 __device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int x, int y, uint64_t *bar) {
@@ -318,6 +324,39 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap ta, const __grid_constant_
                         for (int i = 0; n0 + c0 + i < g.N; ++i) {
                             ph[i] = (bf16_t)((hi[i >> 1] >> (16 * (i & 1))) & 0xFFFFu);
                             pl[i] = (bf16_t)((lo[i >> 1] >> (16 * (i & 1))) & 0xFFFFu);
+                        }
+                    }
+                }
+            } else if (EPI == PF_QKV) {
+                // acc[j] = unit u0 + j of the stacked q / k / v units: one head of token t
+                const int u0 = n0 + hsel * 128;
+                if (u0 < g.N) {
+                    if (u0 < g.nA + g.nB) {                     // a q or a k head: rotary embedding, pairs (i, i + 64)
+                        const float2 *cs = g.rope + (size_t)t * 64;
+#pragma unroll
+                        for (int i = 0; i < 64; ++i) {
+                            const float2 c = cs[i];
+                            const float a = acc[i], b = acc[64 + i];
+                            acc[i] = a * c.x - b * c.y;
+                            acc[64 + i] = b * c.x + a * c.y;
+                        }
+                    }
+                    if (u0 < g.nA) {
+                        float *yp = g.y + (size_t)t * g.ldy + g.col0 + u0;
+#pragma unroll
+                        for (int i = 0; i < 128; i += 4)
+                            *reinterpret_cast<float4 *>(yp + i) = make_float4(acc[i], acc[i + 1], acc[i + 2], acc[i + 3]);
+                    } else {
+                        const bool is_k = u0 < g.nA + g.nB;
+                        const int kvh = (u0 - g.nA - (is_k ? 0 : g.nB)) >> 7;
+                        bf16_t *dst = (is_k ? g.kc : g.vc) + ((size_t)kvh * g.max_seq + g.pos0 + t) * 128;
+#pragma unroll
+                        for (int i = 0; i < 128; i += 8) {
+                            uint32_t w[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e)
+                                w[e] = pack_bf16(float_to_bf16_rne(acc[i + 2 * e]), float_to_bf16_rne(acc[i + 2 * e + 1]));
+                            *reinterpret_cast<uint4 *>(dst + i) = make_uint4(w[0], w[1], w[2], w[3]);
                         }
                     }
                 }

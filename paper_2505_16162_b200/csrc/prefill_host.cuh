@@ -51,6 +51,7 @@ inline bool gemm_attrs_once() {
         cudaFuncSetAttribute(gemm_split_kernel<PF_STORE>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM) == cudaSuccess &&
         cudaFuncSetAttribute(gemm_split_kernel<PF_ADD>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM) == cudaSuccess &&
         cudaFuncSetAttribute(gemm_split_kernel<PF_SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM) == cudaSuccess &&
+        cudaFuncSetAttribute(gemm_split_kernel<PF_QKV>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM) == cudaSuccess &&
         cudaFuncSetAttribute(gemm_wide_kernel<PF_STORE>, cudaFuncAttributeMaxDynamicSharedMemorySize, WIDE_SMEM) == cudaSuccess &&
         cudaFuncSetAttribute(gemm_wide_kernel<PF_ADD>, cudaFuncAttributeMaxDynamicSharedMemorySize, WIDE_SMEM) == cudaSuccess &&
         cudaFuncSetAttribute(attn_prompt_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_smem_bytes<128>()) == cudaSuccess &&
@@ -87,9 +88,20 @@ inline int pick_bn(int T, int N, int K, bool swiglu, int n_sms) {
 // SwiGLU: W0 = gate, W1 = up) are [N][K] bf16.  STORE with W1 and W2 given: the three matrices (nA, nB and nC rows, all
 // multiples of BOX_N) are stacked along the output units, N = nA + nB + nC, one launch for q, k and v.
 // Returns false if a tensor map could not be made.
+// What the q / k / v launch needs to finish the heads in its epilogue (rotary embedding, K / V rows into the cache).
+struct QkvFuse {
+    const float2 *rope;    // [T][64]
+    bf16_t *kc, *vc;
+    int max_seq, pos0, head_dim;
+};
+
+// `fuse` (stacked q, k, v only): if the head dimension is 128 and the launch takes 256-column tiles, the epilogue does
+// the rotary embedding and writes K / V to the cache itself; *fused says whether it did (otherwise the caller runs
+// rope_kv_rows_kernel on y).
 inline bool launch_gemm(const CUtensorMap &planes, int cap, const void *W0, const void *W1, int N, int K, int T, int epi, float *y,
                         int ldy, int col0, bf16_t *out_hi, bf16_t *out_lo, int ldo, int *err, int n_sms, cudaStream_t s,
-                        const void *W2 = nullptr, int nA = 0, int nB = 0) {
+                        const void *W2 = nullptr, int nA = 0, int nB = 0, const QkvFuse *fuse = nullptr, bool *fused = nullptr) {
+    if (fused) *fused = false;
     if (!gemm_attrs_once()) return false;
     CUtensorMap tb0, tb1, tb2;
     const bool stacked = epi == PF_STORE && W1 && W2;
@@ -104,10 +116,15 @@ inline bool launch_gemm(const CUtensorMap &planes, int cap, const void *W0, cons
         tb2 = tb0;
     }
     const int bn = pick_bn(T, N, K, epi == PF_SWIGLU, n_sms);
-    GemmArgs g{T, K, N, bn, y, ldy, col0, out_hi, out_lo, ldo, err, stacked ? nA : N, stacked ? nB : 0};
+    GemmArgs g{T, K, N, bn, y, ldy, col0, out_hi, out_lo, ldo, err, stacked ? nA : N, stacked ? nB : 0, nullptr, nullptr, nullptr, 0, 0};
+    const bool fuse_heads = stacked && fuse && fuse->head_dim == 128 && bn == 256 && nA % 128 == 0 && nB % 128 == 0 && N % 128 == 0;
+    if (fuse_heads) { g.rope = fuse->rope; g.kc = fuse->kc; g.vc = fuse->vc; g.max_seq = fuse->max_seq; g.pos0 = fuse->pos0; }
     const int per = epi == PF_SWIGLU ? bn / 2 : bn;
     const dim3 grid((T + BM - 1) / BM, (N + per - 1) / per);
-    if (bn == WIDE_BN && epi == PF_STORE) gemm_wide_kernel<PF_STORE><<<grid, GEMM_THREADS, WIDE_SMEM, s>>>(planes, tb0, tb1, tb2, g, cap);
+    if (fuse_heads) {
+        gemm_split_kernel<PF_QKV><<<grid, GEMM_THREADS, GEMM_SMEM, s>>>(planes, tb0, tb1, tb2, g, cap);
+        if (fused) *fused = true;
+    } else if (bn == WIDE_BN && epi == PF_STORE) gemm_wide_kernel<PF_STORE><<<grid, GEMM_THREADS, WIDE_SMEM, s>>>(planes, tb0, tb1, tb2, g, cap);
     else if (bn == WIDE_BN) gemm_wide_kernel<PF_ADD><<<grid, GEMM_THREADS, WIDE_SMEM, s>>>(planes, tb0, tb1, tb2, g, cap);
     else if (epi == PF_STORE) gemm_split_kernel<PF_STORE><<<grid, GEMM_THREADS, GEMM_SMEM, s>>>(planes, tb0, tb1, tb2, g, cap);
     else if (epi == PF_ADD) gemm_split_kernel<PF_ADD><<<grid, GEMM_THREADS, GEMM_SMEM, s>>>(planes, tb0, tb1, tb2, g, cap);
