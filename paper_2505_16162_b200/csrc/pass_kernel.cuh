@@ -343,10 +343,9 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
                                            int warp, int lane, bool defer_merge, int row0, bool all_cached) {
     constexpr int DL = HD / 4;         // dimensions of q / o per lane
     constexpr int NW = HD / 8;         // 32-bit words of a K row per lane
-    constexpr int KS = HD / 16;        // k-steps of Q K^T
     constexpr int VW = HD / 16;        // 32-bit words of a V row per lane
     constexpr int VJ = HD / 8;         // V tiles (8 dimensions each)
-    constexpr int HALF = HD / 2, DPL = HD / 32;
+    constexpr int HALF = HD / 2;
     constexpr int NT = SEGP / 8;       // position tiles per segment
     constexpr int NR = R16 ? 2 : 1;    // pass rows per lane: row0 + g8 and, with R16, row0 + g8 + 8 (rows 8..15 of the MMA operand)
     const int g8 = lane >> 2, t4 = lane & 3;
