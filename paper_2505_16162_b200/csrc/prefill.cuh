@@ -57,6 +57,7 @@ struct GemmArgs {
     bf16_t *out_lo;
     int ldo;
     int *err;          // set non-zero if a bounded wait gave up
+    int tiles_x, tiles_y;   // gemm_split_kernel: row tiles and column tiles of the launch (its CTAs walk tile = ty tiles_x + tx)
     int nA, nB;        // STORE over stacked matrices (q, k, v in one launch): units [0, nA) are rows of map tb0,
                        // [nA, nA + nB) rows of tb1, the rest rows of tb2; all multiples of BOX_N.  One matrix: nA = N
     // PF_QKV (stacked q, k, v; head dimension 128, bn = 256: an epilogue thread holds one head of its token): the q
@@ -164,9 +165,9 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap ta, const __grid_constant_
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_empty + 2);
     volatile int *cta_abort = reinterpret_cast<volatile int *>(tmem_slot + 1);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int t0 = blockIdx.x * BM;
     const int bn = g.bn, per = EPI == PF_SWIGLU ? bn / 2 : bn;      // units of a matrix per tile
-    const int n0 = blockIdx.y * per;
+    // tiles: row tile fastest (tile = ty * tiles_x + tx); this CTA takes tiles blockIdx.x, + gridDim.x, ..
+    const int n_tiles = g.tiles_x * g.tiles_y;
     const int nkb = g.K / BK, nchunks = (nkb + CHUNK_KB - 1) / CHUNK_KB;
     constexpr int EPI_WARPS = GEMM_THREADS / 32 - 2;
 
@@ -189,11 +190,14 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap ta, const __grid_constant_
     if (warp == 0) {
         if (lane == 0) {
             // ---- TMA producer: a stage is refilled once the MMAs that read it have finished ----
-            int armed = 0;
+            int armed = 0;                   // k-blocks armed so far, over all of this CTA's tiles: stage and phase follow it
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+            const int t0 = (tile % g.tiles_x) * BM, n0 = (tile / g.tiles_x) * per;
             for (int kb = 0; kb < nkb; ++kb) {
-                const int s = kb % STAGES;
-                const uint32_t ph = (uint32_t)(kb / STAGES) & 1u;
-                if (!pf_wait(&empty[s], ph ^ 1u, cta_abort, g.err, 21)) break;
+                const int s = armed % STAGES;
+                const uint32_t ph = (uint32_t)(armed / STAGES) & 1u;
+                if (!pf_wait(&empty[s], ph ^ 1u, cta_abort, g.err, 21)) { ok = false; break; }
                 unsigned char *st = smem + s * STAGE_BYTES;
                 stream::mbar_expect_tx(&full[s], 2 * A_BYTES + bn * BK * 2);
                 tma_load_2d(st, &ta, kb * BK, t0, &full[s]);
@@ -209,7 +213,8 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap ta, const __grid_constant_
                     }
                     tma_load_2d(st + 2 * A_BYTES + r * BK * 2, wm, kb * BK, wrow, &full[s]);
                 }
-                armed = kb + 1;
+                ++armed;
+            }
             }
             if (*cta_abort) {
                 // copies in flight land in this CTA's shared memory: let them finish before the CTA goes away
@@ -224,16 +229,18 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap ta, const __grid_constant_
             // ---- MMA issue: chunk c goes to accumulator c & 1; per stage 4 k-steps of 16 columns, hi and lo term ----
             bool ok = true;
             const uint32_t idesc = umma_idesc(bn);
-            for (int c = 0; c < nchunks && ok; ++c) {
-                const int b = c & 1;
-                ok = pf_wait(&acc_empty[b], ((uint32_t)(c >> 1) & 1u) ^ 1u, cta_abort, g.err, 24);
+            int kbg = 0, cg = 0;             // k-blocks and chunks issued so far, over all of this CTA's tiles
+            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x)
+            for (int c = 0; c < nchunks && ok; ++c, ++cg) {
+                const int b = cg & 1;
+                ok = pf_wait(&acc_empty[b], ((uint32_t)(cg >> 1) & 1u) ^ 1u, cta_abort, g.err, 24);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t acc_addr = tmem + (uint32_t)(b * BN_MAX);
                 const int kb1 = min(nkb, (c + 1) * CHUNK_KB);
-                for (int kb = c * CHUNK_KB; kb < kb1 && ok; ++kb) {
-                    const int s = kb % STAGES;
-                    const uint32_t ph = (uint32_t)(kb / STAGES) & 1u;
+                for (int kb = c * CHUNK_KB; kb < kb1 && ok; ++kb, ++kbg) {
+                    const int s = kbg % STAGES;
+                    const uint32_t ph = (uint32_t)(kbg / STAGES) & 1u;
                     ok = pf_wait(&full[s], ph, cta_abort, g.err, 22);
                     if (!ok) break;
                     tc_fence_after();
@@ -257,7 +264,6 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap ta, const __grid_constant_
         //      store / add: columns [hsel bn / 2, + bn / 2) in groups of 32; SwiGLU: acc[0 .. 63] gate columns
         //      [hsel bn / 4, + bn / 4), acc[64 .. 127] the up columns of the same units ----
         const int q = warp & 3, hsel = (warp - 2) >> 2;
-        const int t = t0 + 32 * q + lane;
         const uint32_t trow = tmem + ((uint32_t)(32 * q) << 16);
         const int half = bn / 2, qtr = bn / 4;
         // tile column of register group gi (32 columns), or -1 if the group is not in use
@@ -269,14 +275,18 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap ta, const __grid_constant_
             }
             return 32 * gi < half ? hsel * half + 32 * gi : -1;
         };
+        bool ok = true;
+        int cg = 0;                          // chunks taken so far, over all of this CTA's tiles
+        for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        const int t0 = (tile % g.tiles_x) * BM, n0 = (tile / g.tiles_x) * per;
+        const int t = t0 + 32 * q + lane;
         float acc[128];
 #pragma unroll
         for (int i = 0; i < 128; ++i) acc[i] = 0.f;
-        bool ok = true;
-        for (int c = 0; c < nchunks && ok; ++c) {
-            const int b = c & 1;
+        for (int c = 0; c < nchunks && ok; ++c, ++cg) {
+            const int b = cg & 1;
             // the loads from tensor memory are warp-wide: the warp goes on only if all of its threads saw the accumulator
-            ok = __all_sync(0xffffffffu, pf_wait(&acc_full[b], (uint32_t)(c >> 1) & 1u, cta_abort, g.err, 23) && !*cta_abort);
+            ok = __all_sync(0xffffffffu, pf_wait(&acc_full[b], (uint32_t)(cg >> 1) & 1u, cta_abort, g.err, 23) && !*cta_abort);
             if (!ok) break;
             tc_fence_after();
 #pragma unroll
@@ -384,6 +394,7 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap ta, const __grid_constant_
                 }
             }
         }
+        }                                    // next tile: its first chunks are already accumulating in tensor memory
     }
     tc_fence_before();
     __syncthreads();

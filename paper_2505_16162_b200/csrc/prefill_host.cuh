@@ -60,13 +60,14 @@ inline bool gemm_attrs_once() {
     return ok;
 }
 
-// Accumulator columns per tile.  All CTAs of a launch run at once on n_sms SMs, round after round.  The main loop is
-// bound by shared-memory traffic (measured: 0.50 / 0.69 / 0.70 us per k-block at 128 / 192 / 256 columns, 1.0 - 1.3 at
-// 2 x 160): per k-block TMA writes the two activation planes (32 KB) and bn / 8 KB of weights, and the tensor core reads
-// the planes once and the weights twice (hi and lo products), 64 + 3 bn / 8 KB in all; the 320-column tiles of
-// gemm_wide_kernel (returned as WIDE_BN; store and add epilogues only) read the planes once per half and are charged
-// 15 % on top, as measured.  A round also costs a fixed ~10 us (tensor-memory allocation, first copies, epilogue),
-// 1960 KB at that rate.  The width with the lowest rounds x (traffic x k-blocks + fixed) wins (ties: the wider tile).
+// Accumulator columns per tile.  gemm_split_kernel runs one CTA per SM that walks the tiles round after round;
+// gemm_wide_kernel one CTA per tile.  The main loop is bound by shared-memory traffic (measured per k-block and CTA:
+// 0.57 / 0.69 / 0.81 us at 128 / 192 / 256 columns, 1.1 - 1.4 at 2 x 160): per k-block TMA writes the two activation
+// planes (32 KB) and bn / 8 KB of weights, and the tensor core reads the planes once and the weights twice (hi and lo
+// products), 64 + 3 bn / 8 KB in all; the 320-column tiles of gemm_wide_kernel (returned as WIDE_BN; store and add
+// epilogues only) read the planes once per half and are charged 15 % on top, as measured, plus ~10 us per round for the
+// prologue and epilogue that nothing overlaps there (1960 KB at that rate; the walking kernel pays ~3 us once).  The
+// width with the lowest rounds x traffic x k-blocks + fixed cost wins (ties: the wider tile).
 inline int pick_bn(int T, int N, int K, bool swiglu, int n_sms) {
     const int row_tiles = (T + BM - 1) / BM;
     const long nkb = K / BK;
@@ -78,7 +79,8 @@ inline int pick_bn(int T, int N, int K, bool swiglu, int n_sms) {
         const int per = swiglu ? bn / 2 : bn;
         const long ctas = (long)row_tiles * ((N + per - 1) / per);
         const long traffic = bn == WIDE_BN ? 248 : 64 + 3 * bn / 8;
-        const long cost = ((ctas + n_sms - 1) / n_sms) * (traffic * nkb + 1960);
+        const long rounds = (ctas + n_sms - 1) / n_sms;
+        const long cost = bn == WIDE_BN ? rounds * (traffic * nkb + 1960) : rounds * traffic * nkb + 600;
         if (!best || cost <= best_cost) { best = bn; best_cost = cost; }
     }
     return best;
@@ -116,19 +118,23 @@ inline bool launch_gemm(const CUtensorMap &planes, int cap, const void *W0, cons
         tb2 = tb0;
     }
     const int bn = pick_bn(T, N, K, epi == PF_SWIGLU, n_sms);
-    GemmArgs g{T, K, N, bn, y, ldy, col0, out_hi, out_lo, ldo, err, stacked ? nA : N, stacked ? nB : 0, nullptr, nullptr, nullptr, 0, 0};
-    const bool fuse_heads = stacked && fuse && fuse->head_dim == 128 && bn == 256 && nA % 128 == 0 && nB % 128 == 0 && N % 128 == 0;
-    if (fuse_heads) { g.rope = fuse->rope; g.kc = fuse->kc; g.vc = fuse->vc; g.max_seq = fuse->max_seq; g.pos0 = fuse->pos0; }
     const int per = epi == PF_SWIGLU ? bn / 2 : bn;
     const dim3 grid((T + BM - 1) / BM, (N + per - 1) / per);
+    GemmArgs g{T, K, N, bn, y, ldy, col0, out_hi, out_lo, ldo, err, (int)grid.x, (int)grid.y, stacked ? nA : N, stacked ? nB : 0,
+               nullptr, nullptr, nullptr, 0, 0};
+    // gemm_split_kernel: one CTA per SM walks the tiles (the epilogue of a tile runs under the next tile's products)
+    const int n_tiles = (int)(grid.x * grid.y);
+    const dim3 pgrid(n_tiles < n_sms ? n_tiles : n_sms);
+    const bool fuse_heads = stacked && fuse && fuse->head_dim == 128 && bn == 256 && nA % 128 == 0 && nB % 128 == 0 && N % 128 == 0;
+    if (fuse_heads) { g.rope = fuse->rope; g.kc = fuse->kc; g.vc = fuse->vc; g.max_seq = fuse->max_seq; g.pos0 = fuse->pos0; }
     if (fuse_heads) {
-        gemm_split_kernel<PF_QKV><<<grid, GEMM_THREADS, GEMM_SMEM, s>>>(planes, tb0, tb1, tb2, g, cap);
+        gemm_split_kernel<PF_QKV><<<pgrid, GEMM_THREADS, GEMM_SMEM, s>>>(planes, tb0, tb1, tb2, g, cap);
         if (fused) *fused = true;
     } else if (bn == WIDE_BN && epi == PF_STORE) gemm_wide_kernel<PF_STORE><<<grid, GEMM_THREADS, WIDE_SMEM, s>>>(planes, tb0, tb1, tb2, g, cap);
     else if (bn == WIDE_BN) gemm_wide_kernel<PF_ADD><<<grid, GEMM_THREADS, WIDE_SMEM, s>>>(planes, tb0, tb1, tb2, g, cap);
-    else if (epi == PF_STORE) gemm_split_kernel<PF_STORE><<<grid, GEMM_THREADS, GEMM_SMEM, s>>>(planes, tb0, tb1, tb2, g, cap);
-    else if (epi == PF_ADD) gemm_split_kernel<PF_ADD><<<grid, GEMM_THREADS, GEMM_SMEM, s>>>(planes, tb0, tb1, tb2, g, cap);
-    else gemm_split_kernel<PF_SWIGLU><<<grid, GEMM_THREADS, GEMM_SMEM, s>>>(planes, tb0, tb1, tb2, g, cap);
+    else if (epi == PF_STORE) gemm_split_kernel<PF_STORE><<<pgrid, GEMM_THREADS, GEMM_SMEM, s>>>(planes, tb0, tb1, tb2, g, cap);
+    else if (epi == PF_ADD) gemm_split_kernel<PF_ADD><<<pgrid, GEMM_THREADS, GEMM_SMEM, s>>>(planes, tb0, tb1, tb2, g, cap);
+    else gemm_split_kernel<PF_SWIGLU><<<pgrid, GEMM_THREADS, GEMM_SMEM, s>>>(planes, tb0, tb1, tb2, g, cap);
     return true;
 }
 
