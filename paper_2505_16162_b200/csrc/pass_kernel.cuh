@@ -473,7 +473,7 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
             const bf16_t *src = p < Pc ? kbase + (size_t)p * HD + DL * t4 : stash_k + (p - P0) * HD + DL * t4;
 #pragma unroll
             for (int q = 0; q < NW / 4; ++q)
-                dst[q] = p < p_end ? *reinterpret_cast<const uint4 *>(src + 8 * q) : make_uint4(0u, 0u, 0u, 0u);
+                dst[q] = p < p_end ? (p < Pc ? __ldcs(reinterpret_cast<const uint4 *>(src + 8 * q)) : *reinterpret_cast<const uint4 *>(src + 8 * q)) : make_uint4(0u, 0u, 0u, 0u);
         };
         float sc[NT][2 * NR];                                // scores of (row g8, positions 8*nt + 2*t4 + {0, 1}); R16: [2], [3] = row g8 + 8
         {
@@ -515,7 +515,7 @@ __device__ __forceinline__ void attn_phase(const Model &md, const Op &op, const 
                 if (VW >= 4) {
 #pragma unroll
                     for (int q = 0; q < VW / 4; ++q)
-                        dst[rr][q] = p < p_end ? *reinterpret_cast<const uint4 *>(src + 8 * q) : make_uint4(0u, 0u, 0u, 0u);
+                        dst[rr][q] = p < p_end ? (p < Pc ? __ldcs(reinterpret_cast<const uint4 *>(src + 8 * q)) : *reinterpret_cast<const uint4 *>(src + 8 * q)) : make_uint4(0u, 0u, 0u, 0u);
                 } else {
                     const uint2 v = p < p_end ? *reinterpret_cast<const uint2 *>(src) : make_uint2(0u, 0u);
                     dst[rr][0] = make_uint4(v.x, v.y, 0u, 0u);
