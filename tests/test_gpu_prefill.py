@@ -50,9 +50,12 @@ GEMM_CASES = [(512, 256, 128), (1000, 320, 77), (136, 64, 5), (640, 1024, 300), 
               # tile widths other than 128 columns (the launch picks the width with the fewest column-rounds on the
               # GPU's SMs): 192, 320 and 256 on a 148-SM part
               (5120, 256, 520), (5120, 256, 900), (4608, 256, 1024),
-              # 320-column tiles on three rotating accumulators: several staggered chunks per half with a short last
-              # one; a ragged last tile (136 of 320 columns, a weight box partly past the end)
-              (5120, 2176, 900), (4936, 512, 1000)]
+              # more tiles than SMs (a CTA walks several tiles); a ragged last tile
+              (5120, 2176, 900), (4936, 512, 1000),
+              # 320-column tiles on three rotating accumulators (picked where they save a round and the input is long
+              # enough to pay for their one-tile CTAs): staggered chunks with short last ones (69 k-blocks), a ragged
+              # last tile (136 of 320 columns, a weight box partly past the end)
+              (4936, 4416, 900)]
 
 
 @pytest.mark.parametrize("n_out,n_in,T", GEMM_CASES)
@@ -63,7 +66,7 @@ def test_gemm_store_matches_oracle(kb, n_out, n_in, T):
     assert np.abs(got - want).max() < _tol(n_in, want)
 
 
-@pytest.mark.parametrize("n_out,n_in,T", [(1000, 320, 77), (5120, 5120, 260)])
+@pytest.mark.parametrize("n_out,n_in,T", [(1000, 320, 77), (5120, 5120, 260), (4936, 4416, 900)])
 def test_gemm_add_matches_oracle(kb, n_out, n_in, T):
     W, x = _inputs(n_out, n_in, T)
     y0 = si.normal_f32(9, 79, torch.arange(T * n_out), 1.0).view(T, n_out).contiguous()
