@@ -89,6 +89,7 @@ struct knnssd_ctx {
     int pf_cap = 0;                                          // rows per chunk, a multiple of 128
     float *pf_x = nullptr, *pf_qkv = nullptr;                // residual stream [cap][d]; q, k, v [cap][nq + 2 nkv]
     float2 *pf_cs = nullptr;                                 // rotary (cos, sin) of the chunk's rows [cap][hd / 2]
+    float *pf_rinv = nullptr;                                // RMSNorm scale of the chunk's rows [cap]
     bf16_t *pf_ad = nullptr, *pf_aq = nullptr, *pf_af = nullptr;   // hi / lo planes [2][cap][d], [2][cap][nq], [2][cap][d_ff]
     CUtensorMap pf_map_d{}, pf_map_q{}, pf_map_f{};
 
@@ -477,7 +478,7 @@ void free_all(knnssd_ctx *c) {
                     c->anchor_inv_norm, c->cosines, c->amax_v, c->part_ml, c->rope_cs, c->pool_sum, c->inv_freq, c->chain,
                     c->target, c->prompt, c->out_tokens, c->accept_log, c->amax_i, c->flag, c->knn_out, c->state,
                     c->ops_full, c->ops_draft, c->bar, c->gabort, c->attn_cnt, c->amax_cnt, c->mpart_o, c->mamax_v, c->mpart_ml,
-                    c->mamax_i, c->trace, c->xs_x, c->xs_attn, c->xs_act, c->ssp, c->pf_x, c->pf_qkv, c->pf_ad, c->pf_aq, c->pf_af, c->pf_cs,
+                    c->mamax_i, c->trace, c->xs_x, c->xs_attn, c->xs_act, c->ssp, c->pf_x, c->pf_qkv, c->pf_ad, c->pf_aq, c->pf_af, c->pf_cs, c->pf_rinv,
                     c->samp_p, c->samp_q, c->samp_res};
     for (void *p : ptrs)
         if (p) cudaFree(p);
@@ -522,29 +523,29 @@ bool prefill_tensor(knnssd_ctx *c, int n) {
             const Layer &ly = c->layers[l];
             bf16_t *kc = reinterpret_cast<bf16_t *>(c->kcache) + (size_t)l * layer_stride;
             bf16_t *vc = reinterpret_cast<bf16_t *>(c->vcache) + (size_t)l * layer_stride;
-            prefill::norm_split_kernel<<<T, 256, 0, s>>>(c->pf_x, d, ly.attn_norm, g.rms_eps, c->pf_ad, c->pf_ad + (size_t)cap * d);
+            prefill::norm_split_kernel<<<T, 256, 0, s>>>(c->pf_x, d, ly.attn_norm, g.rms_eps, c->pf_ad, c->pf_ad + (size_t)cap * d, c->pf_rinv);
             bool heads_done = false;     // rotary embedding and K / V rows done by the q / k / v launch's epilogue
             if (nq % prefill::BOX_N == 0 && nkv % prefill::BOX_N == 0) {
                 // q, k and v in one launch over the stacked units (their columns of the projection buffer are adjacent)
                 const prefill::QkvFuse fuse{c->pf_cs, kc, vc, g.max_seq, t0, HD};
                 ok = ok && prefill::launch_gemm(c->pf_map_d, cap, ly.wq, ly.wk, ldq, d, T, prefill::PF_STORE, c->pf_qkv, ldq, 0, nullptr,
-                                                nullptr, 0, err, c->n_sms, s, ly.wv, nq, nkv, &fuse, &heads_done);
+                                                nullptr, 0, err, c->n_sms, s, ly.wv, nq, nkv, &fuse, &heads_done, c->pf_rinv);
             } else {
                 ok = ok && prefill::launch_gemm(c->pf_map_d, cap, ly.wq, nullptr, nq, d, T, prefill::PF_STORE, c->pf_qkv, ldq, 0, nullptr,
-                                                nullptr, 0, err, c->n_sms, s);
+                                                nullptr, 0, err, c->n_sms, s, nullptr, 0, 0, nullptr, nullptr, c->pf_rinv);
                 ok = ok && prefill::launch_gemm(c->pf_map_d, cap, ly.wk, nullptr, nkv, d, T, prefill::PF_STORE, c->pf_qkv, ldq, nq, nullptr,
-                                                nullptr, 0, err, c->n_sms, s);
+                                                nullptr, 0, err, c->n_sms, s, nullptr, 0, 0, nullptr, nullptr, c->pf_rinv);
                 ok = ok && prefill::launch_gemm(c->pf_map_d, cap, ly.wv, nullptr, nkv, d, T, prefill::PF_STORE, c->pf_qkv, ldq, nq + nkv,
-                                                nullptr, nullptr, 0, err, c->n_sms, s);
+                                                nullptr, nullptr, 0, err, c->n_sms, s, nullptr, 0, 0, nullptr, nullptr, c->pf_rinv);
             }
             if (!heads_done) prefill::rope_kv_rows_kernel<<<T, 256, 0, s>>>(c->pf_qkv, H, Hkv, HD, c->pf_cs, kc, vc, g.max_seq, t0);
             prefill::attn_prompt_kernel<HD><<<dim3(H, (T + 63) / 64), 128, prefill::attn_smem_bytes<HD>(), s>>>(
                 c->pf_qkv, H, Hkv, kc, vc, g.max_seq, t0, T, c->pf_aq, c->pf_aq + (size_t)cap * nq);
             ok = ok && prefill::launch_gemm(c->pf_map_q, cap, ly.wo, nullptr, d, nq, T, prefill::PF_ADD, c->pf_x, d, 0, nullptr, nullptr, 0,
                                             err, c->n_sms, s);
-            prefill::norm_split_kernel<<<T, 256, 0, s>>>(c->pf_x, d, ly.mlp_norm, g.rms_eps, c->pf_ad, c->pf_ad + (size_t)cap * d);
+            prefill::norm_split_kernel<<<T, 256, 0, s>>>(c->pf_x, d, ly.mlp_norm, g.rms_eps, c->pf_ad, c->pf_ad + (size_t)cap * d, c->pf_rinv);
             ok = ok && prefill::launch_gemm(c->pf_map_d, cap, ly.w_gate, ly.w_up, F, d, T, prefill::PF_SWIGLU, nullptr, 0, 0, c->pf_af,
-                                            c->pf_af + (size_t)cap * F, F, err, c->n_sms, s);
+                                            c->pf_af + (size_t)cap * F, F, err, c->n_sms, s, nullptr, 0, 0, nullptr, nullptr, c->pf_rinv);
             ok = ok && prefill::launch_gemm(c->pf_map_f, cap, ly.w_down, nullptr, d, F, T, prefill::PF_ADD, c->pf_x, d, 0, nullptr, nullptr,
                                             0, err, c->n_sms, s);
             c->launches += ((nq % prefill::BOX_N == 0 && nkv % prefill::BOX_N == 0) ? 9 : 11) - (heads_done ? 1 : 0);
@@ -796,6 +797,7 @@ knnssd_status knnssd_init(const knnssd_config *cfg, const knnssd_weights *w, con
             ok3 &= dev_alloc(&c->pf_x, cap * d) == cudaSuccess;
             ok3 &= dev_alloc(&c->pf_qkv, cap * (nq + 2 * nkv)) == cudaSuccess;
             ok3 &= dev_alloc(&c->pf_cs, cap * (hd / 2)) == cudaSuccess;
+            ok3 &= dev_alloc(&c->pf_rinv, cap) == cudaSuccess;
             ok3 &= dev_alloc(&c->pf_ad, 2 * cap * d) == cudaSuccess;
             ok3 &= dev_alloc(&c->pf_aq, 2 * cap * nq) == cudaSuccess;
             ok3 &= dev_alloc(&c->pf_af, 2 * cap * g.d_ff) == cudaSuccess;

@@ -63,6 +63,8 @@ struct GemmArgs {
     // PF_QKV (stacked q, k, v; head dimension 128, bn = 256: an epilogue thread holds one head of its token): the q
     // heads are rotated and stored to y, the k heads rotated, the k and v heads rounded to bf16 into the cache rows
     // of position pos0 + t
+    const float *row_scale;   // if given: every sum of row t is multiplied by row_scale[t] before the epilogue (the RMSNorm
+                              // scale of the row whose gain-weighted, un-normalised values the planes hold)
     const float2 *rope;    // [T][64] (cos, sin) of the rows' positions
     bf16_t *kc, *vc;       // this layer's K and V cache, [kv head][max_seq][128]
     int max_seq, pos0;
@@ -302,6 +304,11 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap ta, const __grid_constant_
             tc_fence_before();
             __syncwarp();
             if (lane == 0) stream::mbar_arrive(&acc_empty[b]);
+        }
+        if (ok && t < g.T && g.row_scale) {
+            const float rs = g.row_scale[t];
+#pragma unroll
+            for (int i = 0; i < 128; ++i) acc[i] *= rs;
         }
         if (ok && t < g.T) {
             if (EPI == PF_SWIGLU) {
@@ -581,6 +588,11 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap ta, const __grid_constant__
             __syncwarp();
             if (lane == 0) stream::mbar_arrive(&acc_empty[buf]);
         }
+        if (ok && t < g.T && g.row_scale) {
+            const float rs = g.row_scale[t];
+#pragma unroll
+            for (int i = 0; i < WIDE_HALF; ++i) acc[i] *= rs;
+        }
         if (ok && t < g.T) {
 #pragma unroll
             for (int gi = 0; gi < WIDE_HALF / 16; ++gi) {
@@ -624,9 +636,12 @@ __global__ void embed_rows_kernel(const bf16_t *__restrict__ table, const int *_
     for (int i = threadIdx.x; i < d; i += blockDim.x) xr[i] = bf16_bits_to_float(row[i]);
 }
 
-// RMSNorm of row t (gain g, epsilon eps), written as hi = bf16(v) and lo = bf16(v - hi).  grid = T, 256 threads.
+// RMSNorm of row t (gain g, epsilon eps) for the contraction that follows: the planes hold v = x g WITHOUT the row's
+// scale, hi = bf16(v) and lo = bf16(v - hi), and rinv[t] = 1 / sqrt(mean(x^2) + eps) goes to the contraction's epilogue
+// (a linear map commutes with a per-row scale).  Same operands as the decode passes use: values that are exact in two
+// bf16 terms - embedding rows with unit gains - stay exact.  grid = T, 256 threads.
 __global__ void __launch_bounds__(256) norm_split_kernel(const float *__restrict__ x, int d, const float *__restrict__ gain, float eps,
-                                                         bf16_t *__restrict__ hi, bf16_t *__restrict__ lo) {
+                                                         bf16_t *__restrict__ hi, bf16_t *__restrict__ lo, float *__restrict__ rinv_out) {
     __shared__ float part[8];
     const float *xr = x + (size_t)blockIdx.x * d;
     float ss = 0.f;
@@ -641,11 +656,12 @@ __global__ void __launch_bounds__(256) norm_split_kernel(const float *__restrict
 #pragma unroll
     for (int w = 0; w < 8; ++w) tot += part[w];
     const float rinv = 1.0f / sqrtf(tot / (float)d + eps);
+    if (threadIdx.x == 0) rinv_out[blockIdx.x] = rinv;
     bf16_t *hr = hi + (size_t)blockIdx.x * d, *lr = lo + (size_t)blockIdx.x * d;
     for (int i = threadIdx.x * 4; i < d; i += 1024) {
         const float4 v = *reinterpret_cast<const float4 *>(xr + i);
         const float4 g = *reinterpret_cast<const float4 *>(gain + i);
-        const float a[4] = {v.x * rinv * g.x, v.y * rinv * g.y, v.z * rinv * g.z, v.w * rinv * g.w};
+        const float a[4] = {v.x * g.x, v.y * g.y, v.z * g.z, v.w * g.w};
         uint32_t h[4], l[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) {

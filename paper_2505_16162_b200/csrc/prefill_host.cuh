@@ -102,7 +102,8 @@ struct QkvFuse {
 // rope_kv_rows_kernel on y).
 inline bool launch_gemm(const CUtensorMap &planes, int cap, const void *W0, const void *W1, int N, int K, int T, int epi, float *y,
                         int ldy, int col0, bf16_t *out_hi, bf16_t *out_lo, int ldo, int *err, int n_sms, cudaStream_t s,
-                        const void *W2 = nullptr, int nA = 0, int nB = 0, const QkvFuse *fuse = nullptr, bool *fused = nullptr) {
+                        const void *W2 = nullptr, int nA = 0, int nB = 0, const QkvFuse *fuse = nullptr, bool *fused = nullptr,
+                        const float *row_scale = nullptr) {
     if (fused) *fused = false;
     if (!gemm_attrs_once()) return false;
     CUtensorMap tb0, tb1, tb2;
@@ -121,7 +122,7 @@ inline bool launch_gemm(const CUtensorMap &planes, int cap, const void *W0, cons
     const int per = epi == PF_SWIGLU ? bn / 2 : bn;
     const dim3 grid((T + BM - 1) / BM, (N + per - 1) / per);
     GemmArgs g{T, K, N, bn, y, ldy, col0, out_hi, out_lo, ldo, err, (int)grid.x, (int)grid.y, stacked ? nA : N, stacked ? nB : 0,
-               nullptr, nullptr, nullptr, 0, 0};
+               row_scale, nullptr, nullptr, nullptr, 0, 0};
     // gemm_split_kernel: one CTA per SM walks the tiles (the epilogue of a tile runs under the next tile's products)
     const int n_tiles = (int)(grid.x * grid.y);
     const dim3 pgrid(n_tiles < n_sms ? n_tiles : n_sms);
