@@ -12,8 +12,8 @@
 // NP > 0 (the paired form; NP = 1: passes of up to 4 rows - every draft step; NP = 3: passes of 9..12 rows): the rows
 // are taken four at a time and the two bf16 terms of a row sit in neighbouring columns of ONE 8-column operand
 // (column 2 r = hi term of row 4 b + r, 2 r + 1 = its lo term), so a weight fragment takes one MMA per four rows
-// instead of two per eight: 1 instead of 2 for up to 4 rows, 3 instead of 4 for 9..12.  The tensor pipe is what bounds the consumers' rate at these row counts, and a consumer that is
-// faster than the HBM stream drains the ring after a barrier and lets the producer run ahead again.  An output is
+// instead of two per eight: 1 instead of 2 for up to 4 rows, 3 instead of 4 for 9..12.  A consumer that is faster
+// than the HBM stream drains the ring after a barrier and lets the producer run ahead again.  An output is
 // still (sum of the lo products) + (sum of the hi products), each sum accumulated over the same k-steps in the same
 // order as in the unpaired form: the numbers do not depend on which form computed them.
 //
