@@ -239,8 +239,8 @@ def _run(shape_name, mask, k, max_new, prompt_len=12, seed=0, damp=None, max_seq
     return shape, spec, plain, first, first2
 
 
-@pytest.mark.parametrize("mask_kind,k", [(m, k) for m in ("seeded", "all_on", "damped") for k in (1, 2, 4, 8)]
-                         + [("all_off", 1), ("all_off", 8), ("attn_only", 2), ("attn_only", 8)])
+@pytest.mark.parametrize("k", [1, 2, 4, 8])
+@pytest.mark.parametrize("mask_kind", ["seeded", "all_on", "all_off", "attn_only", "damped"])
 def test_speculative_output_is_plain_greedy_output(k, mask_kind):
     """Losslessness (Sec. 1, Sec. 3.1, Sec. 7): whatever the mask and k, the tokens are those
     of plain greedy decoding with the full model."""
@@ -257,7 +257,7 @@ def test_speculative_output_is_plain_greedy_output(k, mask_kind):
     else:
         mask = si.skip_mask(0, 2 * L, 3)
         damp = {int(j): 0.02 for j in np.nonzero(mask)[0]}
-    max_new = 19
+    max_new = 23
     shape, spec, plain, f1, f2 = _run("tiny", mask, k, max_new, damp=damp)
     assert f1 == f2
     assert np.array_equal(spec["tokens"], plain)
@@ -282,7 +282,7 @@ def test_speculative_output_is_plain_greedy_output(k, mask_kind):
 
 
 def test_last_round_never_overshoots():
-    for max_new in (1, 2, 6, 7):
+    for max_new in (1, 2, 3, 6, 7):
         _, spec, plain, _, _ = _run("tiny", np.zeros(8, np.uint8), 4, max_new)
         assert len(spec["tokens"]) == max_new and np.array_equal(spec["tokens"], plain)
 

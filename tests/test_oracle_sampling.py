@@ -127,9 +127,9 @@ def test_sampled_loop_is_the_greedy_loop_as_temperature_goes_to_zero():
     for k in (0, 2, 4):
         om = oracle.OracleModel(shape, w, 96)
         _, first, _ = om.prefill(prompt)
-        want = om.generate(first, 14, k, mask)
+        want = om.generate(first, 20, k, mask)
         om2 = oracle.OracleModel(shape, w, 96)
         om2.prefill(prompt)
-        got = osamp.generate_sampled(om2, first, 14, k, mask, 1e-7, 0.85, si.uniforms(k, 3, 13 * (2 * k + 1)))
+        got = osamp.generate_sampled(om2, first, 20, k, mask, 1e-7, 0.85, si.uniforms(k, 3, 19 * (2 * k + 1)))
         assert np.array_equal(got["tokens"], want["tokens"]) and np.array_equal(got["accepts"], want["accepts"])
-        assert len(got["tokens"]) == 14
+        assert len(got["tokens"]) == 20
