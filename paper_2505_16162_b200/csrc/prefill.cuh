@@ -644,23 +644,13 @@ __global__ void __launch_bounds__(256) norm_split_kernel(const float *__restrict
                                                          bf16_t *__restrict__ hi, bf16_t *__restrict__ lo, float *__restrict__ rinv_out) {
     __shared__ float part[8];
     const float *xr = x + (size_t)blockIdx.x * d;
-    float ss = 0.f;
-    for (int i = threadIdx.x * 4; i < d; i += 1024) {
-        const float4 v = *reinterpret_cast<const float4 *>(xr + i);
-        ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
-    }
-    ss = warp_sum(ss);
-    if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = ss;
-    __syncthreads();
-    float tot = 0.f;
-#pragma unroll
-    for (int w = 0; w < 8; ++w) tot += part[w];
-    const float rinv = 1.0f / sqrtf(tot / (float)d + eps);
-    if (threadIdx.x == 0) rinv_out[blockIdx.x] = rinv;
     bf16_t *hr = hi + (size_t)blockIdx.x * d, *lr = lo + (size_t)blockIdx.x * d;
+    float ss = 0.f;
+    // one walk over the row: the planes do not depend on the row's scale
     for (int i = threadIdx.x * 4; i < d; i += 1024) {
         const float4 v = *reinterpret_cast<const float4 *>(xr + i);
         const float4 g = *reinterpret_cast<const float4 *>(gain + i);
+        ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
         const float a[4] = {v.x * g.x, v.y * g.y, v.z * g.z, v.w * g.w};
         uint32_t h[4], l[4];
 #pragma unroll
@@ -670,6 +660,15 @@ __global__ void __launch_bounds__(256) norm_split_kernel(const float *__restrict
         }
         *reinterpret_cast<uint2 *>(hr + i) = make_uint2(pack_bf16(h[0], h[1]), pack_bf16(h[2], h[3]));
         *reinterpret_cast<uint2 *>(lr + i) = make_uint2(pack_bf16(l[0], l[1]), pack_bf16(l[2], l[3]));
+    }
+    ss = warp_sum(ss);
+    if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float tot = 0.f;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) tot += part[w];
+        rinv_out[blockIdx.x] = 1.0f / sqrtf(tot / (float)d + eps);
     }
 }
 
